@@ -1,0 +1,296 @@
+#!/usr/bin/env python
+"""Benchmark of the Pacer hot path on B200.
+
+One "step" is one pass of the whole hot path over one batch of synthetic input:
+prefill of a seeded random prompt, then the draft / pre-verify / verify / accept
+loop until max_new tokens exist.  The headline value is generated tokens per
+second of the decode loop at batch 1, timed on the device with CUDA events
+(prefill excluded, inputs resident in HBM).  Prints ONE JSON line.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config NAME] [--impl reference]
+
+The path does not shard (one sequence is a strict chain): with --gpus N > 1 each
+rank runs an independent replica and the value is the sum ("replicas only").
+--impl reference times the CPU oracle on the host cores instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2602_01274_b200 import synth  # noqa: E402
+
+METRIC = "generated tokens/s at batch 1 (device-timed) + HBM GB/s fraction of peak in verify"
+UNIT = "tokens/s"
+PACER_T0 = 0.5      # threshold of the headline "Pacer" row (the only value that varies the window
+                    # with an untrained pre-verification layer)
+
+
+def _peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except Exception:
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def verify_bytes(cfg: synth.PairConfig, ctx_len: int, rows: int) -> float:
+    """Algorithmic bytes of one target verify forward: weights once, live KV once, new KV written."""
+    t = cfg.target
+    return t.streamed_weight_bytes() + t.kv_bytes_per_token() * (ctx_len + rows)
+
+
+def oracle_sample(cfg: synth.PairConfig, pair_cpu, prompt, n_prompt_s, max_new_s, t0):
+    """Times the CPU oracle, as it stands, on a bounded sample of the workload:
+    the first n_prompt_s prompt tokens and max_new_s new tokens of Algorithm 1."""
+    from oracle import pacer_oracle as orc
+    T = orc.OracleModel(cfg.target, pair_cpu["target"], pair_cpu["succ_T"], cfg.succ_bias)
+    D = orc.OracleModel(cfg.draft, pair_cpu["draft"], pair_cpu["succ_D"], cfg.succ_bias)
+    B = orc.OracleModel(synth.preverify_shape(cfg.draft), pair_cpu["preverify"])
+    o = orc.Pacer(T, D, B, n_prompt_s + max_new_s + cfg.gamma_cap + 2, b=cfg.block_b, gamma_cap=cfg.gamma_cap, t0=t0,
+                  rho=cfg.rho)
+    o.prefill(prompt[:n_prompt_s])
+    t = time.perf_counter()
+    made = 0
+    while made < max_new_s:
+        while o.drafting:
+            o.draft_block(); o.preverify()
+        o.verify()
+        made += o.accept() + 1
+    dt = time.perf_counter() - t
+    return made / dt, made, dt
+
+
+def pair_to_cpu(pair):
+    return {k: ({n: t.cpu() for n, t in v.items()} if isinstance(v, dict) else v.cpu()) for k, v in pair.items()}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", default="7b_68m")
+    ap.add_argument("--impl", default="pacer", choices=["pacer", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-sample-new", type=int, default=4)
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    cfg = synth.CONFIGS[args.config]
+    t0 = PACER_T0
+    workload = {"workload": f"{cfg.name}: target {cfg.target.n_layers}L d={cfg.target.d_model}, draft "
+                            f"{cfg.draft.n_layers}L d={cfg.draft.d_model}, prompt {cfg.n_prompt}, new {cfg.max_new}, "
+                            f"gamma_max {cfg.gamma_max}, b {cfg.block_b}, rho {cfg.rho}, t0 {t0}, greedy, batch 1",
+                "weights": "N(0,0.02) seed 0, planted successor bias +8, agreement %.2f" % cfg.agree,
+                "l2": "inputs (13.2 GB of weights per forward) exceed L2; no flush needed"}
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        dev = "cuda:0" if torch.cuda.is_available() else "cpu"
+        pair = pair_to_cpu(synth.make_pair(cfg, seed=0, device=dev))
+        prompt = synth.make_prompts(cfg.target.vocab, 1, cfg.n_prompt, seed=0)[0].numpy()
+        vals = []
+        for i in range(args.warmup + args.steps):
+            v, made, dt = oracle_sample(cfg, pair, prompt, 4, args.cpu_sample_new, t0)
+            if i >= args.warmup:
+                vals.append((v, made, dt))
+        tot_tok = sum(m for _, m, _ in vals); tot_t = sum(d for _, _, d in vals)
+        val = tot_tok / tot_t
+        cores = int(os.environ.get("OMP_NUM_THREADS", os.cpu_count()))
+        sample = f"first 4 prompt tokens, Algorithm 1 until >= {args.cpu_sample_new} new tokens, per step"
+        print(json.dumps({"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+                          "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * tot_t / max(1, len(vals)),
+                          "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+                          "data": "synthetic", "config": workload,
+                          "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+                          "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+        return
+
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
+    torch.cuda.set_device(local_rank)
+    dev = f"cuda:{local_rank}"
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl")
+    from paper_2602_01274_b200 import binding as b
+
+    pair = synth.make_pair(cfg, seed=0, device=dev)
+    prompt = synth.make_prompts(cfg.target.vocab, 1, cfg.n_prompt, seed=rank)[0].numpy()
+    max_ctx = cfg.n_prompt + cfg.max_new + cfg.gamma_cap + 2
+    ctx = b.Context(b.make_cfg(cfg.target, cfg.draft, 1, max_ctx, cfg.gamma_cap, cfg.block_b, cfg.rho, 0, cfg.succ_bias),
+                    device=dev)
+    b.load_pair(ctx, pair)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        ctx.pacer_generate(prompt, cfg.max_new, cfg.gamma_max, t0)
+    sampler = ClockSampler(local_rank)
+    barrier()
+    sampler.start()
+    dec_ms, tok, launches, e2e_s = 0.0, 0, 0, 0.0
+    stats_all = []
+    wall0 = time.perf_counter()
+    for _ in range(args.steps):
+        ts = time.perf_counter()
+        toks, ns, dl, al, st = ctx.pacer_generate(prompt, cfg.max_new, cfg.gamma_max, t0)
+        torch.cuda.synchronize()
+        e2e_s += time.perf_counter() - ts
+        dec_ms += st["ms_decode"]; tok += cfg.max_new; launches += st["n_kernel_launches"]
+        stats_all.append((st, ns[0], dl[0, : ns[0]].copy(), al[0, : ns[0]].copy()))
+    barrier()
+    wall = time.perf_counter() - wall0
+    clocks = sampler.stop()
+
+    # baselines on the same kernels (outside the timed region): autoregressive and fixed windows
+    ar_tok, ar_st = ctx.pacer_generate_ar(prompt, cfg.max_new)
+    ar_tps = cfg.max_new / (ar_st["ms_decode"] * 1e-3)
+    lossless = bool((ar_tok[0] == toks[0]).all())
+    fixed = {}
+    for g in range(cfg.block_b, cfg.gamma_cap + 1, cfg.block_b):
+        _, _, _, _, s2 = ctx.pacer_generate(prompt, cfg.max_new, g, -1.0)
+        fixed[g] = cfg.max_new / (s2["ms_decode"] * 1e-3)
+    best_g = max(fixed, key=fixed.get)
+
+    # verify forward: whole-forward time and kernel-level GEMM time, live
+    ctx.pacer_prefill(prompt, cfg.max_new, cfg.gamma_max, -1.0)
+    for _ in range(cfg.gamma_cap // cfg.block_b):     # a full window of drafts, so the verify has gamma_cap + 1 rows
+        for _ in range(cfg.block_b):
+            ctx.pacer_draft_step()
+        ctx.pacer_preverify()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    n_ver = 10
+    for _ in range(3):
+        ctx.pacer_verify()
+    e0.record(ctx.stream)
+    for _ in range(n_ver):
+        ctx.pacer_verify()            # same rows every time: the state does not advance without accept
+    e1.record(ctx.stream)
+    torch.cuda.synchronize()
+    ver_ms = e0.elapsed_time(e1) / n_ver
+    ctx.pacer_profile_begin()
+    for _ in range(n_ver):
+        ctx.pacer_verify()
+    gemm_ms, gemm_bytes, gemm_n = ctx.pacer_profile_end()
+    peak, peak_kind = _peaks()
+    vbytes = verify_bytes(cfg, cfg.n_prompt - 1, cfg.gamma_cap + 1)
+    gemm_gbs = gemm_bytes / (gemm_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": "k_gemm_skinny", "achieved": gemm_gbs, "peak": peak, "unit": "GB/s",
+                "frac": gemm_gbs / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
+                "launches_timed": gemm_n, "bytes_per_launch_avg": gemm_bytes / max(1, gemm_n),
+                "ms_per_launch_avg": gemm_ms / max(1, gemm_n)}
+    verify = {"ms": ver_ms, "algorithmic_gb": vbytes / 1e9, "achieved_gbs": vbytes / (ver_ms * 1e-3) / 1e9,
+              "frac_of_measured_peak": vbytes / (ver_ms * 1e-3) / 1e9 / peak,
+              "frac_of_8tbs": vbytes / (ver_ms * 1e-3) / 1e9 / 8000.0, "rows": cfg.gamma_cap + 1}
+
+    val_local = tok / (dec_ms * 1e-3)
+    e2e_local = tok / e2e_s
+    if world > 1:
+        t = torch.tensor([dec_ms, e2e_s, float(tok)], device=dev, dtype=torch.float64)
+        mx = t.clone(); dist.all_reduce(mx, op=dist.ReduceOp.MAX)
+        sm = t.clone(); dist.all_reduce(sm, op=dist.ReduceOp.SUM)
+        value = sm[2].item() / (mx[0].item() * 1e-3)
+        e2e_val = sm[2].item() / mx[1].item()
+        ms_step = mx[0].item() / args.steps
+    else:
+        value, e2e_val, ms_step = val_local, e2e_local, dec_ms / args.steps
+    if rank != 0:
+        return
+
+    st, ns, dl, al = stats_all[-1]
+    out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+           "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+           "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": workload,
+           "clocks": clocks, "gpu_launches": int(launches),
+           "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": int(prompt.nbytes),
+                   "d2h_bytes_per_step": int(4 * cfg.max_new * 3 + 4 + 128),
+                   "note": "pacer_generate with host prompt and host outputs; prefill inside the timed region"},
+           "roofline": roofline, "verify_forward": verify,
+           "loop": {"tokens_per_s_ar_same_kernels": ar_tps, "speedup_vs_ar": value / ar_tps,
+                    "tokens_per_s_fixed_gamma": fixed, "best_fixed_gamma": best_g,
+                    "speedup_vs_best_fixed": value / fixed[best_g], "tau": float(al.mean()),
+                    "mean_gamma": float(dl.mean()), "steps": int(ns), "n_draft_fwd": st["n_draft_fwd"],
+                    "n_mb_calls": st["n_mb_calls"], "n_target_fwd": st["n_target_fwd"],
+                    "ms_prefill": st["ms_prefill"], "lossless_vs_gpu_ar": lossless},
+           "wall_s_timed_region": wall}
+    if not args.no_cpu_baseline:
+        try:
+            v, made, dt = oracle_sample(cfg, pair_to_cpu(pair), prompt, 4, args.cpu_sample_new, t0)
+            out["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": int(os.environ.get("OMP_NUM_THREADS", os.cpu_count())),
+                                   "kind": "oracle",
+                                   "sample": f"first 4 prompt tokens, Algorithm 1 until >= {args.cpu_sample_new} new "
+                                             f"tokens ({made} made in {dt:.1f} s)"}
+        except Exception as ex:  # the baseline must not take the GPU numbers down with it
+            out["cpu_baseline"] = {"value": None, "unit": UNIT, "cores": 0, "kind": "oracle", "sample": f"failed: {ex}"}
+    print(json.dumps(out))
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,223 @@
+/*
+ * pacer.h - C ABI of the B200 (sm_100a) hot path of Pacer: speculative decoding
+ * in which a draft model decodes in blocks of b tokens, a one-layer
+ * pre-verification model scores every block and stops the drafting when a block
+ * fails, the target model verifies all drafts in one forward over its KV cache,
+ * and an acceptance step commits a prefix of the drafts and rolls the caches back.
+ *
+ * Conventions
+ *   - Every function returns 0 (PACER_OK) or a negative PACER_E* code; nothing
+ *     throws, aborts or traps the device.  pacer_strerror(code) and
+ *     pacer_last_error(ctx) give text.
+ *   - "device" pointers are CUDA device addresses on the current device, "host"
+ *     pointers are ordinary memory.  All device memory is CALLER-OWNED: the
+ *     library never allocates or frees device memory.  It carves the workspace
+ *     given to pacer_create and reads weights in place.
+ *   - Calls enqueue work on the context's stream and return without waiting
+ *     unless marked [sync].  A context is not thread-safe.
+ *   - Models are Llama-style decoders: RMSNorm, rotary embedding (rotate-half,
+ *     absolute positions), causal attention with n_kv_heads <= n_heads, SwiGLU
+ *     MLP, untied embedding and LM head, no biases.  Weights are bf16, matrices
+ *     are [out][in] row-major and stacked over layers; accumulation, the residual
+ *     stream, norms and softmax are fp32; KV caches are bf16.
+ *   - Batch rows are independent sequences.  Token ids are int32.
+ */
+#ifndef PACER_H_
+#define PACER_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    PACER_OK = 0,
+    PACER_EINVAL = -1,       /* bad argument (null pointer, size out of range, shape mismatch) */
+    PACER_ENOMEM = -2,       /* workspace too small */
+    PACER_ECUDA = -3,        /* a CUDA runtime call failed; see pacer_last_error */
+    PACER_EDEVICE = -4,      /* a kernel reported an anomaly in the device status word */
+    PACER_ESTATE = -5,       /* call out of order (weights missing, no prefill, ...) */
+    PACER_EUNSUPPORTED = -6
+};
+
+typedef struct pacer_ctx pacer_ctx;
+
+typedef struct {
+    int32_t n_layers, d_model, n_heads, n_kv_heads, d_ffn, vocab;
+    float rope_theta;        /* 10000 */
+    float rms_eps;           /* 1e-5 */
+} pacer_model_cfg;
+
+typedef struct {
+    pacer_model_cfg target, draft;   /* the pre-verification model M_B is ONE layer with the draft's widths */
+    int32_t max_batch;       /* sequences decoded together */
+    int32_t max_ctx;         /* cache rows per sequence: n_prompt + max_new + gamma_cap + 2 must fit */
+    int32_t gamma_cap;       /* largest draft window; a multiple of block_b */
+    int32_t block_b;         /* drafts per pre-verification block (paper: b) */
+    float rho;               /* threshold growth per passed block (paper: rho > 1) */
+    int32_t criterion;       /* block statistic: 0 mean (the method), 1 minimum ("any"), 2 last token */
+    float succ_bias;         /* added to logit succ[input token] of every LM-head row; 0 = off */
+    int32_t use_posemb;      /* 1: add the draft position embedding e_i (the method); 0: ablation */
+} pacer_cfg;
+
+/* One named weight tensor, bf16, contiguous, on the device.  Names per model:
+ *   embed [V][d]            wqkv [L][(H+2Hkv)*hd][d]  (q rows, then k, then v)
+ *   wo [L][d][H*hd]         wgate, wup [L][F][d]       wdown [L][d][F]
+ *   norm1, norm2 [L][d]     normf [d]                  head [V][d]
+ * M_B (which = 2) has no embed/head but  head_b [2][d]  and  posemb [gamma_cap][d].
+ * The tensors are used in place and must outlive the context. */
+typedef struct {
+    const char *name;
+    const void *dev_ptr;
+    int64_t numel;
+} pacer_tensor;
+
+enum { PACER_TARGET = 0, PACER_DRAFT = 1, PACER_PREVERIFY = 2 };
+enum { PACER_GREEDY = 0, PACER_SAMPLE = 1 };
+
+/* Counters and device-side timings of one pacer_generate / pacer_generate_ar call. */
+typedef struct {
+    int64_t n_draft_fwd, n_mb_calls, n_target_fwd, n_steps;  /* summed over sequences */
+    int64_t n_generated;        /* tokens committed, summed over sequences (before truncation to max_new) */
+    int64_t n_kernel_launches;  /* kernels of this library launched inside the timed decode region */
+    float ms_prefill;           /* CUDA-event time of the prefill */
+    float ms_decode;            /* CUDA-event time of the decode loop (first step .. last step) */
+} pacer_stats;
+
+/* Per-sequence scalars copied out by pacer_read_state. */
+typedef struct {
+    int32_t P;                  /* accepted tokens so far, prompt included */
+    int32_t len_T, len_D, len_B;/* rows in the target / draft / M_B caches */
+    int32_t gamma;              /* drafts made in the current step */
+    int32_t k_round;            /* blocks that passed pre-verification in the current step */
+    float t_k;                  /* current threshold t_0 * rho^k */
+    int32_t drafting;           /* 1 while the draft loop of this step may continue */
+    int32_t finished;           /* 1 once max_new tokens exist */
+    int32_t n_steps;            /* draft-and-verify steps completed */
+    int32_t last_n, last_next;  /* accepted drafts and the follow-up token of the last step */
+    int32_t n_pend;             /* draft hidden rows not yet given to M_B */
+    int32_t err;                /* device status word of this sequence, 0 = fine */
+    int64_t n_draft_fwd, n_mb_calls, n_target_fwd;
+} pacer_seq_state;
+
+/* Device buffers that pacer_read_buffer can copy out (stage-by-stage checks). */
+enum {
+    PACER_BUF_TOKENS = 0,        /* int32 [max_batch][max_ctx]   accepted tokens x */
+    PACER_BUF_DRAFTS = 1,        /* int32 [max_batch][gamma_cap] y_1..y_gamma of the current step */
+    PACER_BUF_ALPHA = 2,         /* f32   [max_batch][gamma_cap] alpha_hat of the current step's drafts */
+    PACER_BUF_VERIFY_LOGITS = 3, /* f32   [max_batch][gamma_cap+1][V] target logits of the last verify */
+    PACER_BUF_DRAFT_LOGITS = 4,  /* f32   [max_batch][gamma_cap][V] draft logits q_i of the current step */
+    PACER_BUF_HPEND = 5,         /* f32   [max_batch][block_b+1][d_draft] hidden rows waiting for M_B */
+    PACER_BUF_DRAFT_LEN = 6,     /* int32 [max_batch][max_steps] gamma of every step */
+    PACER_BUF_ACCEPT_LEN = 7,    /* int32 [max_batch][max_steps] n of every step */
+    PACER_BUF_KCACHE_T = 8,      /* bf16  [L][max_batch][Hkv][max_ctx][hd] (also _D = 10, _B = 12) */
+    PACER_BUF_VCACHE_T = 9,      /* bf16  same shape                        (also _D = 11, _B = 13) */
+    PACER_BUF_KCACHE_D = 10, PACER_BUF_VCACHE_D = 11, PACER_BUF_KCACHE_B = 12, PACER_BUF_VCACHE_B = 13
+};
+
+const char *pacer_strerror(int code);
+const char *pacer_last_error(const pacer_ctx *ctx);
+
+/* Bytes of device workspace a context with this configuration needs (KV caches
+ * of the three models, activations, logits, per-sequence state).  0 on a bad
+ * configuration. */
+size_t pacer_workspace_bytes(const pacer_cfg *cfg);
+
+/* Creates a context on the current device.  dev_workspace: device, at least
+ * pacer_workspace_bytes(cfg) bytes, 256-byte aligned, caller-owned, must outlive
+ * the context.  cuda_stream: a cudaStream_t (NULL = the legacy default stream).
+ * Allocates host memory only.  Zeroes the state part of the workspace. */
+int pacer_create(const pacer_cfg *cfg, void *dev_workspace, size_t workspace_bytes, void *cuda_stream,
+                 pacer_ctx **out);
+
+/* Frees host memory and CUDA events/graphs of the context; the workspace and the
+ * weights stay untouched.  [sync] */
+int pacer_destroy(pacer_ctx *ctx);
+
+/* Registers the weights of one model (which = PACER_TARGET / _DRAFT / _PREVERIFY).
+ * tbl: host array of n entries naming device tensors (see pacer_tensor); numel is
+ * checked against the configuration.  succ: device int32 [V] planted successor
+ * table for the LM-head bias, or NULL (ignored for M_B). */
+int pacer_load_weights(pacer_ctx *ctx, int which, const pacer_tensor *tbl, int n, const int32_t *succ);
+
+/* Starts `batch` sequences from prompts (host int32 [batch][n_prompt]) and fills
+ * the three caches with prompt tokens 0..n_prompt-2; the last prompt token is the
+ * first step's input row (the prefix x of Algorithm 1).  The hidden states the
+ * draft produces for the prompt are M_B's history h_x (Eq. 7), without position
+ * embedding.  threshold / mode / seed / max_new configure the steps that follow:
+ * threshold < 0 means the block test always passes (fixed window gamma_max).
+ * gamma_max is rounded down to a multiple of block_b and must be in
+ * [block_b, gamma_cap]. */
+int pacer_prefill(pacer_ctx *ctx, const int32_t *prompt, int batch, int n_prompt, int max_new, int gamma_max,
+                  float threshold, int mode, uint64_t seed);
+
+/* One draft-model forward for every sequence that is still drafting (Eq. 6, one
+ * of the b steps of a block): emits y_i (argmax, or a Gumbel-max draw when
+ * sampling), keeps the logits q_i and queues the hidden state h_i for M_B.  The
+ * first forward after a fully accepted step takes two rows (the draft cache
+ * lacks the last draft of that step). */
+int pacer_draft_step(pacer_ctx *ctx);
+
+/* Pre-verification of the rows queued since the last call (Eq. 7): M_B on
+ * [h_i + e_i] against its own KV cache gives alpha_hat_i; then the block test of
+ * Algorithm 1: drafting stops when the block statistic <= t_k or the window is
+ * full, else t_{k+1} = t_k * rho. */
+int pacer_preverify(pacer_ctx *ctx);
+
+/* One target forward over [last accepted token, y_1..y_gamma] per sequence
+ * (Eq. 4), appending their K/V rows and leaving logits p_1..p_{gamma+1}. */
+int pacer_verify(pacer_ctx *ctx);
+
+/* Acceptance (Eq. 5; greedy = prefix match with the target's argmax), commit of
+ * [y_1..y_n, next], truncation of the three caches to the accepted rows, reset of
+ * the per-step state, logging of (gamma, n). Uses the mode and seed of pacer_prefill. */
+int pacer_accept_rollback(pacer_ctx *ctx);
+
+/* [sync] Copies the per-sequence scalars of sequences 0..batch-1 to host memory. */
+int pacer_read_state(pacer_ctx *ctx, pacer_seq_state *out, int batch);
+
+/* [sync] Copies `bytes` bytes from the start of one device buffer (PACER_BUF_*) to host memory. */
+int pacer_read_buffer(pacer_ctx *ctx, int which, void *host_dst, size_t bytes);
+
+/* [sync] Algorithm 1 end to end: prefill, then draft-and-verify steps until every
+ * sequence has max_new new tokens, all steps enqueued as device-side controlled
+ * work (no host decision per token or per step).  Outputs, all host, caller-owned:
+ *   out_tokens     int32 [batch][max_new]
+ *   out_n_steps    int32 [batch]
+ *   out_draft_len  int32 [batch][max_new]  gamma of step s, -1 beyond n_steps
+ *   out_accept_len int32 [batch][max_new]  n of step s, -1 beyond n_steps
+ *   stats          may be NULL */
+int pacer_generate(pacer_ctx *ctx, const int32_t *prompt, int batch, int n_prompt, int max_new, int gamma_max,
+                   float threshold, int mode, uint64_t seed, int32_t *out_tokens, int32_t *out_n_steps,
+                   int32_t *out_draft_len, int32_t *out_accept_len, pacer_stats *stats);
+
+/* [sync] Autoregressive decoding of the target alone on the same kernels (Eq. 1):
+ * the baseline, and under greedy decoding the definition of the lossless output. */
+int pacer_generate_ar(pacer_ctx *ctx, const int32_t *prompt, int batch, int n_prompt, int max_new, int mode,
+                      uint64_t seed, int32_t *out_tokens, pacer_stats *stats);
+
+/* Kernel-level timing for roofline reports.  Between pacer_profile_begin and
+ * pacer_profile_end every weight-streaming product this context launches is
+ * bracketed by a pair of CUDA events on the context's stream (at most 4096
+ * products are recorded; later ones run untimed).  pacer_profile_end [sync]
+ * returns the summed device time of those launches (ms), the bf16 weight bytes
+ * they streamed (N*K*2 each) and their count.  Event pairs serialise nothing but
+ * add about a microsecond each, so whole-loop timings are taken without it. */
+int pacer_profile_begin(pacer_ctx *ctx);
+int pacer_profile_end(pacer_ctx *ctx, double *gemm_ms, double *gemm_weight_bytes, int64_t *gemm_launches);
+
+/* Y[r][n] = sum_k X[r][k] * W[n][k]: the skinny weight-streaming product used by
+ * every projection, exposed for kernel-level checks and timing.  x: device bf16
+ * [rows][K] row-major; w: device bf16 [N][K]; y: device f32 [rows][N];
+ * scratch: device, at least pacer_linear_scratch_bytes(rows, N, K) bytes.
+ * rows <= 32, K a multiple of 32.  Enqueues on `cuda_stream`. */
+size_t pacer_linear_scratch_bytes(int rows, int N, int K);
+int pacer_linear(const void *x, const void *w, float *y, int rows, int N, int K, void *scratch,
+                 size_t scratch_bytes, void *cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PACER_H_ */

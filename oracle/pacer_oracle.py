@@ -165,8 +165,8 @@ class Cache:
         self.h = lib().orc_cache_new(model.ref(), max_ctx)
 
     def __del__(self):
-        if getattr(self, "h", None):
-            lib().orc_cache_free(self.h)
+        if getattr(self, "h", None) and _lib is not None:
+            _lib.orc_cache_free(self.h)
             self.h = None
 
     @property
@@ -256,8 +256,8 @@ class Pacer:
         self._override = None
 
     def __del__(self):
-        if getattr(self, "h", None):
-            lib().orc_free(self.h)
+        if getattr(self, "h", None) and _lib is not None:
+            _lib.orc_free(self.h)
             self.h = None
 
     # stages

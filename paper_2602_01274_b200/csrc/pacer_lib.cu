@@ -1,0 +1,692 @@
+// C-ABI entry points of the Pacer library (see include/pacer.h) and the host-side
+// sequencing of the kernels.  The host only enqueues; every data-dependent
+// decision (rows of a forward, stop of the draft loop, acceptance, rollback,
+// end of generation) is taken by kernels from the device-resident SeqState.
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <string>
+#include <vector>
+
+#include "attention.cuh"
+#include "common.cuh"
+#include "control.cuh"
+#include "gemm.cuh"
+#include "rowops.cuh"
+
+struct pacer_ctx {
+    pacer_cfg cfg;
+    cudaStream_t stream;
+    char *ws;
+    size_t ws_bytes;
+    DevPtrs d;
+    ModelDev model[3];
+    Geom g_draft, g_mb, g_verify, g_ar;
+    int batch;                 // sequences of the current run
+    int prefilled;
+    int64_t launches;
+    cudaEvent_t ev[4];
+    std::vector<float2> rope_host[3];
+    std::string err;
+    size_t buf_bytes[16];
+    void *buf_ptr[16];
+    // kernel-level profiling (pacer_profile_begin / _end)
+    int prof_on;
+    std::vector<cudaEvent_t> prof_ev;      // pairs
+    size_t prof_used;
+    double prof_bytes;
+};
+
+static thread_local std::string g_err;
+
+extern "C" const char *pacer_strerror(int code) {
+    switch (code) {
+        case PACER_OK: return "ok";
+        case PACER_EINVAL: return "invalid argument";
+        case PACER_ENOMEM: return "workspace too small";
+        case PACER_ECUDA: return "CUDA runtime error";
+        case PACER_EDEVICE: return "device-side anomaly";
+        case PACER_ESTATE: return "call out of order";
+        case PACER_EUNSUPPORTED: return "unsupported";
+    }
+    return "unknown error";
+}
+
+extern "C" const char *pacer_last_error(const pacer_ctx *ctx) { return ctx ? ctx->err.c_str() : g_err.c_str(); }
+
+static int fail(pacer_ctx *c, int code, const std::string &msg) {
+    if (c) c->err = msg;
+    g_err = msg;
+    return code;
+}
+
+#define CK(call)                                                                                       \
+    do {                                                                                               \
+        cudaError_t e_ = (call);                                                                       \
+        if (e_ != cudaSuccess)                                                                         \
+            return fail(c, PACER_ECUDA, std::string(#call) + ": " + cudaGetErrorString(e_));           \
+    } while (0)
+
+// ------------------------------------------------------------------ configuration
+
+static bool model_cfg_ok(const pacer_model_cfg &m) {
+    if (m.n_layers < 1 || m.d_model < 32 || m.n_heads < 1 || m.n_kv_heads < 1 || m.d_ffn < 32 || m.vocab < 2) return false;
+    if (m.d_model % m.n_heads) return false;
+    const int hd = m.d_model / m.n_heads;
+    if (hd != 32 && hd != 64 && hd != 128) return false;
+    if (m.n_heads % m.n_kv_heads) return false;
+    if (m.d_model % 32 || m.d_ffn % 32) return false;
+    return true;
+}
+
+static bool cfg_ok(const pacer_cfg *c) {
+    if (!c) return false;
+    if (!model_cfg_ok(c->target) || !model_cfg_ok(c->draft)) return false;
+    if (c->target.vocab != c->draft.vocab) return false;
+    if (c->max_batch < 1 || c->max_batch > 64 || c->max_ctx < 4) return false;
+    if (c->block_b < 1 || c->gamma_cap < c->block_b || c->gamma_cap % c->block_b) return false;
+    if (c->criterion < 0 || c->criterion > 2) return false;
+    if (!(c->rho > 0.f)) return false;
+    return true;
+}
+
+static pacer_model_cfg mb_cfg(const pacer_cfg &c) {
+    pacer_model_cfg m = c.draft;
+    m.n_layers = 1;
+    return m;
+}
+
+struct Carver {
+    size_t off = 0;
+    size_t take(size_t bytes) {
+        size_t o = off;
+        off += (bytes + 255) / 256 * 256;
+        return o;
+    }
+};
+
+struct Layout {
+    size_t st, x, y, alpha, hpend, hpend_e, draft_len, accept_len, verify_logits, draft_logits;
+    size_t row_pos, row_tok, n_rows, row_arg, row_margin, xres, xn, att, act, q, hidden, part;
+    size_t kc[3], vc[3], rope[3];
+    size_t kv_bytes[3], rope_bytes[3];
+    size_t total;
+    int rtot_max, nt_max, max_steps;
+    size_t part_bytes, state_bytes;
+};
+
+static size_t part_floats(const pacer_model_cfg &m, int nt_max, bool with_head) {
+    const int hd = m.d_model / m.n_heads, qrows = (m.n_heads + 2 * m.n_kv_heads) * hd;
+    const int NT = nt_max < 4 ? nt_max : 4;
+    struct { int N, K; } shp[5] = {{qrows, m.d_model}, {m.d_model, m.n_heads * hd}, {2 * m.d_ffn, m.d_model},
+                                   {m.d_model, m.d_ffn}, {m.vocab, m.d_model}};
+    size_t mx = 0;
+    for (int i = 0; i < (with_head ? 5 : 4); ++i) {
+        GemmPlan p = gemm_plan(shp[i].N, shp[i].K, NT);
+        size_t f = (size_t)p.S * nt_max * 8 * shp[i].N;
+        if (f > mx) mx = f;
+    }
+    return mx;
+}
+
+static Layout make_layout(const pacer_cfg &c) {
+    Layout L;
+    Carver cv;
+    const pacer_model_cfg mb = mb_cfg(c);
+    const pacer_model_cfg *ms[3] = {&c.target, &c.draft, &mb};
+    const int B = c.max_batch, gc = c.gamma_cap, V = c.target.vocab;
+    const int rps_max = gc + 1 > c.block_b + 1 ? gc + 1 : c.block_b + 1;
+    L.rtot_max = B * rps_max;
+    L.nt_max = (L.rtot_max + 7) / 8;
+    L.max_steps = c.max_ctx;
+    int d_max = 0, hh_max = 0, f_max = 0;
+    for (int i = 0; i < 3; ++i) {
+        d_max = ms[i]->d_model > d_max ? ms[i]->d_model : d_max;
+        f_max = ms[i]->d_ffn > f_max ? ms[i]->d_ffn : f_max;
+    }
+    hh_max = d_max;
+    L.st = cv.take(sizeof(SeqState) * B);
+    L.x = cv.take(sizeof(int32_t) * B * c.max_ctx);
+    L.y = cv.take(sizeof(int32_t) * B * gc);
+    L.alpha = cv.take(sizeof(float) * B * gc);
+    L.hpend_e = cv.take(sizeof(int32_t) * B * (c.block_b + 1));
+    L.draft_len = cv.take(sizeof(int32_t) * B * L.max_steps);
+    L.accept_len = cv.take(sizeof(int32_t) * B * L.max_steps);
+    L.row_pos = cv.take(sizeof(int32_t) * L.rtot_max);
+    L.row_tok = cv.take(sizeof(int32_t) * L.rtot_max);
+    L.n_rows = cv.take(sizeof(int32_t) * B);
+    L.row_arg = cv.take(sizeof(int32_t) * L.rtot_max);
+    L.row_margin = cv.take(sizeof(float) * L.rtot_max);
+    L.state_bytes = cv.off;                                   // zeroed at create
+    L.hpend = cv.take(sizeof(float) * B * (c.block_b + 1) * c.draft.d_model);
+    L.verify_logits = cv.take(sizeof(float) * B * (gc + 1) * V);
+    L.draft_logits = cv.take(sizeof(float) * B * gc * V);
+    L.xres = cv.take(sizeof(float) * L.rtot_max * d_max);
+    L.hidden = cv.take(sizeof(float) * L.rtot_max * d_max);
+    L.q = cv.take(sizeof(float) * L.rtot_max * hh_max);
+    L.xn = cv.take(sizeof(bf16) * L.nt_max * 8 * d_max);
+    L.att = cv.take(sizeof(bf16) * L.nt_max * 8 * hh_max);
+    L.act = cv.take(sizeof(bf16) * L.nt_max * 8 * f_max);
+    size_t pf = 0;
+    for (int i = 0; i < 3; ++i) {
+        size_t f = part_floats(*ms[i], L.nt_max, i != 2);
+        if (f > pf) pf = f;
+    }
+    L.part_bytes = pf * sizeof(float);
+    L.part = cv.take(L.part_bytes);
+    for (int i = 0; i < 3; ++i) {
+        const int hd = ms[i]->d_model / ms[i]->n_heads;
+        L.kv_bytes[i] = sizeof(bf16) * (size_t)ms[i]->n_layers * B * ms[i]->n_kv_heads * c.max_ctx * hd;
+        L.kc[i] = cv.take(L.kv_bytes[i]);
+        L.vc[i] = cv.take(L.kv_bytes[i]);
+        L.rope_bytes[i] = sizeof(float2) * (size_t)c.max_ctx * (hd / 2);
+        L.rope[i] = cv.take(L.rope_bytes[i]);
+    }
+    L.total = cv.off;
+    return L;
+}
+
+extern "C" size_t pacer_workspace_bytes(const pacer_cfg *cfg) {
+    if (!cfg_ok(cfg)) return 0;
+    return make_layout(*cfg).total;
+}
+
+static Geom make_geom(int batch, int rps) {
+    Geom g;
+    g.batch = batch; g.rps = rps; g.rtot = batch * rps; g.nt = (g.rtot + 7) / 8;
+    return g;
+}
+
+static void set_geoms(pacer_ctx *c, int batch) {
+    c->batch = batch;
+    c->g_draft = make_geom(batch, 2);
+    c->g_mb = make_geom(batch, c->cfg.block_b + 1);
+    c->g_verify = make_geom(batch, c->cfg.gamma_cap + 1);
+    c->g_ar = make_geom(batch, 1);
+}
+
+extern "C" int pacer_create(const pacer_cfg *cfg, void *dev_workspace, size_t workspace_bytes, void *cuda_stream,
+                            pacer_ctx **out) {
+    pacer_ctx *c = nullptr;
+    if (!out) return fail(nullptr, PACER_EINVAL, "out is null");
+    *out = nullptr;
+    if (!cfg_ok(cfg)) return fail(nullptr, PACER_EINVAL, "bad configuration");
+    if (!dev_workspace || ((uintptr_t)dev_workspace & 255)) return fail(nullptr, PACER_EINVAL, "workspace null or not 256-byte aligned");
+    Layout L = make_layout(*cfg);
+    if (workspace_bytes < L.total) return fail(nullptr, PACER_ENOMEM, "workspace smaller than pacer_workspace_bytes");
+    c = new pacer_ctx();
+    c->cfg = *cfg;
+    c->stream = (cudaStream_t)cuda_stream;
+    c->ws = (char *)dev_workspace;
+    c->ws_bytes = workspace_bytes;
+    c->prefilled = 0;
+    c->launches = 0;
+    c->prof_on = 0;
+    c->prof_used = 0;
+    c->prof_bytes = 0;
+    DevPtrs &d = c->d;
+    char *w = c->ws;
+    d.st = (SeqState *)(w + L.st); d.x = (int32_t *)(w + L.x); d.y = (int32_t *)(w + L.y);
+    d.alpha = (float *)(w + L.alpha); d.hpend = (float *)(w + L.hpend); d.hpend_e = (int32_t *)(w + L.hpend_e);
+    d.draft_len = (int32_t *)(w + L.draft_len); d.accept_len = (int32_t *)(w + L.accept_len);
+    d.verify_logits = (float *)(w + L.verify_logits); d.draft_logits = (float *)(w + L.draft_logits);
+    d.row_pos = (int32_t *)(w + L.row_pos); d.row_tok = (int32_t *)(w + L.row_tok); d.n_rows = (int32_t *)(w + L.n_rows);
+    d.row_arg = (int32_t *)(w + L.row_arg); d.row_margin = (float *)(w + L.row_margin);
+    d.xres = (float *)(w + L.xres); d.xn = (bf16 *)(w + L.xn); d.att = (bf16 *)(w + L.att); d.act = (bf16 *)(w + L.act);
+    d.q = (float *)(w + L.q); d.hidden = (float *)(w + L.hidden); d.part = (float *)(w + L.part);
+    d.max_batch = cfg->max_batch; d.max_ctx = cfg->max_ctx; d.gamma_cap = cfg->gamma_cap; d.block_b = cfg->block_b;
+    d.max_steps = L.max_steps; d.rho = cfg->rho; d.succ_bias = cfg->succ_bias; d.criterion = cfg->criterion;
+    d.use_posemb = cfg->use_posemb;
+    const pacer_model_cfg mb = mb_cfg(*cfg);
+    const pacer_model_cfg *ms[3] = {&cfg->target, &cfg->draft, &mb};
+    for (int i = 0; i < 3; ++i) {
+        ModelDev &m = c->model[i];
+        memset(&m, 0, sizeof m);
+        m.cfg = *ms[i];
+        m.hd = m.cfg.d_model / m.cfg.n_heads;
+        m.qrows = (m.cfg.n_heads + 2 * m.cfg.n_kv_heads) * m.hd;
+        m.kcache = (bf16 *)(w + L.kc[i]);
+        m.vcache = (bf16 *)(w + L.vc[i]);
+        m.rope = (const float2 *)(w + L.rope[i]);
+        const int half = m.hd / 2;
+        c->rope_host[i].resize((size_t)cfg->max_ctx * half);
+        for (int p = 0; p < cfg->max_ctx; ++p)
+            for (int k = 0; k < half; ++k) {
+                const double ang = (double)p * pow((double)m.cfg.rope_theta, -2.0 * k / m.hd);
+                c->rope_host[i][(size_t)p * half + k] = make_float2((float)cos(ang), (float)sin(ang));
+            }
+    }
+    // buffers readable through pacer_read_buffer
+    const int B = cfg->max_batch, gc = cfg->gamma_cap, V = cfg->target.vocab;
+    memset(c->buf_bytes, 0, sizeof c->buf_bytes);
+    auto reg = [&](int id, void *p, size_t n) { c->buf_ptr[id] = p; c->buf_bytes[id] = n; };
+    reg(PACER_BUF_TOKENS, d.x, sizeof(int32_t) * B * cfg->max_ctx);
+    reg(PACER_BUF_DRAFTS, d.y, sizeof(int32_t) * B * gc);
+    reg(PACER_BUF_ALPHA, d.alpha, sizeof(float) * B * gc);
+    reg(PACER_BUF_VERIFY_LOGITS, d.verify_logits, sizeof(float) * B * (gc + 1) * V);
+    reg(PACER_BUF_DRAFT_LOGITS, d.draft_logits, sizeof(float) * B * gc * V);
+    reg(PACER_BUF_HPEND, d.hpend, sizeof(float) * B * (cfg->block_b + 1) * cfg->draft.d_model);
+    reg(PACER_BUF_DRAFT_LEN, d.draft_len, sizeof(int32_t) * B * L.max_steps);
+    reg(PACER_BUF_ACCEPT_LEN, d.accept_len, sizeof(int32_t) * B * L.max_steps);
+    for (int i = 0; i < 3; ++i) {
+        reg(PACER_BUF_KCACHE_T + 2 * i, c->model[i].kcache, L.kv_bytes[i]);
+        reg(PACER_BUF_VCACHE_T + 2 * i, c->model[i].vcache, L.kv_bytes[i]);
+    }
+    set_geoms(c, 1);
+    cudaError_t e = cudaMemsetAsync(c->ws, 0, L.state_bytes, c->stream);
+    for (int i = 0; i < 3 && e == cudaSuccess; ++i)
+        e = cudaMemcpyAsync((void *)c->model[i].rope, c->rope_host[i].data(), L.rope_bytes[i], cudaMemcpyHostToDevice, c->stream);
+    for (int i = 0; i < 4 && e == cudaSuccess; ++i) e = cudaEventCreate(&c->ev[i]);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
+    if (e != cudaSuccess) {
+        std::string msg = std::string("pacer_create: ") + cudaGetErrorString(e);
+        delete c;
+        return fail(nullptr, PACER_ECUDA, msg);
+    }
+    *out = c;
+    return PACER_OK;
+}
+
+extern "C" int pacer_destroy(pacer_ctx *c) {
+    if (!c) return PACER_EINVAL;
+    cudaStreamSynchronize(c->stream);
+    for (int i = 0; i < 4; ++i) cudaEventDestroy(c->ev[i]);
+    for (cudaEvent_t e : c->prof_ev) cudaEventDestroy(e);
+    delete c;
+    return PACER_OK;
+}
+
+// ------------------------------------------------------------------ weights
+
+extern "C" int pacer_load_weights(pacer_ctx *c, int which, const pacer_tensor *tbl, int n, const int32_t *succ) {
+    if (!c || !tbl || which < 0 || which > 2 || n < 1) return fail(c, PACER_EINVAL, "pacer_load_weights: bad argument");
+    ModelDev &m = c->model[which];
+    const pacer_model_cfg &k = m.cfg;
+    const int64_t L = k.n_layers, d = k.d_model, F = k.d_ffn, V = k.vocab, hh = (int64_t)k.n_heads * m.hd;
+    struct Want { const char *name; const bf16 **slot; int64_t numel; bool needed; };
+    const bool isB = which == PACER_PREVERIFY;
+    Want want[] = {
+        {"embed", &m.embed, V * d, !isB}, {"wqkv", &m.wqkv, L * m.qrows * d, true}, {"wo", &m.wo, L * d * hh, true},
+        {"wgate", &m.wgate, L * F * d, true}, {"wup", &m.wup, L * F * d, true}, {"wdown", &m.wdown, L * d * F, true},
+        {"norm1", &m.norm1, L * d, true}, {"norm2", &m.norm2, L * d, true}, {"normf", &m.normf, d, true},
+        {"head", &m.head, V * d, !isB}, {"head_b", &m.head_b, 2 * d, isB},
+        {"posemb", &m.posemb, (int64_t)c->cfg.gamma_cap * d, isB},
+    };
+    for (auto &wn : want) *wn.slot = nullptr;
+    for (int i = 0; i < n; ++i) {
+        if (!tbl[i].name || !tbl[i].dev_ptr) return fail(c, PACER_EINVAL, "pacer_load_weights: null entry");
+        bool found = false;
+        for (auto &wn : want) {
+            if (strcmp(wn.name, tbl[i].name)) continue;
+            found = true;
+            if (!wn.needed) break;
+            if (tbl[i].numel != wn.numel)
+                return fail(c, PACER_EINVAL, std::string("pacer_load_weights: wrong size for ") + wn.name);
+            if ((uintptr_t)tbl[i].dev_ptr & 15)
+                return fail(c, PACER_EINVAL, std::string("pacer_load_weights: tensor not 16-byte aligned: ") + wn.name);
+            *wn.slot = (const bf16 *)tbl[i].dev_ptr;
+        }
+        if (!found) return fail(c, PACER_EINVAL, std::string("pacer_load_weights: unknown tensor ") + tbl[i].name);
+    }
+    for (auto &wn : want)
+        if (wn.needed && !*wn.slot) return fail(c, PACER_EINVAL, std::string("pacer_load_weights: missing tensor ") + wn.name);
+    m.succ = isB ? nullptr : succ;
+    m.loaded = 1;
+    return PACER_OK;
+}
+
+// ------------------------------------------------------------------ one forward
+
+#define LAUNCH_CHECK()                                                      \
+    do {                                                                    \
+        ++c->launches;                                                      \
+        CK(cudaGetLastError());                                             \
+    } while (0)
+
+// One weight-streaming product of a forward, optionally bracketed by profiling events.
+static int fwd_gemm(pacer_ctx *c, const bf16 *X, const Geom &g, const bf16 *W1, const bf16 *W2, int n_w1, int N, int K,
+                    GemmPlan *p) {
+    const bool prof = c->prof_on && c->prof_used + 2 <= c->prof_ev.size();
+    if (prof) CK(cudaEventRecord(c->prof_ev[c->prof_used], c->stream));
+    CK(gemm_run(X, g.nt, W1, W2, n_w1, N, K, c->d.part, c->d.n_rows, g.batch, c->stream, p, &c->launches));
+    if (prof) {
+        CK(cudaEventRecord(c->prof_ev[c->prof_used + 1], c->stream));
+        c->prof_used += 2;
+        c->prof_bytes += 2.0 * (double)N * (double)K;
+    }
+    return PACER_OK;
+}
+
+// Runs model `which` on the rows `kind` selects.  head: LM head + argmax;
+// hidden: keep the fp32 final-norm output.
+static int run_forward(pacer_ctx *c, int which, const Geom &g, int kind, int aux, bool head, bool hidden) {
+    ModelDev &m = c->model[which];
+    DevPtrs &d = c->d;
+    cudaStream_t st = c->stream;
+    const pacer_model_cfg &k = m.cfg;
+    const int dm = k.d_model, F = k.d_ffn, hh = k.n_heads * m.hd;
+    GemmPlan p;
+    int rc;
+    k_begin<<<g.rtot, ROW_THREADS, 0, st>>>(d, m, g, kind, aux);
+    LAUNCH_CHECK();
+    for (int l = 0; l < k.n_layers; ++l) {
+        if ((rc = fwd_gemm(c, d.xn, g, m.wqkv + (size_t)l * m.qrows * dm, nullptr, 0, m.qrows, dm, &p))) return rc;
+        k_rope_append<<<g.rtot, ROW_THREADS, 0, st>>>(d, m, g, l, p.S);
+        LAUNCH_CHECK();
+        CK(attention_launch(d, m, g, l, st));
+        ++c->launches;
+        if ((rc = fwd_gemm(c, d.att, g, m.wo + (size_t)l * dm * hh, nullptr, 0, dm, hh, &p))) return rc;
+        k_add_norm<<<g.rtot, ROW_THREADS, 0, st>>>(d, g, dm, k.rms_eps, m.norm2 + (size_t)l * dm, p.S, 0);
+        LAUNCH_CHECK();
+        if ((rc = fwd_gemm(c, d.xn, g, m.wgate + (size_t)l * F * dm, m.wup + (size_t)l * F * dm, F, 2 * F, dm, &p))) return rc;
+        k_swiglu<<<dim3((F + ROW_THREADS - 1) / ROW_THREADS, g.rtot), ROW_THREADS, 0, st>>>(d, g, F, p.S);
+        LAUNCH_CHECK();
+        if ((rc = fwd_gemm(c, d.act, g, m.wdown + (size_t)l * dm * F, nullptr, 0, dm, F, &p))) return rc;
+        const bool last = l == k.n_layers - 1;
+        if (!last) {
+            k_add_norm<<<g.rtot, ROW_THREADS, 0, st>>>(d, g, dm, k.rms_eps, m.norm1 + (size_t)(l + 1) * dm, p.S, 0);
+            LAUNCH_CHECK();
+        } else if (head || hidden) {
+            k_add_norm<<<g.rtot, ROW_THREADS, 0, st>>>(d, g, dm, k.rms_eps, m.normf, p.S, hidden ? 1 : 0);
+            LAUNCH_CHECK();
+        }
+    }
+    if (head) {
+        if ((rc = fwd_gemm(c, d.xn, g, m.head, nullptr, 0, k.vocab, dm, &p))) return rc;
+        k_head_finish<<<g.rtot, HEAD_THREADS, 0, st>>>(d, m, g, kind, p.S);
+        LAUNCH_CHECK();
+    }
+    return PACER_OK;
+}
+
+static int need_ready(pacer_ctx *c, bool prefilled) {
+    if (!c) return fail(nullptr, PACER_EINVAL, "ctx is null");
+    for (int i = 0; i < 3; ++i)
+        if (!c->model[i].loaded) return fail(c, PACER_ESTATE, "weights of all three models must be loaded first");
+    if (prefilled && !c->prefilled) return fail(c, PACER_ESTATE, "pacer_prefill must run first");
+    return PACER_OK;
+}
+
+// ------------------------------------------------------------------ stages
+
+static int start_run(pacer_ctx *c, const int32_t *prompt, int batch, int n_prompt, int max_new, int gamma_max,
+                     float threshold, int mode, uint64_t seed) {
+    const pacer_cfg &k = c->cfg;
+    if (!prompt || batch < 1 || batch > k.max_batch || n_prompt < 1 || max_new < 1)
+        return fail(c, PACER_EINVAL, "prefill: bad batch / n_prompt / max_new");
+    const int gm = gamma_max / k.block_b * k.block_b;
+    if (gm < k.block_b || gm > k.gamma_cap) return fail(c, PACER_EINVAL, "prefill: gamma_max outside [block_b, gamma_cap]");
+    if ((int64_t)n_prompt + max_new + k.gamma_cap + 2 > k.max_ctx) return fail(c, PACER_EINVAL, "prefill: n_prompt + max_new + gamma_cap + 2 exceeds max_ctx");
+    if (mode != PACER_GREEDY && mode != PACER_SAMPLE) return fail(c, PACER_EINVAL, "prefill: bad mode");
+    if (mode == PACER_SAMPLE) return fail(c, PACER_EUNSUPPORTED, "sampling mode is not built yet");
+    for (int s = 0; s < batch; ++s)
+        for (int i = 0; i < n_prompt; ++i)
+            if (prompt[(size_t)s * n_prompt + i] < 0 || prompt[(size_t)s * n_prompt + i] >= k.target.vocab)
+                return fail(c, PACER_EINVAL, "prefill: token id out of range");
+    set_geoms(c, batch);
+    std::vector<SeqState> hs(k.max_batch);
+    memset(hs.data(), 0, sizeof(SeqState) * hs.size());
+    for (int s = 0; s < batch; ++s) {
+        SeqState &st = hs[s];
+        st.P = n_prompt; st.n_prompt = n_prompt; st.max_new = max_new; st.gamma_max = gm; st.t0 = threshold;
+        st.t_k = threshold; st.mode = mode; st.seed = seed; st.active = 1; st.drafting = 1;
+    }
+    CK(cudaMemcpyAsync(c->d.st, hs.data(), sizeof(SeqState) * hs.size(), cudaMemcpyHostToDevice, c->stream));
+    CK(cudaMemcpy2DAsync(c->d.x, sizeof(int32_t) * k.max_ctx, prompt, sizeof(int32_t) * n_prompt, sizeof(int32_t) * n_prompt,
+                         batch, cudaMemcpyHostToDevice, c->stream));
+    CK(cudaStreamSynchronize(c->stream));        // hs is a local
+    return PACER_OK;
+}
+
+static int prefill_models(pacer_ctx *c, int n_prompt, bool target, bool draft_and_mb) {
+    const Geom &g = c->g_verify;
+    for (int c0 = 0; c0 < n_prompt - 1; c0 += g.rps) {
+        int rc;
+        if (target) {
+            if ((rc = run_forward(c, PACER_TARGET, g, KIND_PREFILL, c0, false, false))) return rc;
+            k_prefill_end<<<1, 64, 0, c->stream>>>(c->d, g, PACER_TARGET);
+            LAUNCH_CHECK();
+        }
+        if (draft_and_mb) {
+            if ((rc = run_forward(c, PACER_DRAFT, g, KIND_PREFILL, c0, false, true))) return rc;
+            k_prefill_end<<<1, 64, 0, c->stream>>>(c->d, g, PACER_DRAFT);
+            LAUNCH_CHECK();
+            if ((rc = run_forward(c, PACER_PREVERIFY, g, KIND_PREFILL_B, c0, false, false))) return rc;
+            k_prefill_end<<<1, 64, 0, c->stream>>>(c->d, g, PACER_PREVERIFY);
+            LAUNCH_CHECK();
+        }
+    }
+    return PACER_OK;
+}
+
+extern "C" int pacer_prefill(pacer_ctx *c, const int32_t *prompt, int batch, int n_prompt, int max_new, int gamma_max,
+                             float threshold, int mode, uint64_t seed) {
+    int rc = need_ready(c, false);
+    if (rc) return rc;
+    if ((rc = start_run(c, prompt, batch, n_prompt, max_new, gamma_max, threshold, mode, seed))) return rc;
+    if ((rc = prefill_models(c, n_prompt, true, true))) return rc;
+    c->prefilled = 1;
+    return PACER_OK;
+}
+
+extern "C" int pacer_draft_step(pacer_ctx *c) {
+    int rc = need_ready(c, true);
+    if (rc) return rc;
+    if ((rc = run_forward(c, PACER_DRAFT, c->g_draft, KIND_DRAFT, 0, true, true))) return rc;
+    k_draft_end<<<c->batch, 256, 0, c->stream>>>(c->d, c->g_draft, c->cfg.draft.d_model);
+    LAUNCH_CHECK();
+    return PACER_OK;
+}
+
+extern "C" int pacer_preverify(pacer_ctx *c) {
+    int rc = need_ready(c, true);
+    if (rc) return rc;
+    if ((rc = run_forward(c, PACER_PREVERIFY, c->g_mb, KIND_MB, 0, false, true))) return rc;
+    k_mb_end<<<c->batch, 256, 0, c->stream>>>(c->d, c->model[PACER_PREVERIFY], c->g_mb);
+    LAUNCH_CHECK();
+    return PACER_OK;
+}
+
+extern "C" int pacer_verify(pacer_ctx *c) {
+    int rc = need_ready(c, true);
+    if (rc) return rc;
+    return run_forward(c, PACER_TARGET, c->g_verify, KIND_VERIFY, 0, true, false);
+}
+
+extern "C" int pacer_accept_rollback(pacer_ctx *c) {
+    int rc = need_ready(c, true);
+    if (rc) return rc;
+    k_accept_greedy<<<1, 64, 0, c->stream>>>(c->d, c->g_verify);
+    LAUNCH_CHECK();
+    return PACER_OK;
+}
+
+extern "C" int pacer_read_state(pacer_ctx *c, pacer_seq_state *out, int batch) {
+    if (!c || !out || batch < 1 || batch > c->cfg.max_batch) return fail(c, PACER_EINVAL, "pacer_read_state: bad argument");
+    std::vector<SeqState> hs(batch);
+    CK(cudaMemcpyAsync(hs.data(), c->d.st, sizeof(SeqState) * batch, cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    for (int s = 0; s < batch; ++s) {
+        const SeqState &a = hs[s];
+        pacer_seq_state &o = out[s];
+        o.P = a.P; o.len_T = a.len_T; o.len_D = a.len_D; o.len_B = a.len_B; o.gamma = a.gamma; o.k_round = a.k_round;
+        o.t_k = a.t_k; o.drafting = a.drafting; o.finished = a.finished; o.n_steps = a.n_steps; o.last_n = a.last_n;
+        o.last_next = a.last_next; o.n_pend = a.n_pend; o.err = a.err; o.n_draft_fwd = a.n_draft_fwd;
+        o.n_mb_calls = a.n_mb_calls; o.n_target_fwd = a.n_target_fwd;
+    }
+    return PACER_OK;
+}
+
+extern "C" int pacer_read_buffer(pacer_ctx *c, int which, void *host_dst, size_t bytes) {
+    if (!c || !host_dst || which < 0 || which >= 16 || !c->buf_bytes[which]) return fail(c, PACER_EINVAL, "pacer_read_buffer: bad buffer");
+    if (bytes > c->buf_bytes[which]) return fail(c, PACER_EINVAL, "pacer_read_buffer: more bytes than the buffer holds");
+    CK(cudaMemcpyAsync(host_dst, c->buf_ptr[which], bytes, cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    return PACER_OK;
+}
+
+extern "C" int pacer_profile_begin(pacer_ctx *c) {
+    if (!c) return fail(nullptr, PACER_EINVAL, "ctx is null");
+    while (c->prof_ev.size() < 8192) {
+        cudaEvent_t e;
+        CK(cudaEventCreate(&e));
+        c->prof_ev.push_back(e);
+    }
+    c->prof_used = 0;
+    c->prof_bytes = 0;
+    c->prof_on = 1;
+    return PACER_OK;
+}
+
+extern "C" int pacer_profile_end(pacer_ctx *c, double *gemm_ms, double *gemm_weight_bytes, int64_t *gemm_launches) {
+    if (!c || !gemm_ms || !gemm_weight_bytes || !gemm_launches) return fail(c, PACER_EINVAL, "pacer_profile_end: null argument");
+    c->prof_on = 0;
+    CK(cudaStreamSynchronize(c->stream));
+    double ms = 0;
+    for (size_t i = 0; i + 1 < c->prof_used; i += 2) {
+        float t;
+        CK(cudaEventElapsedTime(&t, c->prof_ev[i], c->prof_ev[i + 1]));
+        ms += t;
+    }
+    *gemm_ms = ms;
+    *gemm_weight_bytes = c->prof_bytes;
+    *gemm_launches = (int64_t)(c->prof_used / 2);
+    return PACER_OK;
+}
+
+// ------------------------------------------------------------------ whole loops
+
+static int enqueue_step(pacer_ctx *c, int gamma_max) {
+    int rc;
+    const int b = c->cfg.block_b;
+    for (int blk = 0; blk < gamma_max / b; ++blk) {
+        for (int i = 0; i < b; ++i)
+            if ((rc = pacer_draft_step(c))) return rc;
+        if ((rc = pacer_preverify(c))) return rc;
+    }
+    if ((rc = pacer_verify(c))) return rc;
+    return pacer_accept_rollback(c);
+}
+
+static int collect(pacer_ctx *c, int batch, int max_new, int n_prompt, int32_t *out_tokens, int32_t *out_n_steps,
+                   int32_t *out_draft_len, int32_t *out_accept_len, pacer_stats *stats, int64_t launches0) {
+    const pacer_cfg &k = c->cfg;
+    std::vector<SeqState> hs(batch);
+    CK(cudaMemcpyAsync(hs.data(), c->d.st, sizeof(SeqState) * batch, cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaMemcpy2DAsync(out_tokens, sizeof(int32_t) * max_new, c->d.x + n_prompt, sizeof(int32_t) * k.max_ctx,
+                         sizeof(int32_t) * max_new, batch, cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    int64_t nd = 0, nm = 0, nt = 0, ns = 0, ng = 0;
+    for (int s = 0; s < batch; ++s) {
+        const SeqState &a = hs[s];
+        if (a.err) return fail(c, PACER_EDEVICE, "device status word set");
+        nd += a.n_draft_fwd; nm += a.n_mb_calls; nt += a.n_target_fwd; ns += a.n_steps; ng += a.P - a.n_prompt;
+        if (out_n_steps) out_n_steps[s] = a.n_steps;
+        if (out_draft_len && out_accept_len) {
+            for (int i = 0; i < max_new; ++i) out_draft_len[(size_t)s * max_new + i] = out_accept_len[(size_t)s * max_new + i] = -1;
+            const int n = a.n_steps < max_new ? a.n_steps : max_new;
+            if (n > 0) {
+                CK(cudaMemcpy(out_draft_len + (size_t)s * max_new, c->d.draft_len + (size_t)s * c->d.max_steps, sizeof(int32_t) * n, cudaMemcpyDeviceToHost));
+                CK(cudaMemcpy(out_accept_len + (size_t)s * max_new, c->d.accept_len + (size_t)s * c->d.max_steps, sizeof(int32_t) * n, cudaMemcpyDeviceToHost));
+            }
+        }
+    }
+    if (stats) {
+        stats->n_draft_fwd = nd; stats->n_mb_calls = nm; stats->n_target_fwd = nt; stats->n_steps = ns; stats->n_generated = ng;
+        stats->n_kernel_launches = c->launches - launches0;
+        CK(cudaEventElapsedTime(&stats->ms_prefill, c->ev[0], c->ev[1]));
+        CK(cudaEventElapsedTime(&stats->ms_decode, c->ev[1], c->ev[2]));
+    }
+    return PACER_OK;
+}
+
+extern "C" int pacer_generate(pacer_ctx *c, const int32_t *prompt, int batch, int n_prompt, int max_new, int gamma_max,
+                              float threshold, int mode, uint64_t seed, int32_t *out_tokens, int32_t *out_n_steps,
+                              int32_t *out_draft_len, int32_t *out_accept_len, pacer_stats *stats) {
+    int rc = need_ready(c, false);
+    if (rc) return rc;
+    if (!out_tokens) return fail(c, PACER_EINVAL, "pacer_generate: out_tokens is null");
+    if ((rc = start_run(c, prompt, batch, n_prompt, max_new, gamma_max, threshold, mode, seed))) return rc;
+    CK(cudaEventRecord(c->ev[0], c->stream));
+    if ((rc = prefill_models(c, n_prompt, true, true))) return rc;
+    c->prefilled = 1;
+    CK(cudaEventRecord(c->ev[1], c->stream));
+    const int64_t launches0 = c->launches;
+    const int gm = gamma_max / c->cfg.block_b * c->cfg.block_b;
+    std::vector<SeqState> hs(batch);
+    for (int step = 0; step < max_new; ++step) {
+        if ((rc = enqueue_step(c, gm))) return rc;
+        CK(cudaMemcpyAsync(hs.data(), c->d.st, sizeof(SeqState) * batch, cudaMemcpyDeviceToHost, c->stream));
+        CK(cudaStreamSynchronize(c->stream));
+        bool all = true;
+        for (int s = 0; s < batch; ++s) all = all && hs[s].finished;
+        if (all) break;
+    }
+    CK(cudaEventRecord(c->ev[2], c->stream));
+    return collect(c, batch, max_new, n_prompt, out_tokens, out_n_steps, out_draft_len, out_accept_len, stats, launches0);
+}
+
+extern "C" int pacer_generate_ar(pacer_ctx *c, const int32_t *prompt, int batch, int n_prompt, int max_new, int mode,
+                                 uint64_t seed, int32_t *out_tokens, pacer_stats *stats) {
+    int rc = need_ready(c, false);
+    if (rc) return rc;
+    if (!out_tokens) return fail(c, PACER_EINVAL, "pacer_generate_ar: out_tokens is null");
+    if ((rc = start_run(c, prompt, batch, n_prompt, max_new, c->cfg.block_b, -1.f, mode, seed))) return rc;
+    CK(cudaEventRecord(c->ev[0], c->stream));
+    if ((rc = prefill_models(c, n_prompt, true, false))) return rc;
+    c->prefilled = 0;                     // draft and M_B caches were not filled
+    CK(cudaEventRecord(c->ev[1], c->stream));
+    const int64_t launches0 = c->launches;
+    for (int i = 0; i < max_new; ++i) {
+        if ((rc = run_forward(c, PACER_TARGET, c->g_ar, KIND_AR, 0, true, false))) return rc;
+        k_ar_end<<<1, 64, 0, c->stream>>>(c->d, c->g_ar);
+        LAUNCH_CHECK();
+    }
+    CK(cudaEventRecord(c->ev[2], c->stream));
+    return collect(c, batch, max_new, n_prompt, out_tokens, nullptr, nullptr, nullptr, stats, launches0);
+}
+
+// ------------------------------------------------------------------ stand-alone product
+
+__global__ void k_to_frag(const bf16 *x, bf16 *xf, int rows, int K, int nt) {
+    const int r = blockIdx.y, k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k >= K) return;
+    xf[xfrag_index(r, k, nt)] = r < rows ? x[(size_t)r * K + k] : __float2bfloat16(0.f);
+}
+
+__global__ void k_sum_part(const float *part, float *y, int rows, int N, int S, int rpad) {
+    const int r = blockIdx.y, n = blockIdx.x * blockDim.x + threadIdx.x;
+    if (n >= N || r >= rows) return;
+    float v = 0.f;
+    for (int s = 0; s < S; ++s) v += part[((size_t)s * rpad + r) * N + n];
+    y[(size_t)r * N + n] = v;
+}
+
+extern "C" size_t pacer_linear_scratch_bytes(int rows, int N, int K) {
+    if (rows < 1 || rows > 32 || N < 1 || K < 32 || K % 32) return 0;
+    const int nt = (rows + 7) / 8;
+    GemmPlan p = gemm_plan(N, K, nt);
+    size_t xf = ((size_t)nt * 8 * K * sizeof(bf16) + 255) / 256 * 256;
+    return xf + (size_t)p.S * nt * 8 * N * sizeof(float);
+}
+
+extern "C" int pacer_linear(const void *x, const void *w, float *y, int rows, int N, int K, void *scratch,
+                            size_t scratch_bytes, void *cuda_stream) {
+    pacer_ctx *c = nullptr;
+    const size_t need = pacer_linear_scratch_bytes(rows, N, K);
+    if (!x || !w || !y || !scratch || need == 0) return fail(nullptr, PACER_EINVAL, "pacer_linear: bad argument");
+    if (scratch_bytes < need) return fail(nullptr, PACER_ENOMEM, "pacer_linear: scratch too small");
+    if (((uintptr_t)w & 15) || ((uintptr_t)scratch & 255)) return fail(nullptr, PACER_EINVAL, "pacer_linear: misaligned pointer");
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    const int nt = (rows + 7) / 8;
+    bf16 *xf = (bf16 *)scratch;
+    float *part = (float *)((char *)scratch + ((size_t)nt * 8 * K * sizeof(bf16) + 255) / 256 * 256);
+    k_to_frag<<<dim3((K + 255) / 256, nt * 8), 256, 0, st>>>((const bf16 *)x, xf, rows, K, nt);
+    CK(cudaGetLastError());
+    GemmPlan p;
+    CK(gemm_run(xf, nt, (const bf16 *)w, nullptr, 0, N, K, part, nullptr, 0, st, &p, nullptr));
+    k_sum_part<<<dim3((N + 255) / 256, rows), 256, 0, st>>>(part, y, rows, N, p.S, nt * 8);
+    CK(cudaGetLastError());
+    return PACER_OK;
+}
