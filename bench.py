@@ -120,6 +120,41 @@ def oracle_sample(cfg: synth.PairConfig, pair_cpu, prompt, n_prompt_s, max_new_s
     return made / dt, made, dt
 
 
+def verify_forward_numbers(ctx, cfg, prompt, n_ver, n_warm):
+    """Times the target verify forward with a full draft window (gamma_cap + 1 rows): the whole forward with
+    CUDA events on the context's stream, and its weight-streaming products one by one (pacer_profile_*)."""
+    ctx.pacer_prefill(prompt, cfg.max_new, cfg.gamma_max, -1.0)
+    for _ in range(cfg.gamma_cap // cfg.block_b):
+        for _ in range(cfg.block_b):
+            ctx.pacer_draft_step()
+        ctx.pacer_preverify()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for _ in range(n_warm):
+        ctx.pacer_verify()            # same rows every time: the state does not advance without accept
+    e0.record(ctx.stream)
+    for _ in range(n_ver):
+        ctx.pacer_verify()
+    e1.record(ctx.stream)
+    torch.cuda.synchronize()
+    ver_ms = e0.elapsed_time(e1) / n_ver
+    ctx.pacer_profile_begin()
+    for _ in range(n_ver):
+        ctx.pacer_verify()
+    gemm_ms, gemm_bytes, gemm_n = ctx.pacer_profile_end()
+    peak, peak_kind = _peaks()
+    vbytes = verify_bytes(cfg, cfg.n_prompt - 1, cfg.gamma_cap + 1)
+    gemm_gbs = gemm_bytes / (gemm_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": "k_gemm_skinny", "achieved": gemm_gbs, "peak": peak, "unit": "GB/s",
+                "frac": gemm_gbs / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
+                "launches_timed": gemm_n, "bytes_per_launch_avg": gemm_bytes / max(1, gemm_n),
+                "ms_per_launch_avg": gemm_ms / max(1, gemm_n)}
+    verify = {"ms": ver_ms, "algorithmic_gb": vbytes / 1e9, "achieved_gbs": vbytes / (ver_ms * 1e-3) / 1e9,
+              "frac_of_measured_peak": vbytes / (ver_ms * 1e-3) / 1e9 / peak,
+              "frac_of_8tbs": vbytes / (ver_ms * 1e-3) / 1e9 / 8000.0, "rows": cfg.gamma_cap + 1}
+    return {"roofline": roofline, "verify_forward": verify}
+
+
 def pair_to_cpu(pair):
     return {k: ({n: t.cpu() for n, t in v.items()} if isinstance(v, dict) else v.cpu()) for k, v in pair.items()}
 
@@ -133,12 +168,21 @@ def main():
     ap.add_argument("--impl", default="pacer", choices=["pacer", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-sample-new", type=int, default=4)
+    ap.add_argument("--only", default="all", choices=["all", "verify"],
+                    help="verify: short prefill, one full draft window, then timed verify forwards only "
+                         "(the small, few-launch command the ncu captures use)")
+    ap.add_argument("--layers", type=int, default=0, help="with --only verify: keep this many target layers")
+    ap.add_argument("--n-prompt", type=int, default=0, help="with --only verify: prompt length override")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     cfg = synth.CONFIGS[args.config]
+    if args.only == "verify":
+        import dataclasses
+        tgt = dataclasses.replace(cfg.target, n_layers=args.layers) if args.layers else cfg.target
+        cfg = dataclasses.replace(cfg, target=tgt, n_prompt=args.n_prompt or cfg.n_prompt)
     t0 = PACER_T0
     workload = {"workload": f"{cfg.name}: target {cfg.target.n_layers}L d={cfg.target.d_model}, draft "
                             f"{cfg.draft.n_layers}L d={cfg.draft.d_model}, prompt {cfg.n_prompt}, new {cfg.max_new}, "
@@ -189,6 +233,12 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    if args.only == "verify":
+        if rank == 0:
+            print(json.dumps({"only": "verify", "config": workload, **verify_forward_numbers(ctx, cfg, prompt, args.steps,
+                                                                                             args.warmup)}))
+        return
+
     for _ in range(args.warmup):
         ctx.pacer_generate(prompt, cfg.max_new, cfg.gamma_max, t0)
     sampler = ClockSampler(local_rank)
@@ -218,37 +268,8 @@ def main():
         fixed[g] = cfg.max_new / (s2["ms_decode"] * 1e-3)
     best_g = max(fixed, key=fixed.get)
 
-    # verify forward: whole-forward time and kernel-level GEMM time, live
-    ctx.pacer_prefill(prompt, cfg.max_new, cfg.gamma_max, -1.0)
-    for _ in range(cfg.gamma_cap // cfg.block_b):     # a full window of drafts, so the verify has gamma_cap + 1 rows
-        for _ in range(cfg.block_b):
-            ctx.pacer_draft_step()
-        ctx.pacer_preverify()
-    torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    n_ver = 10
-    for _ in range(3):
-        ctx.pacer_verify()
-    e0.record(ctx.stream)
-    for _ in range(n_ver):
-        ctx.pacer_verify()            # same rows every time: the state does not advance without accept
-    e1.record(ctx.stream)
-    torch.cuda.synchronize()
-    ver_ms = e0.elapsed_time(e1) / n_ver
-    ctx.pacer_profile_begin()
-    for _ in range(n_ver):
-        ctx.pacer_verify()
-    gemm_ms, gemm_bytes, gemm_n = ctx.pacer_profile_end()
-    peak, peak_kind = _peaks()
-    vbytes = verify_bytes(cfg, cfg.n_prompt - 1, cfg.gamma_cap + 1)
-    gemm_gbs = gemm_bytes / (gemm_ms * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": "k_gemm_skinny", "achieved": gemm_gbs, "peak": peak, "unit": "GB/s",
-                "frac": gemm_gbs / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
-                "launches_timed": gemm_n, "bytes_per_launch_avg": gemm_bytes / max(1, gemm_n),
-                "ms_per_launch_avg": gemm_ms / max(1, gemm_n)}
-    verify = {"ms": ver_ms, "algorithmic_gb": vbytes / 1e9, "achieved_gbs": vbytes / (ver_ms * 1e-3) / 1e9,
-              "frac_of_measured_peak": vbytes / (ver_ms * 1e-3) / 1e9 / peak,
-              "frac_of_8tbs": vbytes / (ver_ms * 1e-3) / 1e9 / 8000.0, "rows": cfg.gamma_cap + 1}
+    vf = verify_forward_numbers(ctx, cfg, prompt, 10, 3)
+    roofline, verify = vf["roofline"], vf["verify_forward"]
 
     val_local = tok / (dec_ms * 1e-3)
     e2e_local = tok / e2e_s
