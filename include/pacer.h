@@ -217,6 +217,29 @@ size_t pacer_linear_scratch_bytes(int rows, int N, int K);
 int pacer_linear(const void *x, const void *w, float *y, int rows, int N, int K, void *scratch,
                  size_t scratch_bytes, void *cuda_stream);
 
+/* The same product as pacer_linear for callers that cannot allocate device memory.
+ * (The paper has no counterpart: this is a service entry point of the library.)
+ * Who needs it: a serving process that handed all device memory to its own arena
+ * at start-up, or a plug-in host without an allocator of its own, has nothing to
+ * offer as `scratch`, and a cudaMalloc inside the decode loop would stall the whole
+ * device (it synchronises) or simply fail once the arena owns the memory.  Here the
+ * scratch is a fixed array of PACER_LINEAR_STATIC_BYTES bytes inside the library
+ * image; every GPU that loads the library holds it until the process exits.
+ *   - x, w, y, rows, N, K, cuda_stream: exactly as pacer_linear; inputs and the
+ *     output remain caller-owned device memory.
+ *   - Shapes whose pacer_linear_scratch_bytes(rows, N, K) exceeds
+ *     PACER_LINEAR_STATIC_BYTES are refused with PACER_ENOMEM before any launch.
+ *   - No cudaMalloc, cudaFree or allocating library routine is called, ever.
+ *   - The first call on each device looks up the device address of the array
+ *     (cudaGetSymbolAddress, with that device current) and remembers it; make that
+ *     first call before starting any stream capture on the device.
+ *   - All calls on one device share the one array, which keeps whatever the last
+ *     call left in it.  Nothing in it has to start at zero: the kernels overwrite
+ *     every element they later read.  Two calls that overlap on the GPU (different
+ *     streams, no ordering between them) race on the array; order them. */
+#define PACER_LINEAR_STATIC_BYTES (4u << 20)
+int pacer_linear_static(const void *x, const void *w, float *y, int rows, int N, int K, void *cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -88,6 +88,8 @@ _lib.pacer_profile_end.argtypes = [_P, C.POINTER(C.c_double), C.POINTER(C.c_doub
 _lib.pacer_linear_scratch_bytes.restype = C.c_size_t
 _lib.pacer_linear_scratch_bytes.argtypes = [C.c_int, C.c_int, C.c_int]
 _lib.pacer_linear.argtypes = [_P, _P, _P, C.c_int, C.c_int, C.c_int, _P, C.c_size_t, _P]
+_lib.pacer_linear_static.argtypes = [_P, _P, _P, C.c_int, C.c_int, C.c_int, _P]
+PACER_LINEAR_STATIC_BYTES = 4 << 20
 
 
 class PacerError(RuntimeError):
@@ -99,7 +101,7 @@ def exported_symbols():
     return ["pacer_strerror", "pacer_last_error", "pacer_workspace_bytes", "pacer_create", "pacer_destroy",
             "pacer_load_weights", "pacer_prefill", "pacer_draft_step", "pacer_preverify", "pacer_verify",
             "pacer_accept_rollback", "pacer_read_state", "pacer_read_buffer", "pacer_generate", "pacer_generate_ar",
-            "pacer_profile_begin", "pacer_profile_end", "pacer_linear_scratch_bytes", "pacer_linear"]
+            "pacer_profile_begin", "pacer_profile_end", "pacer_linear_scratch_bytes", "pacer_linear", "pacer_linear_static"]
 
 
 def _model_cfg(s) -> ModelCfg:
@@ -264,6 +266,24 @@ def pacer_linear(x: torch.Tensor, w: torch.Tensor) -> torch.Tensor:
     if rc != 0:
         raise PacerError(f"pacer_linear: {_lib.pacer_strerror(rc).decode()}: {_lib.pacer_last_error(None).decode()}")
     return y
+
+
+def pacer_linear_static(x: torch.Tensor, w: torch.Tensor, out: torch.Tensor) -> torch.Tensor:
+    """y = x @ w.T written into the caller's `out` (f32 [rows][N]) with the library's built-in scratch: the call
+    itself allocates nothing on the device, for callers whose device memory is all spoken for.  Shapes that need
+    more than PACER_LINEAR_STATIC_BYTES of scratch raise PacerError.  Calls on one device share the scratch, so
+    they must not overlap on the GPU."""
+    assert x.is_cuda and w.is_cuda and out.is_cuda and x.dtype == torch.bfloat16 and w.dtype == torch.bfloat16
+    assert x.is_contiguous() and w.is_contiguous() and out.is_contiguous() and out.dtype == torch.float32
+    rows, K = x.shape
+    N = w.shape[0]
+    assert tuple(out.shape) == (rows, N)
+    with torch.cuda.device(x.device):
+        rc = _lib.pacer_linear_static(x.data_ptr(), w.data_ptr(), out.data_ptr(), rows, N, K,
+                                      torch.cuda.current_stream(x.device).cuda_stream)
+    if rc != 0:
+        raise PacerError(f"pacer_linear_static: {_lib.pacer_strerror(rc).decode()}: {_lib.pacer_last_error(None).decode()}")
+    return out
 
 
 def load_pair(ctx: Context, pair: dict):

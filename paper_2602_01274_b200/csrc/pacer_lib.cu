@@ -690,3 +690,28 @@ extern "C" int pacer_linear(const void *x, const void *w, float *y, int rows, in
     CK(cudaGetLastError());
     return PACER_OK;
 }
+
+// ------------------------------------------------------------------ product without caller scratch
+
+// Scratch of pacer_linear_static.  In host code this name is only a handle for
+// cudaGetSymbolAddress; the device address is looked up once per device.
+static __device__ __align__(256) unsigned char g_linear_static_scratch[PACER_LINEAR_STATIC_BYTES];
+static void *g_linear_static_ptr[64];
+
+extern "C" int pacer_linear_static(const void *x, const void *w, float *y, int rows, int N, int K, void *cuda_stream) {
+    pacer_ctx *c = nullptr;
+    const size_t need = pacer_linear_scratch_bytes(rows, N, K);
+    if (!x || !w || !y || need == 0) return fail(nullptr, PACER_EINVAL, "pacer_linear_static: bad argument");
+    if (need > (size_t)PACER_LINEAR_STATIC_BYTES)
+        return fail(nullptr, PACER_ENOMEM, "pacer_linear_static: shape needs more than PACER_LINEAR_STATIC_BYTES of scratch");
+    int dev = -1;
+    CK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return fail(nullptr, PACER_EUNSUPPORTED, "pacer_linear_static: device index out of range");
+    if (!g_linear_static_ptr[dev]) {
+        void *p = nullptr;
+        CK(cudaGetSymbolAddress(&p, g_linear_static_scratch));
+        if (!p) return fail(nullptr, PACER_ECUDA, "pacer_linear_static: no device address for the scratch array");
+        g_linear_static_ptr[dev] = p;
+    }
+    return pacer_linear(x, w, y, rows, N, K, g_linear_static_ptr[dev], (size_t)PACER_LINEAR_STATIC_BYTES, cuda_stream);
+}
