@@ -123,6 +123,7 @@ struct Ctx {
     int32_t *row_pos, *row_tok;    // [MAX_ROWS]
     int32_t *n_rows;               // [MAX_ROWS] per sequence
     float *inv_rms;                // [MAX_ROWS]
+    int32_t *flag;                 // block-wide scratch word
     // registers
     unsigned long long bar_target; // used by thread 0
     int warp, lane, cta, ncta;

@@ -1,0 +1,346 @@
+// The forward kernel itself, the tails that take the loop's decisions, the host
+// planner that cuts the projections into items, and the cooperative launch.
+#pragma once
+#include <algorithm>
+#include <vector>
+
+#include "fwd_attention.cuh"
+
+namespace fwd {
+
+// ------------------------------------------------------------------ tails (one block per sequence)
+
+__device__ __forceinline__ float hidden_at(const Args &a, const Ctx &c, int r, int i) {
+    return __ldcg(a.d.xres + (size_t)r * a.m.cfg.d_model + i) * c.inv_rms[r] * __bfloat162float(a.m.normf[i]);
+}
+
+// End of one draft forward (Eq. 6): y_i, h_i queued for the pre-verification model, cache length.
+__device__ __forceinline__ void tail_draft(Ctx &c, const Args &a, int s) {
+    const DevPtrs &d = a.d;
+    SeqState &st = d.st[s];
+    const int n_in = c.n_rows[s], dm = a.m.cfg.d_model;
+    if (n_in == 0) return;
+    const int gamma = st.gamma, n_pend = st.n_pend, r_last = s * a.g.rps + n_in - 1;
+    for (int jj = 0; jj < n_in; ++jj) {
+        float *dst = d.hpend + ((size_t)s * (d.block_b + 1) + n_pend + jj) * dm;
+        for (int i = threadIdx.x; i < dm; i += THREADS) dst[i] = hidden_at(a, c, s * a.g.rps + jj, i);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int jj = 0; jj < n_in; ++jj)
+            d.hpend_e[s * (d.block_b + 1) + n_pend + jj] = (jj == n_in - 1) ? gamma + 1 : 0;
+        d.y[(size_t)s * d.gamma_cap + gamma] = d.row_arg[r_last];
+        st.n_pend = n_pend + n_in;
+        st.gamma = gamma + 1;
+        st.len_D += n_in;
+        st.n_draft_fwd += 1;
+    }
+}
+
+// End of a pre-verification call (Eq. 7 + the block test of Algorithm 1).
+__device__ __forceinline__ void tail_mb(Ctx &c, const Args &a, int s) {
+    const DevPtrs &d = a.d;
+    SeqState &st = d.st[s];
+    const int n = c.n_rows[s], dm = a.m.cfg.d_model;
+    if (n == 0) return;
+    float *red = reinterpret_cast<float *>(c.scratch);
+    for (int j = 0; j < n; ++j) {
+        const int r = s * a.g.rps + j, e = c.row_tok[r];
+        if (e == 0) continue;
+        float z0 = 0.f, z1 = 0.f;
+        for (int i = threadIdx.x; i < dm; i += THREADS) {
+            const float hv = hidden_at(a, c, r, i);
+            z0 += hv * __bfloat162float(a.m.head_b[i]);
+            z1 += hv * __bfloat162float(a.m.head_b[dm + i]);
+        }
+        z0 = block_sum(z0, red);
+        z1 = block_sum(z1, red);
+        if (threadIdx.x == 0) d.alpha[(size_t)s * d.gamma_cap + e - 1] = 1.f / (1.f + expf(z0 - z1));
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const int b = d.block_b, gamma = st.gamma;
+        const float *ab = d.alpha + (size_t)s * d.gamma_cap + (gamma - b);
+        float stat;
+        if (d.criterion == 1) { stat = ab[0]; for (int i = 1; i < b; ++i) stat = fminf(stat, ab[i]); }
+        else if (d.criterion == 2) stat = ab[b - 1];
+        else { stat = 0.f; for (int i = 0; i < b; ++i) stat += ab[i]; stat /= (float)b; }
+        int stop = 0;
+        if (st.t0 >= 0.f && stat <= st.t_k) stop = 1;
+        if (gamma + b > st.gamma_max) stop = 1;
+        if (stop) st.drafting = 0;
+        else { st.t_k = st.t_k * d.rho; st.k_round += 1; }
+        st.len_B += n;
+        st.n_pend = 0;
+        st.n_mb_calls += 1;
+    }
+}
+
+// End of a prefill chunk: the caches grew; the draft's hidden rows are the
+// history rows the pre-verification model is prefilled with.
+__device__ __forceinline__ void tail_prefill(Ctx &c, const Args &a, int s, int which) {
+    const DevPtrs &d = a.d;
+    const int n = c.n_rows[s], dm = a.m.cfg.d_model;
+    if (n == 0) return;
+    if (which == PACER_DRAFT)
+        for (int j = 0; j < n; ++j) {
+            const int r = s * a.g.rps + j;
+            for (int i = threadIdx.x; i < dm; i += THREADS) d.hidden[(size_t)r * dm + i] = hidden_at(a, c, r, i);
+        }
+    if (threadIdx.x == 0) {
+        SeqState &st = d.st[s];
+        if (which == PACER_TARGET) st.len_T += n;
+        else if (which == PACER_DRAFT) st.len_D += n;
+        else st.len_B += n;
+    }
+}
+
+// End of one autoregressive target step (Eq. 1).
+__device__ __forceinline__ void tail_ar(Ctx &c, const Args &a, int s) {
+    if (c.n_rows[s] == 0 || threadIdx.x != 0) return;
+    const DevPtrs &d = a.d;
+    SeqState &st = d.st[s];
+    d.x[(size_t)s * d.max_ctx + st.P] = d.row_arg[s * a.g.rps];
+    st.P += 1;
+    st.len_T += 1;
+    st.n_target_fwd += 1;
+    st.n_steps += 1;
+    if (st.P - st.n_prompt >= st.max_new) st.finished = 1;
+}
+
+// ------------------------------------------------------------------ the kernel
+
+template <int NT>
+__global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ Args a, const int which) {
+    extern __shared__ __align__(1024) unsigned char smem[];
+    Ctx c;
+    c.warp = threadIdx.x >> 5; c.lane = threadIdx.x & 31; c.cta = blockIdx.x; c.ncta = gridDim.x;
+    c.scratch = smem;
+    c.ring = smem + SCRATCH_BYTES + c.warp * (STAGES * STAGE_BYTES);
+    unsigned char *misc = smem + SCRATCH_BYTES + RING_BYTES;
+    c.mbar = reinterpret_cast<uint64_t *>(misc) + c.warp * STAGES;           // 8 * STAGES * 8 bytes
+    c.row_pos = reinterpret_cast<int32_t *>(misc + 256);
+    c.row_tok = c.row_pos + MAX_ROWS;
+    c.n_rows = c.row_tok + MAX_ROWS;
+    c.inv_rms = reinterpret_cast<float *>(c.n_rows + MAX_ROWS);
+    c.flag = reinterpret_cast<int32_t *>(c.inv_rms + MAX_ROWS);              // 4 words
+    float **row_dst = reinterpret_cast<float **>(misc + 1024);               // [MAX_ROWS]
+    int32_t *bias_at = reinterpret_cast<int32_t *>(misc + 1024 + 256);       // [MAX_ROWS]
+    Top2 *top_sm = reinterpret_cast<Top2 *>(misc + 1024 + 384);              // [32]
+    c.bar_target = 0;
+    c.policy = policy_evict_first();
+    const DevPtrs &d = a.d;
+    const ModelDev &m = a.m;
+    const Geom &g = a.g;
+    const int kind = a.kind;
+
+    // rows of this forward, from the sequence state
+    if (threadIdx.x < MAX_ROWS) {
+        const int r = threadIdx.x;
+        int pos = -1, tok = 0;
+        if (r < g.rtot) {
+            const RowDesc rd = row_desc(kind, d, r / g.rps, r % g.rps, a.aux);
+            if (rd.active) { pos = rd.pos; tok = rd.tok; }
+        }
+        c.row_pos[r] = pos; c.row_tok[r] = tok;
+    }
+    __syncthreads();
+    if (threadIdx.x < MAX_ROWS) {
+        const int s = threadIdx.x;
+        int n = 0;
+        if (s < g.batch)
+            for (int j = 0; j < g.rps; ++j) n += c.row_pos[s * g.rps + j] >= 0;
+        c.n_rows[s] = n;
+    }
+    __syncthreads();
+    int any = 0;
+    for (int s = 0; s < g.batch; ++s) any |= c.n_rows[s];
+    if (c.cta == 0 && threadIdx.x < MAX_ROWS) {
+        if (threadIdx.x < g.batch) d.n_rows[threadIdx.x] = c.n_rows[threadIdx.x];
+        if (threadIdx.x < g.rtot) { d.row_pos[threadIdx.x] = c.row_pos[threadIdx.x]; d.row_tok[threadIdx.x] = c.row_tok[threadIdx.x]; }
+    }
+    if (!any) return;                       // every sequence idles: the same decision in every block
+
+    if (threadIdx.x < MAX_ROWS) {           // where the LM-head rows go
+        const int r = threadIdx.x;
+        float *dst = nullptr;
+        int b = -1;
+        if (r < g.rtot && c.row_pos[r] >= 0 && a.P.has_head) {
+            const int s = r / g.rps, j = r - s * g.rps, V = m.cfg.vocab;
+            if (kind == KIND_DRAFT) {
+                if (j == c.n_rows[s] - 1) dst = d.draft_logits + ((size_t)s * d.gamma_cap + d.st[s].gamma) * V;
+            } else {
+                dst = d.verify_logits + ((size_t)s * (d.gamma_cap + 1) + j) * V;
+            }
+            if (m.succ) b = m.succ[c.row_tok[r]];
+        }
+        row_dst[r] = dst; bias_at[r] = b;
+    }
+    if (threadIdx.x == 0) {
+        const unsigned long long v = ld_acquire_u64(a.fb.bar);
+        c.bar_target = v / (unsigned long long)c.ncta * (unsigned long long)c.ncta;
+    }
+    if (c.lane == 0)
+        for (int i = 0; i < STAGES; ++i) mbar_init(c.mbar + i, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_proxy_async();
+    __syncthreads();
+
+    // start the weight stream: it runs ahead of the phases from here on
+    Stream st;
+    st.cu.q = st.cu.m = st.cu.j = st.cu.u = 0; st.cu.done = 0;
+    st.pn = st.cn = 0;
+    settle(st.cu, a.P, c.cta, c.ncta, c.warp);
+    for (int i = 0; i < STAGES; ++i) issue_unit(c, st, a.P);
+
+    constexpr int RPAD = NT * 8;
+    const int dm = m.cfg.d_model;
+    phase_begin(c, a, RPAD);
+    grid_barrier(c, a.fb);
+
+    for (int l = 0; l < a.P.n_layers; ++l) {
+        compute_inv(c, a);
+        gemm_op<NT>(c, a.fb, a.P, OP_QKV, st,
+                    [&](int k_lo, int k_hi) { xload_normed<NT>(c, a, m.norm1 + (size_t)l * dm, k_lo, k_hi); },
+                    [&](int tile, float (&acc)[NT][4]) { epi_qkv<NT>(c, a, tile, acc); });
+        grid_barrier(c, a.fb);
+        phase_attention(c, a, l, NT);
+        grid_barrier(c, a.fb);
+        gemm_op<NT>(c, a.fb, a.P, OP_O, st,
+                    [&](int k_lo, int k_hi) { xload_frag<NT>(c, d.att, k_lo, k_hi); },
+                    [&](int tile, float (&acc)[NT][4]) { epi_residual<NT>(c, a, tile, acc); });
+        grid_barrier(c, a.fb);
+        compute_inv(c, a);
+        gemm_op<NT>(c, a.fb, a.P, OP_GU, st,
+                    [&](int k_lo, int k_hi) { xload_normed<NT>(c, a, m.norm2 + (size_t)l * dm, k_lo, k_hi); },
+                    [&](int tile, float (&acc)[NT][4]) { epi_swiglu<NT>(c, a, tile, acc); });
+        grid_barrier(c, a.fb);
+        gemm_op<NT>(c, a.fb, a.P, OP_DOWN, st,
+                    [&](int k_lo, int k_hi) { xload_frag<NT>(c, d.act, k_lo, k_hi); },
+                    [&](int tile, float (&acc)[NT][4]) { epi_residual<NT>(c, a, tile, acc); });
+        grid_barrier(c, a.fb);
+    }
+    compute_inv(c, a);                      // final RMSNorm statistics (LM head and tails)
+    if (a.P.has_head) {
+        gemm_op<NT>(c, a.fb, a.P, OP_HEAD, st,
+                    [&](int k_lo, int k_hi) { xload_normed<NT>(c, a, m.normf, k_lo, k_hi); },
+                    [&](int tile, float (&acc)[NT][4]) { epi_head<NT>(c, a, row_dst, bias_at, tile, acc); });
+        grid_barrier(c, a.fb);
+        if (kind == KIND_VERIFY) {
+            if (c.cta < g.rtot && row_dst[c.cta]) head_row_argmax(a, c.cta, top_sm);
+        } else if (c.cta < g.batch && c.n_rows[c.cta] > 0) {
+            head_row_argmax(a, c.cta * g.rps + c.n_rows[c.cta] - 1, top_sm);
+        }
+    }
+    if (c.cta < g.batch) {
+        if (kind == KIND_DRAFT) tail_draft(c, a, c.cta);
+        else if (kind == KIND_MB) tail_mb(c, a, c.cta);
+        else if (kind == KIND_AR) tail_ar(c, a, c.cta);
+        else if (kind == KIND_PREFILL || kind == KIND_PREFILL_B) tail_prefill(c, a, c.cta, which);
+    }
+    // nothing of this warp's stream may still be in flight at exit
+    while (st.cn < st.pn) { wait_unit(c, a.fb, st.cn); ++st.cn; }
+}
+
+}  // namespace fwd
+
+// ------------------------------------------------------------------ host: planning and launch
+
+namespace fwd {
+
+// Cuts one projection into S k-slices x G tile groups.  The slice must fit the
+// activation buffer; among the admissible cuts the one with the smallest
+// per-block maximum of streamed bytes wins (more slices cost a little: their
+// partial sums travel through L2).
+static inline void plan_op(GemmOp &op, int ncta, int NT, int rot) {
+    const int chunks = op.K / 32, MT = op.MT;
+    const int maxchunks = std::max(1, XBUF_BYTES / (NT * 512));
+    const int s_min = (chunks + maxchunks - 1) / maxchunks;
+    double best = 1e300;
+    int bS = s_min, bKS = 0, bG = 1, bTPG = MT;
+    std::vector<long long> load(ncta);
+    for (int S0 = s_min; S0 <= std::min(chunks, s_min + 24); ++S0) {
+        const int ksc = (chunks + S0 - 1) / S0, S = (chunks + ksc - 1) / ksc;
+        if (S != S0) continue;
+        for (int mlt = 1; mlt <= 6; ++mlt) {
+            for (int dg = 0; dg < 2; ++dg) {
+                int G = (int)((long long)ncta * mlt / S) + dg;
+                G = std::max(1, std::min(G, MT));
+                const int TPG = (MT + G - 1) / G;
+                G = (MT + TPG - 1) / TPG;
+                std::fill(load.begin(), load.end(), 0LL);
+                const int items = S * G;
+                for (int i = 0; i < items; ++i) {
+                    const int s = i % S, g = i / S;
+                    const int tiles = std::min(TPG, MT - g * TPG), len = std::min(ksc, chunks - s * ksc);
+                    // bytes in units of one tile x one 32-chunk, plus the price of loading the item's activations
+                    load[(i + rot) % ncta] += (long long)((tiles + WARPS - 1) / WARPS) * WARPS * len / 2 +
+                                              (long long)tiles * len / 2 + 3 * len;
+                }
+                const long long mk = *std::max_element(load.begin(), load.end());
+                const double score = (double)mk * (1.0 + 0.01 * (S - 1));
+                if (score < best) { best = score; bS = S; bKS = ksc * 32; bG = G; bTPG = TPG; }
+            }
+        }
+    }
+    op.S = bS; op.KS = bKS; op.G = bG; op.TPG = bTPG; op.items = bS * bG; op.rot = rot;
+}
+
+static inline Plan make_plan(const ModelDev &m, int ncta, int NT, bool has_head) {
+    Plan P;
+    memset(&P, 0, sizeof P);
+    const pacer_model_cfg &k = m.cfg;
+    const long long dm = k.d_model, F = k.d_ffn, hh = (long long)k.n_heads * m.hd;
+    auto set = [&](int i, const bf16 *w1, const bf16 *w2, long long lstride, int N, int K, int MT, int inter) {
+        GemmOp &o = P.op[i];
+        o.W1 = w1; o.W2 = w2 ? w2 : w1; o.lstride = lstride; o.N = N; o.K = K; o.MT = MT; o.interleave = inter;
+    };
+    set(OP_QKV, m.wqkv, nullptr, (long long)m.qrows * dm, m.qrows, (int)dm, (m.qrows + 15) / 16, 0);
+    set(OP_O, m.wo, nullptr, dm * hh, (int)dm, (int)hh, ((int)dm + 15) / 16, 0);
+    set(OP_GU, m.wgate, m.wup, F * dm, (int)(2 * F), (int)dm, ((int)F + 7) / 8, 1);
+    set(OP_DOWN, m.wdown, nullptr, dm * F, (int)dm, (int)F, ((int)dm + 15) / 16, 0);
+    set(OP_HEAD, m.head, nullptr, 0, k.vocab, (int)dm, (k.vocab + 15) / 16, 0);
+    int rot = 0;
+    for (int i = 0; i < N_OPS; ++i) {
+        if (i == OP_HEAD && !has_head) { P.op[i].S = 1; P.op[i].KS = 32; P.op[i].G = 0; P.op[i].TPG = 1; P.op[i].items = 0; continue; }
+        plan_op(P.op[i], ncta, NT, rot);
+        rot = (rot + P.op[i].items) % ncta;
+    }
+    P.n_layers = k.n_layers;
+    P.has_head = has_head ? 1 : 0;
+    return P;
+}
+
+// Floats of split-k partials the plan needs.
+static inline size_t plan_part_floats(const Plan &P, int NT) {
+    size_t mx = 0;
+    for (int i = 0; i < N_OPS; ++i) {
+        if (P.op[i].items == 0 || P.op[i].S == 1) continue;
+        mx = std::max(mx, (size_t)P.op[i].S * P.op[i].MT * (size_t)NT * 8 * 16);
+    }
+    return mx;
+}
+
+template <int NT>
+static inline cudaError_t launch_nt(const Args &a, int which, int ncta, cudaStream_t st) {
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(k_forward<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    void *params[] = {(void *)&a, (void *)&which};
+    return cudaLaunchCooperativeKernel((const void *)k_forward<NT>, dim3(ncta), dim3(THREADS), params, SMEM_BYTES, st);
+}
+
+static inline cudaError_t launch(const Args &a, int which, int ncta, cudaStream_t st) {
+    switch (a.g.nt) {
+        case 1: return launch_nt<1>(a, which, ncta, st);
+        case 2: return launch_nt<2>(a, which, ncta, st);
+        case 3: return launch_nt<3>(a, which, ncta, st);
+        case 4: return launch_nt<4>(a, which, ncta, st);
+    }
+    return cudaErrorInvalidValue;
+}
+
+}  // namespace fwd
