@@ -1,10 +1,9 @@
-// Device-side control of the loop: LM-head finish (bias, argmax), end of a draft
-// step, block test of the pre-verification (Algorithm 1), acceptance and cache
-// rollback (Eq. 5).  All decisions are taken on the device from SeqState.
+// Device-side control of the loop: top-2 reductions for the LM head, and the
+// acceptance + cache rollback kernel (Eq. 5).  The ends of the draft /
+// pre-verification / autoregressive forwards are tails of the forward kernel.
+// All decisions are taken on the device from SeqState.
 #pragma once
 #include "common.cuh"
-
-constexpr int HEAD_THREADS = 1024;
 
 struct Top2 {
     float v1; int i1; float v2;
@@ -47,107 +46,6 @@ __device__ __forceinline__ Top2 block_top2(Top2 t, Top2 *sm) {
     return sm[0];
 }
 
-// Sums the LM-head partials of one row, adds the planted bias on succ[input
-// token], stores the logits where the stage wants them, and finds the argmax
-// (lowest index on ties) with the gap to the runner-up.
-// kind DRAFT: only the last active row of each sequence matters (it emits y_i);
-// its logits go to draft_logits[seq][gamma].  kind VERIFY: every active row j
-// goes to verify_logits[seq][j].  kind AR: row 0 to verify_logits[seq][0].
-__global__ void __launch_bounds__(HEAD_THREADS) k_head_finish(DevPtrs d, ModelDev m, Geom g, int kind, int S) {
-    __shared__ Top2 sm[32];
-    const int r = blockIdx.x, s = r / g.rps, j = r - s * g.rps;
-    if (d.row_pos[r] < 0) return;
-    const int V = m.cfg.vocab;
-    float *dst;
-    if (kind == KIND_DRAFT) {
-        if (j != d.n_rows[s] - 1) return;
-        dst = d.draft_logits + ((size_t)s * d.gamma_cap + d.st[s].gamma) * V;
-    } else {
-        dst = d.verify_logits + ((size_t)s * (d.gamma_cap + 1) + j) * V;
-    }
-    const size_t sstride = (size_t)g.nt * 8 * V;
-    const float *p = d.part + (size_t)r * V;
-    const int bias_at = m.succ ? m.succ[d.row_tok[r]] : -1;
-    Top2 t{-INFINITY, 0x7fffffff, -INFINITY};
-    for (int v = threadIdx.x; v < V; v += blockDim.x) {
-        float val = 0.f;
-        for (int ss = 0; ss < S; ++ss) val += p[ss * sstride + v];
-        if (v == bias_at) val += d.succ_bias;
-        dst[v] = val;
-        if (val > t.v1) { t.v2 = t.v1; t.v1 = val; t.i1 = v; }
-        else if (val > t.v2) t.v2 = val;
-    }
-    t = block_top2(t, sm);
-    if (threadIdx.x == 0) { d.row_arg[r] = t.i1; d.row_margin[r] = t.v1 - t.v2; }
-}
-
-// End of one draft forward (Eq. 6): y_i, h_i queued for M_B, cache length.
-__global__ void __launch_bounds__(256) k_draft_end(DevPtrs d, Geom g, int dm) {
-    const int s = blockIdx.x;
-    SeqState &st = d.st[s];
-    const int n_in = d.n_rows[s];
-    if (n_in == 0) return;
-    const int r_last = s * g.rps + n_in - 1;
-    const int gamma = st.gamma, n_pend = st.n_pend;
-    for (int jj = 0; jj < n_in; ++jj) {
-        const float *h = d.hidden + (size_t)(s * g.rps + jj) * dm;
-        float *dst = d.hpend + ((size_t)s * (d.block_b + 1) + n_pend + jj) * dm;
-        for (int i = threadIdx.x; i < dm; i += blockDim.x) dst[i] = h[i];
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        for (int jj = 0; jj < n_in; ++jj)
-            d.hpend_e[s * (d.block_b + 1) + n_pend + jj] = (jj == n_in - 1) ? gamma + 1 : 0;
-        d.y[(size_t)s * d.gamma_cap + gamma] = d.row_arg[r_last];
-        st.n_pend = n_pend + n_in;
-        st.gamma = gamma + 1;
-        st.len_D += n_in;
-        st.n_draft_fwd += 1;
-    }
-}
-
-// End of a pre-verification call (Eq. 7 + block test): alpha_hat of the new
-// drafts from the 2-way head, block statistic, stop decision, threshold growth.
-__global__ void __launch_bounds__(256) k_mb_end(DevPtrs d, ModelDev m, Geom g) {
-    __shared__ float red[33];
-    const int s = blockIdx.x;
-    SeqState &st = d.st[s];
-    const int n = d.n_rows[s];
-    if (n == 0) return;
-    const int dm = m.cfg.d_model;
-    for (int j = 0; j < n; ++j) {
-        const int e = d.row_tok[s * g.rps + j];
-        if (e == 0) continue;
-        const float *h = d.hidden + (size_t)(s * g.rps + j) * dm;
-        float z0 = 0.f, z1 = 0.f;
-        for (int i = threadIdx.x; i < dm; i += blockDim.x) {
-            const float hv = h[i];
-            z0 += hv * __bfloat162float(m.head_b[i]);
-            z1 += hv * __bfloat162float(m.head_b[dm + i]);
-        }
-        z0 = block_sum(z0, red);
-        z1 = block_sum(z1, red);
-        if (threadIdx.x == 0) d.alpha[(size_t)s * d.gamma_cap + e - 1] = 1.f / (1.f + expf(z0 - z1));
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        const int b = d.block_b, gamma = st.gamma;
-        const float *ab = d.alpha + (size_t)s * d.gamma_cap + (gamma - b);
-        float stat;
-        if (d.criterion == 1) { stat = ab[0]; for (int i = 1; i < b; ++i) stat = fminf(stat, ab[i]); }
-        else if (d.criterion == 2) stat = ab[b - 1];
-        else { stat = 0.f; for (int i = 0; i < b; ++i) stat += ab[i]; stat /= (float)b; }
-        int stop = 0;
-        if (st.t0 >= 0.f && stat <= st.t_k) stop = 1;
-        if (gamma + b > st.gamma_max) stop = 1;
-        if (stop) st.drafting = 0;
-        else { st.t_k = st.t_k * d.rho; st.k_round += 1; }
-        st.len_B += n;
-        st.n_pend = 0;
-        st.n_mb_calls += 1;
-    }
-}
-
 // Greedy acceptance (Eq. 5 with one-hot distributions), commit, rollback, logs.
 __global__ void k_accept_greedy(DevPtrs d, Geom g) {
     const int s = blockIdx.x * blockDim.x + threadIdx.x;
@@ -177,30 +75,4 @@ __global__ void k_accept_greedy(DevPtrs d, Geom g) {
     st.n_target_fwd += 1;
     st.gamma = 0; st.k_round = 0; st.t_k = st.t0; st.drafting = 1; st.n_pend = 0;
     if (st.P - st.n_prompt >= st.max_new) { st.finished = 1; st.drafting = 0; }
-}
-
-// End of one autoregressive target step (Eq. 1).
-__global__ void k_ar_end(DevPtrs d, Geom g) {
-    const int s = blockIdx.x * blockDim.x + threadIdx.x;
-    if (s >= g.batch) return;
-    SeqState &st = d.st[s];
-    if (!st.active || st.finished || d.n_rows[s] == 0) return;
-    d.x[(size_t)s * d.max_ctx + st.P] = d.row_arg[s * g.rps];
-    st.P += 1;
-    st.len_T += 1;
-    st.n_target_fwd += 1;
-    st.n_steps += 1;
-    if (st.P - st.n_prompt >= st.max_new) st.finished = 1;
-}
-
-// After a prefill chunk: nothing to decide, the caches grow by the rows written.
-__global__ void k_prefill_end(DevPtrs d, Geom g, int which) {
-    const int s = blockIdx.x * blockDim.x + threadIdx.x;
-    if (s >= g.batch) return;
-    SeqState &st = d.st[s];
-    if (!st.active) return;
-    const int n = d.n_rows[s];
-    if (which == PACER_TARGET) st.len_T += n;
-    else if (which == PACER_DRAFT) st.len_D += n;
-    else st.len_B += n;
 }

@@ -9,11 +9,12 @@
 #include <string>
 #include <vector>
 
-#include "attention.cuh"
+#include <map>
+
 #include "common.cuh"
 #include "control.cuh"
+#include "fwd_kernel.cuh"
 #include "gemm.cuh"
-#include "rowops.cuh"
 
 struct pacer_ctx {
     pacer_cfg cfg;
@@ -23,6 +24,10 @@ struct pacer_ctx {
     DevPtrs d;
     ModelDev model[3];
     Geom g_draft, g_mb, g_verify, g_ar;
+    fwd::FwdBufs fb;
+    int ncta;                  // blocks of the forward kernel (one per SM)
+    std::map<int, fwd::Plan> plans;   // key: which * 16 + nt * 2 + has_head
+    size_t part_floats;        // capacity of the split-k partial buffer
     int batch;                 // sequences of the current run
     int prefilled;
     int64_t launches;
@@ -88,6 +93,7 @@ static bool cfg_ok(const pacer_cfg *c) {
     if (c->block_b < 1 || c->gamma_cap < c->block_b || c->gamma_cap % c->block_b) return false;
     if (c->criterion < 0 || c->criterion > 2) return false;
     if (!(c->rho > 0.f)) return false;
+    if ((int64_t)c->max_batch * (c->gamma_cap + 1) > fwd::MAX_ROWS) return false;   // rows of one verify forward
     return true;
 }
 
@@ -108,7 +114,8 @@ struct Carver {
 
 struct Layout {
     size_t st, x, y, alpha, hpend, hpend_e, draft_len, accept_len, verify_logits, draft_logits;
-    size_t row_pos, row_tok, n_rows, row_arg, row_margin, xres, xn, att, act, q, hidden, part;
+    size_t row_pos, row_tok, n_rows, row_arg, row_margin, xres, att, act, hidden, part;
+    size_t tile_cnt, att_cnt, bar, abort_flag, qkv, ssq, tile_top, attp;
     size_t kc[3], vc[3], rope[3];
     size_t kv_bytes[3], rope_bytes[3];
     size_t total;
@@ -116,16 +123,32 @@ struct Layout {
     size_t part_bytes, state_bytes;
 };
 
-static size_t part_floats(const pacer_model_cfg &m, int nt_max, bool with_head) {
-    const int hd = m.d_model / m.n_heads, qrows = (m.n_heads + 2 * m.n_kv_heads) * hd;
-    const int NT = nt_max < 4 ? nt_max : 4;
-    struct { int N, K; } shp[5] = {{qrows, m.d_model}, {m.d_model, m.n_heads * hd}, {2 * m.d_ffn, m.d_model},
-                                   {m.d_model, m.d_ffn}, {m.vocab, m.d_model}};
+static int sm_count_or_default() {
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess &&
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0)
+        return n;
+    cudaGetLastError();
+    return 148;
+}
+
+// Split-k partial floats the forward kernel can need for this configuration (any row-tile count, any model).
+static size_t part_floats_needed(const pacer_cfg &c, int ncta) {
+    const pacer_model_cfg mb = mb_cfg(c);
+    const pacer_model_cfg *ms[3] = {&c.target, &c.draft, &mb};
+    const int rps_max = std::max(c.gamma_cap + 1, c.block_b + 1);
+    const int nt_max = std::min(4, (c.max_batch * rps_max + 7) / 8);
     size_t mx = 0;
-    for (int i = 0; i < (with_head ? 5 : 4); ++i) {
-        GemmPlan p = gemm_plan(shp[i].N, shp[i].K, NT);
-        size_t f = (size_t)p.S * nt_max * 8 * shp[i].N;
-        if (f > mx) mx = f;
+    for (int i = 0; i < 3; ++i) {
+        ModelDev m;
+        memset(&m, 0, sizeof m);
+        m.cfg = *ms[i];
+        m.hd = m.cfg.d_model / m.cfg.n_heads;
+        m.qrows = (m.cfg.n_heads + 2 * m.cfg.n_kv_heads) * m.hd;
+        for (int nt = 1; nt <= nt_max; ++nt) {
+            fwd::Plan P = fwd::make_plan(m, ncta, nt, i != 2);
+            mx = std::max(mx, fwd::plan_part_floats(P, nt));
+        }
     }
     return mx;
 }
@@ -140,12 +163,15 @@ static Layout make_layout(const pacer_cfg &c) {
     L.rtot_max = B * rps_max;
     L.nt_max = (L.rtot_max + 7) / 8;
     L.max_steps = c.max_ctx;
-    int d_max = 0, hh_max = 0, f_max = 0;
+    int d_max = 0, f_max = 0, h_max = 0, hd_max = 0, qrows_max = 0;
     for (int i = 0; i < 3; ++i) {
-        d_max = ms[i]->d_model > d_max ? ms[i]->d_model : d_max;
-        f_max = ms[i]->d_ffn > f_max ? ms[i]->d_ffn : f_max;
+        const int hd = ms[i]->d_model / ms[i]->n_heads;
+        d_max = std::max(d_max, ms[i]->d_model);
+        f_max = std::max(f_max, ms[i]->d_ffn);
+        h_max = std::max(h_max, ms[i]->n_heads);
+        hd_max = std::max(hd_max, hd);
+        qrows_max = std::max(qrows_max, (ms[i]->n_heads + 2 * ms[i]->n_kv_heads) * hd);
     }
-    hh_max = d_max;
     L.st = cv.take(sizeof(SeqState) * B);
     L.x = cv.take(sizeof(int32_t) * B * c.max_ctx);
     L.y = cv.take(sizeof(int32_t) * B * gc);
@@ -153,27 +179,31 @@ static Layout make_layout(const pacer_cfg &c) {
     L.hpend_e = cv.take(sizeof(int32_t) * B * (c.block_b + 1));
     L.draft_len = cv.take(sizeof(int32_t) * B * L.max_steps);
     L.accept_len = cv.take(sizeof(int32_t) * B * L.max_steps);
-    L.row_pos = cv.take(sizeof(int32_t) * L.rtot_max);
-    L.row_tok = cv.take(sizeof(int32_t) * L.rtot_max);
-    L.n_rows = cv.take(sizeof(int32_t) * B);
-    L.row_arg = cv.take(sizeof(int32_t) * L.rtot_max);
-    L.row_margin = cv.take(sizeof(float) * L.rtot_max);
+    L.row_pos = cv.take(sizeof(int32_t) * fwd::MAX_ROWS);
+    L.row_tok = cv.take(sizeof(int32_t) * fwd::MAX_ROWS);
+    L.n_rows = cv.take(sizeof(int32_t) * fwd::MAX_ROWS);
+    L.row_arg = cv.take(sizeof(int32_t) * fwd::MAX_ROWS);
+    L.row_margin = cv.take(sizeof(float) * fwd::MAX_ROWS);
+    L.tile_cnt = cv.take(sizeof(int32_t) * ((size_t)std::max(V, 2 * f_max) / 8 + 16));
+    L.att_cnt = cv.take(sizeof(int32_t) * (size_t)B * h_max);
+    L.bar = cv.take(sizeof(unsigned long long));
+    L.abort_flag = cv.take(sizeof(int32_t));
     L.state_bytes = cv.off;                                   // zeroed at create
     L.hpend = cv.take(sizeof(float) * B * (c.block_b + 1) * c.draft.d_model);
     L.verify_logits = cv.take(sizeof(float) * B * (gc + 1) * V);
     L.draft_logits = cv.take(sizeof(float) * B * gc * V);
-    L.xres = cv.take(sizeof(float) * L.rtot_max * d_max);
-    L.hidden = cv.take(sizeof(float) * L.rtot_max * d_max);
-    L.q = cv.take(sizeof(float) * L.rtot_max * hh_max);
-    L.xn = cv.take(sizeof(bf16) * L.nt_max * 8 * d_max);
-    L.att = cv.take(sizeof(bf16) * L.nt_max * 8 * hh_max);
-    L.act = cv.take(sizeof(bf16) * L.nt_max * 8 * f_max);
-    size_t pf = 0;
-    for (int i = 0; i < 3; ++i) {
-        size_t f = part_floats(*ms[i], L.nt_max, i != 2);
-        if (f > pf) pf = f;
-    }
-    L.part_bytes = pf * sizeof(float);
+    L.xres = cv.take(sizeof(float) * fwd::MAX_ROWS * d_max);
+    L.hidden = cv.take(sizeof(float) * fwd::MAX_ROWS * d_max);
+    L.att = cv.take(sizeof(bf16) * fwd::MAX_ROWS * d_max);
+    L.act = cv.take(sizeof(bf16) * fwd::MAX_ROWS * f_max);
+    L.qkv = cv.take(sizeof(float) * fwd::MAX_ROWS * qrows_max);
+    L.ssq = cv.take(sizeof(float) * fwd::MAX_ROWS * (d_max / 16 + 1));
+    L.tile_top = cv.take(sizeof(float) * 4 * fwd::MAX_ROWS * ((size_t)V / 16 + 1));
+    L.attp = cv.take(sizeof(float) * (size_t)B * h_max * fwd::MAX_SPLIT * rps_max * (hd_max + 2));
+    // planned for 148 blocks and for the device's own count when one is present; twice the need, so that a
+    // device with another SM count still fits
+    size_t pf = std::max(part_floats_needed(c, 148), part_floats_needed(c, sm_count_or_default()));
+    L.part_bytes = 2 * pf * sizeof(float) + 256;
     L.part = cv.take(L.part_bytes);
     for (int i = 0; i < 3; ++i) {
         const int hd = ms[i]->d_model / ms[i]->n_heads;
@@ -233,8 +263,14 @@ extern "C" int pacer_create(const pacer_cfg *cfg, void *dev_workspace, size_t wo
     d.verify_logits = (float *)(w + L.verify_logits); d.draft_logits = (float *)(w + L.draft_logits);
     d.row_pos = (int32_t *)(w + L.row_pos); d.row_tok = (int32_t *)(w + L.row_tok); d.n_rows = (int32_t *)(w + L.n_rows);
     d.row_arg = (int32_t *)(w + L.row_arg); d.row_margin = (float *)(w + L.row_margin);
-    d.xres = (float *)(w + L.xres); d.xn = (bf16 *)(w + L.xn); d.att = (bf16 *)(w + L.att); d.act = (bf16 *)(w + L.act);
-    d.q = (float *)(w + L.q); d.hidden = (float *)(w + L.hidden); d.part = (float *)(w + L.part);
+    d.xres = (float *)(w + L.xres); d.xn = nullptr; d.att = (bf16 *)(w + L.att); d.act = (bf16 *)(w + L.act);
+    d.q = nullptr; d.hidden = (float *)(w + L.hidden); d.part = (float *)(w + L.part);
+    c->fb.qkv = (float *)(w + L.qkv); c->fb.part = (float *)(w + L.part); c->fb.tile_cnt = (int32_t *)(w + L.tile_cnt);
+    c->fb.ssq = (float *)(w + L.ssq); c->fb.tile_top = (float *)(w + L.tile_top); c->fb.attp = (float *)(w + L.attp);
+    c->fb.att_cnt = (int32_t *)(w + L.att_cnt); c->fb.bar = (unsigned long long *)(w + L.bar);
+    c->fb.abort_flag = (int32_t *)(w + L.abort_flag);
+    c->part_floats = L.part_bytes / sizeof(float);
+    c->ncta = sm_count_or_default();
     d.max_batch = cfg->max_batch; d.max_ctx = cfg->max_ctx; d.gamma_cap = cfg->gamma_cap; d.block_b = cfg->block_b;
     d.max_steps = L.max_steps; d.rho = cfg->rho; d.succ_bias = cfg->succ_bias; d.criterion = cfg->criterion;
     d.use_posemb = cfg->use_posemb;
@@ -333,6 +369,7 @@ extern "C" int pacer_load_weights(pacer_ctx *c, int which, const pacer_tensor *t
         if (wn.needed && !*wn.slot) return fail(c, PACER_EINVAL, std::string("pacer_load_weights: missing tensor ") + wn.name);
     m.succ = isB ? nullptr : succ;
     m.loaded = 1;
+    c->plans.clear();
     return PACER_OK;
 }
 
@@ -344,58 +381,35 @@ extern "C" int pacer_load_weights(pacer_ctx *c, int which, const pacer_tensor *t
         CK(cudaGetLastError());                                             \
     } while (0)
 
-// One weight-streaming product of a forward, optionally bracketed by profiling events.
-static int fwd_gemm(pacer_ctx *c, const bf16 *X, const Geom &g, const bf16 *W1, const bf16 *W2, int n_w1, int N, int K,
-                    GemmPlan *p) {
-    const bool prof = c->prof_on && c->prof_used + 2 <= c->prof_ev.size();
+static double model_weight_bytes(const ModelDev &m, bool head) {
+    const pacer_model_cfg &k = m.cfg;
+    const double per_layer = (double)m.qrows * k.d_model + (double)k.d_model * k.n_heads * m.hd + 3.0 * k.d_model * k.d_ffn;
+    return 2.0 * (k.n_layers * per_layer + (head ? (double)k.vocab * k.d_model : 0.0));
+}
+
+// Runs model `which` on the rows `kind` selects: ONE cooperative launch of the
+// persistent forward kernel, which also takes the stage's decisions in its tail.
+static int run_forward(pacer_ctx *c, int which, const Geom &g, int kind, int aux, bool head) {
+    ModelDev &m = c->model[which];
+    if (g.rtot > fwd::MAX_ROWS || g.nt > 4) return fail(c, PACER_EUNSUPPORTED, "more than 32 rows in one forward");
+    const int key = which * 16 + g.nt * 2 + (head ? 1 : 0);
+    auto it = c->plans.find(key);
+    if (it == c->plans.end()) {
+        fwd::Plan P = fwd::make_plan(m, c->ncta, g.nt, head);
+        if (fwd::plan_part_floats(P, g.nt) > c->part_floats)
+            return fail(c, PACER_ENOMEM, "split-k partial buffer too small for this device's SM count");
+        it = c->plans.emplace(key, P).first;
+    }
+    fwd::Args a;
+    a.d = c->d; a.m = m; a.g = g; a.P = it->second; a.fb = c->fb; a.kind = kind; a.aux = aux;
+    const bool prof = c->prof_on && which == PACER_TARGET && c->prof_used + 2 <= c->prof_ev.size();
     if (prof) CK(cudaEventRecord(c->prof_ev[c->prof_used], c->stream));
-    CK(gemm_run(X, g.nt, W1, W2, n_w1, N, K, c->d.part, c->d.n_rows, g.batch, c->stream, p, &c->launches));
+    CK(fwd::launch(a, which, c->ncta, c->stream));
+    ++c->launches;
     if (prof) {
         CK(cudaEventRecord(c->prof_ev[c->prof_used + 1], c->stream));
         c->prof_used += 2;
-        c->prof_bytes += 2.0 * (double)N * (double)K;
-    }
-    return PACER_OK;
-}
-
-// Runs model `which` on the rows `kind` selects.  head: LM head + argmax;
-// hidden: keep the fp32 final-norm output.
-static int run_forward(pacer_ctx *c, int which, const Geom &g, int kind, int aux, bool head, bool hidden) {
-    ModelDev &m = c->model[which];
-    DevPtrs &d = c->d;
-    cudaStream_t st = c->stream;
-    const pacer_model_cfg &k = m.cfg;
-    const int dm = k.d_model, F = k.d_ffn, hh = k.n_heads * m.hd;
-    GemmPlan p;
-    int rc;
-    k_begin<<<g.rtot, ROW_THREADS, 0, st>>>(d, m, g, kind, aux);
-    LAUNCH_CHECK();
-    for (int l = 0; l < k.n_layers; ++l) {
-        if ((rc = fwd_gemm(c, d.xn, g, m.wqkv + (size_t)l * m.qrows * dm, nullptr, 0, m.qrows, dm, &p))) return rc;
-        k_rope_append<<<g.rtot, ROW_THREADS, 0, st>>>(d, m, g, l, p.S);
-        LAUNCH_CHECK();
-        CK(attention_launch(d, m, g, l, st));
-        ++c->launches;
-        if ((rc = fwd_gemm(c, d.att, g, m.wo + (size_t)l * dm * hh, nullptr, 0, dm, hh, &p))) return rc;
-        k_add_norm<<<g.rtot, ROW_THREADS, 0, st>>>(d, g, dm, k.rms_eps, m.norm2 + (size_t)l * dm, p.S, 0);
-        LAUNCH_CHECK();
-        if ((rc = fwd_gemm(c, d.xn, g, m.wgate + (size_t)l * F * dm, m.wup + (size_t)l * F * dm, F, 2 * F, dm, &p))) return rc;
-        k_swiglu<<<dim3((F + ROW_THREADS - 1) / ROW_THREADS, g.rtot), ROW_THREADS, 0, st>>>(d, g, F, p.S);
-        LAUNCH_CHECK();
-        if ((rc = fwd_gemm(c, d.act, g, m.wdown + (size_t)l * dm * F, nullptr, 0, dm, F, &p))) return rc;
-        const bool last = l == k.n_layers - 1;
-        if (!last) {
-            k_add_norm<<<g.rtot, ROW_THREADS, 0, st>>>(d, g, dm, k.rms_eps, m.norm1 + (size_t)(l + 1) * dm, p.S, 0);
-            LAUNCH_CHECK();
-        } else if (head || hidden) {
-            k_add_norm<<<g.rtot, ROW_THREADS, 0, st>>>(d, g, dm, k.rms_eps, m.normf, p.S, hidden ? 1 : 0);
-            LAUNCH_CHECK();
-        }
-    }
-    if (head) {
-        if ((rc = fwd_gemm(c, d.xn, g, m.head, nullptr, 0, k.vocab, dm, &p))) return rc;
-        k_head_finish<<<g.rtot, HEAD_THREADS, 0, st>>>(d, m, g, kind, p.S);
-        LAUNCH_CHECK();
+        c->prof_bytes += model_weight_bytes(m, head);
     }
     return PACER_OK;
 }
@@ -433,6 +447,8 @@ static int start_run(pacer_ctx *c, const int32_t *prompt, int batch, int n_promp
         st.t_k = threshold; st.mode = mode; st.seed = seed; st.active = 1; st.drafting = 1;
     }
     CK(cudaMemcpyAsync(c->d.st, hs.data(), sizeof(SeqState) * hs.size(), cudaMemcpyHostToDevice, c->stream));
+    // arrival counters, grid barrier and abort flag start from zero (they are contiguous in the workspace)
+    CK(cudaMemsetAsync(c->fb.tile_cnt, 0, (char *)c->fb.abort_flag + sizeof(int32_t) - (char *)c->fb.tile_cnt, c->stream));
     CK(cudaMemcpy2DAsync(c->d.x, sizeof(int32_t) * k.max_ctx, prompt, sizeof(int32_t) * n_prompt, sizeof(int32_t) * n_prompt,
                          batch, cudaMemcpyHostToDevice, c->stream));
     CK(cudaStreamSynchronize(c->stream));        // hs is a local
@@ -444,17 +460,11 @@ static int prefill_models(pacer_ctx *c, int n_prompt, bool target, bool draft_an
     for (int c0 = 0; c0 < n_prompt - 1; c0 += g.rps) {
         int rc;
         if (target) {
-            if ((rc = run_forward(c, PACER_TARGET, g, KIND_PREFILL, c0, false, false))) return rc;
-            k_prefill_end<<<1, 64, 0, c->stream>>>(c->d, g, PACER_TARGET);
-            LAUNCH_CHECK();
+            if ((rc = run_forward(c, PACER_TARGET, g, KIND_PREFILL, c0, false))) return rc;
         }
         if (draft_and_mb) {
-            if ((rc = run_forward(c, PACER_DRAFT, g, KIND_PREFILL, c0, false, true))) return rc;
-            k_prefill_end<<<1, 64, 0, c->stream>>>(c->d, g, PACER_DRAFT);
-            LAUNCH_CHECK();
-            if ((rc = run_forward(c, PACER_PREVERIFY, g, KIND_PREFILL_B, c0, false, false))) return rc;
-            k_prefill_end<<<1, 64, 0, c->stream>>>(c->d, g, PACER_PREVERIFY);
-            LAUNCH_CHECK();
+            if ((rc = run_forward(c, PACER_DRAFT, g, KIND_PREFILL, c0, false))) return rc;
+            if ((rc = run_forward(c, PACER_PREVERIFY, g, KIND_PREFILL_B, c0, false))) return rc;
         }
     }
     return PACER_OK;
@@ -473,25 +483,19 @@ extern "C" int pacer_prefill(pacer_ctx *c, const int32_t *prompt, int batch, int
 extern "C" int pacer_draft_step(pacer_ctx *c) {
     int rc = need_ready(c, true);
     if (rc) return rc;
-    if ((rc = run_forward(c, PACER_DRAFT, c->g_draft, KIND_DRAFT, 0, true, true))) return rc;
-    k_draft_end<<<c->batch, 256, 0, c->stream>>>(c->d, c->g_draft, c->cfg.draft.d_model);
-    LAUNCH_CHECK();
-    return PACER_OK;
+    return run_forward(c, PACER_DRAFT, c->g_draft, KIND_DRAFT, 0, true);
 }
 
 extern "C" int pacer_preverify(pacer_ctx *c) {
     int rc = need_ready(c, true);
     if (rc) return rc;
-    if ((rc = run_forward(c, PACER_PREVERIFY, c->g_mb, KIND_MB, 0, false, true))) return rc;
-    k_mb_end<<<c->batch, 256, 0, c->stream>>>(c->d, c->model[PACER_PREVERIFY], c->g_mb);
-    LAUNCH_CHECK();
-    return PACER_OK;
+    return run_forward(c, PACER_PREVERIFY, c->g_mb, KIND_MB, 0, false);
 }
 
 extern "C" int pacer_verify(pacer_ctx *c) {
     int rc = need_ready(c, true);
     if (rc) return rc;
-    return run_forward(c, PACER_TARGET, c->g_verify, KIND_VERIFY, 0, true, false);
+    return run_forward(c, PACER_TARGET, c->g_verify, KIND_VERIFY, 0, true);
 }
 
 extern "C" int pacer_accept_rollback(pacer_ctx *c) {
@@ -577,6 +581,9 @@ static int collect(pacer_ctx *c, int batch, int max_new, int n_prompt, int32_t *
     CK(cudaMemcpy2DAsync(out_tokens, sizeof(int32_t) * max_new, c->d.x + n_prompt, sizeof(int32_t) * k.max_ctx,
                          sizeof(int32_t) * max_new, batch, cudaMemcpyDeviceToHost, c->stream));
     CK(cudaStreamSynchronize(c->stream));
+    int32_t aborted = 0;
+    CK(cudaMemcpy(&aborted, c->fb.abort_flag, sizeof aborted, cudaMemcpyDeviceToHost));
+    if (aborted) return fail(c, PACER_EDEVICE, "a bounded wait inside the forward kernel ran out");
     int64_t nd = 0, nm = 0, nt = 0, ns = 0, ng = 0;
     for (int s = 0; s < batch; ++s) {
         const SeqState &a = hs[s];
@@ -639,9 +646,7 @@ extern "C" int pacer_generate_ar(pacer_ctx *c, const int32_t *prompt, int batch,
     CK(cudaEventRecord(c->ev[1], c->stream));
     const int64_t launches0 = c->launches;
     for (int i = 0; i < max_new; ++i) {
-        if ((rc = run_forward(c, PACER_TARGET, c->g_ar, KIND_AR, 0, true, false))) return rc;
-        k_ar_end<<<1, 64, 0, c->stream>>>(c->d, c->g_ar);
-        LAUNCH_CHECK();
+        if ((rc = run_forward(c, PACER_TARGET, c->g_ar, KIND_AR, 0, true))) return rc;
     }
     CK(cudaEventRecord(c->ev[2], c->stream));
     return collect(c, batch, max_new, n_prompt, out_tokens, nullptr, nullptr, nullptr, stats, launches0);
