@@ -114,7 +114,10 @@ enum {
     PACER_BUF_ACCEPT_LEN = 7,    /* int32 [max_batch][max_steps] n of every step */
     PACER_BUF_KCACHE_T = 8,      /* bf16  [L][max_batch][Hkv][max_ctx][hd] (also _D = 10, _B = 12) */
     PACER_BUF_VCACHE_T = 9,      /* bf16  same shape                        (also _D = 11, _B = 13) */
-    PACER_BUF_KCACHE_D = 10, PACER_BUF_VCACHE_D = 11, PACER_BUF_KCACHE_B = 12, PACER_BUF_VCACHE_B = 13
+    PACER_BUF_KCACHE_D = 10, PACER_BUF_VCACHE_D = 11, PACER_BUF_KCACHE_B = 12, PACER_BUF_VCACHE_B = 13,
+    PACER_BUF_PHASE_NS = 14      /* u64 [1024] device clock (ns) at the phase boundaries of the last profiled target
+                                    forward: start, input rows, barrier, then per layer QKV, barrier, attention,
+                                    barrier, O, barrier, gate/up, barrier, down, barrier; LM head, barrier; end */
 };
 
 const char *pacer_strerror(int code);
@@ -199,14 +202,15 @@ int pacer_generate_ar(pacer_ctx *ctx, const int32_t *prompt, int batch, int n_pr
                       uint64_t seed, int32_t *out_tokens, pacer_stats *stats);
 
 /* Kernel-level timing for roofline reports.  Between pacer_profile_begin and
- * pacer_profile_end every weight-streaming product this context launches is
- * bracketed by a pair of CUDA events on the context's stream (at most 4096
- * products are recorded; later ones run untimed).  pacer_profile_end [sync]
- * returns the summed device time of those launches (ms), the bf16 weight bytes
- * they streamed (N*K*2 each) and their count.  Event pairs serialise nothing but
- * add about a microsecond each, so whole-loop timings are taken without it. */
+ * pacer_profile_end every forward of the TARGET model (one launch of the
+ * persistent forward kernel) is bracketed by a pair of CUDA events on the
+ * context's stream (at most 4096 launches are recorded; later ones run untimed)
+ * and block 0 of the kernel stamps the device clock at its phase boundaries
+ * (PACER_BUF_PHASE_NS).  pacer_profile_end [sync] returns the summed device time
+ * of those launches (ms), the bf16 weight bytes they streamed and their count.
+ * Whole-loop timings are taken without it. */
 int pacer_profile_begin(pacer_ctx *ctx);
-int pacer_profile_end(pacer_ctx *ctx, double *gemm_ms, double *gemm_weight_bytes, int64_t *gemm_launches);
+int pacer_profile_end(pacer_ctx *ctx, double *fwd_ms, double *fwd_weight_bytes, int64_t *fwd_launches);
 
 /* Y[r][n] = sum_k X[r][k] * W[n][k]: the skinny weight-streaming product used by
  * every projection, exposed for kernel-level checks and timing.  x: device bf16

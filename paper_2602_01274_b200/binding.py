@@ -27,7 +27,7 @@ _lib = C.CDLL(LIB_PATH)
 PACER_TARGET, PACER_DRAFT, PACER_PREVERIFY = 0, 1, 2
 PACER_GREEDY, PACER_SAMPLE = 0, 1
 (BUF_TOKENS, BUF_DRAFTS, BUF_ALPHA, BUF_VERIFY_LOGITS, BUF_DRAFT_LOGITS, BUF_HPEND, BUF_DRAFT_LEN, BUF_ACCEPT_LEN,
- BUF_KCACHE_T, BUF_VCACHE_T, BUF_KCACHE_D, BUF_VCACHE_D, BUF_KCACHE_B, BUF_VCACHE_B) = range(14)
+ BUF_KCACHE_T, BUF_VCACHE_T, BUF_KCACHE_D, BUF_VCACHE_D, BUF_KCACHE_B, BUF_VCACHE_B, BUF_PHASE_NS) = range(15)
 
 
 class ModelCfg(C.Structure):

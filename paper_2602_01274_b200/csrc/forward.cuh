@@ -35,6 +35,7 @@ constexpr int SMEM_BYTES = SCRATCH_BYTES + RING_BYTES + MISC_BYTES;
 constexpr int MAX_ROWS = 32;                    // rows of one forward (all sequences together)
 constexpr int MAX_SPLIT = 16;                   // key-range splits of one attention head
 constexpr unsigned SPIN_LIMIT = 1u << 22;
+constexpr int PROF_STAMPS = 1024;             // phase-boundary time stamps kept per forward
 
 enum OpKind { OP_QKV = 0, OP_O = 1, OP_GU = 2, OP_DOWN = 3, OP_HEAD = 4, N_OPS = 5 };
 
@@ -66,6 +67,7 @@ struct FwdBufs {
     int32_t *att_cnt;        // [batch * H]
     unsigned long long *bar; // grid barrier counter
     int32_t *abort_flag;     // set when a bounded wait ran out
+    unsigned long long *prof; // optional: block 0 stamps %globaltimer at every phase boundary (NULL = off)
 };
 
 // ------------------------------------------------------------------ PTX helpers
@@ -97,6 +99,11 @@ __device__ __forceinline__ uint64_t policy_evict_first() {
     uint64_t p;
     asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
     return p;
+}
+__device__ __forceinline__ unsigned long long globaltimer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
 }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 

@@ -195,37 +195,56 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
 
     constexpr int RPAD = NT * 8;
     const int dm = m.cfg.d_model;
+    int n_stamp = 0;
+    auto stamp = [&]() {
+        if (a.fb.prof && c.cta == 0 && threadIdx.x == 0 && n_stamp < PROF_STAMPS) a.fb.prof[n_stamp++] = globaltimer_ns();
+    };
+    stamp();
     phase_begin(c, a, RPAD);
+    stamp();
     grid_barrier(c, a.fb);
+    stamp();
 
     for (int l = 0; l < a.P.n_layers; ++l) {
         compute_inv(c, a);
         gemm_op<NT>(c, a.fb, a.P, OP_QKV, st,
                     [&](int k_lo, int k_hi) { xload_normed<NT>(c, a, m.norm1 + (size_t)l * dm, k_lo, k_hi); },
                     [&](int tile, float (&acc)[NT][4]) { epi_qkv<NT>(c, a, tile, acc); });
+        stamp();
         grid_barrier(c, a.fb);
+        stamp();
         phase_attention(c, a, l, NT);
+        stamp();
         grid_barrier(c, a.fb);
+        stamp();
         gemm_op<NT>(c, a.fb, a.P, OP_O, st,
                     [&](int k_lo, int k_hi) { xload_frag<NT>(c, d.att, k_lo, k_hi); },
                     [&](int tile, float (&acc)[NT][4]) { epi_residual<NT>(c, a, tile, acc); });
+        stamp();
         grid_barrier(c, a.fb);
+        stamp();
         compute_inv(c, a);
         gemm_op<NT>(c, a.fb, a.P, OP_GU, st,
                     [&](int k_lo, int k_hi) { xload_normed<NT>(c, a, m.norm2 + (size_t)l * dm, k_lo, k_hi); },
                     [&](int tile, float (&acc)[NT][4]) { epi_swiglu<NT>(c, a, tile, acc); });
+        stamp();
         grid_barrier(c, a.fb);
+        stamp();
         gemm_op<NT>(c, a.fb, a.P, OP_DOWN, st,
                     [&](int k_lo, int k_hi) { xload_frag<NT>(c, d.act, k_lo, k_hi); },
                     [&](int tile, float (&acc)[NT][4]) { epi_residual<NT>(c, a, tile, acc); });
+        stamp();
         grid_barrier(c, a.fb);
+        stamp();
     }
     compute_inv(c, a);                      // final RMSNorm statistics (LM head and tails)
     if (a.P.has_head) {
         gemm_op<NT>(c, a.fb, a.P, OP_HEAD, st,
                     [&](int k_lo, int k_hi) { xload_normed<NT>(c, a, m.normf, k_lo, k_hi); },
                     [&](int tile, float (&acc)[NT][4]) { epi_head<NT>(c, a, row_dst, bias_at, tile, acc); });
+        stamp();
         grid_barrier(c, a.fb);
+        stamp();
         if (kind == KIND_VERIFY) {
             if (c.cta < g.rtot && row_dst[c.cta]) head_row_argmax(a, c.cta, top_sm);
         } else if (c.cta < g.batch && c.n_rows[c.cta] > 0) {
@@ -238,6 +257,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
         else if (kind == KIND_AR) tail_ar(c, a, c.cta);
         else if (kind == KIND_PREFILL || kind == KIND_PREFILL_B) tail_prefill(c, a, c.cta, which);
     }
+    stamp();
     // nothing of this warp's stream may still be in flight at exit
     while (st.cn < st.pn) { wait_unit(c, a.fb, st.cn); ++st.cn; }
 }

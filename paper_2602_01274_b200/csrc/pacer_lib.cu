@@ -28,6 +28,7 @@ struct pacer_ctx {
     int ncta;                  // blocks of the forward kernel (one per SM)
     std::map<int, fwd::Plan> plans;   // key: which * 16 + nt * 2 + has_head
     size_t part_floats;        // capacity of the split-k partial buffer
+    unsigned long long *prof_stamps;
     int batch;                 // sequences of the current run
     int prefilled;
     int64_t launches;
@@ -115,7 +116,7 @@ struct Carver {
 struct Layout {
     size_t st, x, y, alpha, hpend, hpend_e, draft_len, accept_len, verify_logits, draft_logits;
     size_t row_pos, row_tok, n_rows, row_arg, row_margin, xres, att, act, hidden, part;
-    size_t tile_cnt, att_cnt, bar, abort_flag, qkv, ssq, tile_top, attp;
+    size_t tile_cnt, att_cnt, bar, abort_flag, qkv, ssq, tile_top, attp, prof;
     size_t kc[3], vc[3], rope[3];
     size_t kv_bytes[3], rope_bytes[3];
     size_t total;
@@ -188,6 +189,7 @@ static Layout make_layout(const pacer_cfg &c) {
     L.att_cnt = cv.take(sizeof(int32_t) * (size_t)B * h_max);
     L.bar = cv.take(sizeof(unsigned long long));
     L.abort_flag = cv.take(sizeof(int32_t));
+    L.prof = cv.take(sizeof(unsigned long long) * fwd::PROF_STAMPS);
     L.state_bytes = cv.off;                                   // zeroed at create
     L.hpend = cv.take(sizeof(float) * B * (c.block_b + 1) * c.draft.d_model);
     L.verify_logits = cv.take(sizeof(float) * B * (gc + 1) * V);
@@ -269,6 +271,8 @@ extern "C" int pacer_create(const pacer_cfg *cfg, void *dev_workspace, size_t wo
     c->fb.ssq = (float *)(w + L.ssq); c->fb.tile_top = (float *)(w + L.tile_top); c->fb.attp = (float *)(w + L.attp);
     c->fb.att_cnt = (int32_t *)(w + L.att_cnt); c->fb.bar = (unsigned long long *)(w + L.bar);
     c->fb.abort_flag = (int32_t *)(w + L.abort_flag);
+    c->fb.prof = nullptr;
+    c->prof_stamps = (unsigned long long *)(w + L.prof);
     c->part_floats = L.part_bytes / sizeof(float);
     c->ncta = sm_count_or_default();
     d.max_batch = cfg->max_batch; d.max_ctx = cfg->max_ctx; d.gamma_cap = cfg->gamma_cap; d.block_b = cfg->block_b;
@@ -305,6 +309,7 @@ extern "C" int pacer_create(const pacer_cfg *cfg, void *dev_workspace, size_t wo
     reg(PACER_BUF_HPEND, d.hpend, sizeof(float) * B * (cfg->block_b + 1) * cfg->draft.d_model);
     reg(PACER_BUF_DRAFT_LEN, d.draft_len, sizeof(int32_t) * B * L.max_steps);
     reg(PACER_BUF_ACCEPT_LEN, d.accept_len, sizeof(int32_t) * B * L.max_steps);
+    reg(PACER_BUF_PHASE_NS, c->prof_stamps, sizeof(unsigned long long) * fwd::PROF_STAMPS);
     for (int i = 0; i < 3; ++i) {
         reg(PACER_BUF_KCACHE_T + 2 * i, c->model[i].kcache, L.kv_bytes[i]);
         reg(PACER_BUF_VCACHE_T + 2 * i, c->model[i].vcache, L.kv_bytes[i]);
@@ -402,6 +407,7 @@ static int run_forward(pacer_ctx *c, int which, const Geom &g, int kind, int aux
     }
     fwd::Args a;
     a.d = c->d; a.m = m; a.g = g; a.P = it->second; a.fb = c->fb; a.kind = kind; a.aux = aux;
+    a.fb.prof = (c->prof_on && which == PACER_TARGET) ? c->prof_stamps : nullptr;
     const bool prof = c->prof_on && which == PACER_TARGET && c->prof_used + 2 <= c->prof_ev.size();
     if (prof) CK(cudaEventRecord(c->prof_ev[c->prof_used], c->stream));
     CK(fwd::launch(a, which, c->ncta, c->stream));
