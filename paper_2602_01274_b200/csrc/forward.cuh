@@ -16,26 +16,32 @@
 //     the slices in slice order (deterministic) and applies the row-wise step
 //     that follows the projection in the decoder (residual add + RMS statistics,
 //     SwiGLU, bias/arg-max of the LM head), so no separate row kernels exist;
+//   - the streaming warps never wait on global-memory round trips: each hands
+//     its finished accumulators through shared memory to a partner "epilogue"
+//     warp, which does the stores, fences, arrival counting and row-wise steps;
 //   - phases are separated by grid barriers with bounded waits.
 #pragma once
 #include "common.cuh"
 
 namespace fwd {
 
-constexpr int THREADS = 256, WARPS = 8;
+constexpr int THREADS = 512, WARPS = 16;         // warps 0..7 stream weights and do the MMAs, warps 8..15 are their epilogue partners
+constexpr int MMA_WARPS = 8;
 constexpr int KC = 256;                         // k columns of one weight unit
 constexpr int PITCH = KC * 2 + 64;              // bytes between the rows of a stage (bank-conflict free)
 constexpr int STAGE_BYTES = 16 * PITCH;         // 9216
 constexpr int STAGES = 2;
-constexpr int RING_BYTES = WARPS * STAGES * STAGE_BYTES;   // 147456
+constexpr int RING_BYTES = MMA_WARPS * STAGES * STAGE_BYTES;   // 147456
 constexpr int XBUF_BYTES = 64 * 1024;           // activation slice of a projection item
-constexpr int SCRATCH_BYTES = 80 * 1024;        // XBUF, reused by the attention phase and the tails
+constexpr int HAND_BYTES = MMA_WARPS * 2048;    // accumulator hand-over buffers (4 row tiles x 4 x 32 lanes x fp32 each)
+constexpr int SCRATCH_BYTES = XBUF_BYTES + HAND_BYTES;   // the attention phase and the tails use both, contiguously
 constexpr int MISC_BYTES = 2048;
 constexpr int SMEM_BYTES = SCRATCH_BYTES + RING_BYTES + MISC_BYTES;
 constexpr int MAX_ROWS = 32;                    // rows of one forward (all sequences together)
 constexpr int MAX_SPLIT = 16;                   // key-range splits of one attention head
 constexpr unsigned SPIN_LIMIT = 1u << 22;
-constexpr int PROF_STAMPS = 1024;             // phase-boundary time stamps kept per forward
+constexpr int PROF_STAMPS = 512;              // phase-boundary time stamps kept per block and forward
+constexpr int PROF_BLOCKS = 256;              // blocks the stamp buffer has room for
 
 enum OpKind { OP_QKV = 0, OP_O = 1, OP_GU = 2, OP_DOWN = 3, OP_HEAD = 4, N_OPS = 5 };
 
@@ -67,7 +73,7 @@ struct FwdBufs {
     int32_t *att_cnt;        // [batch * H]
     unsigned long long *bar; // grid barrier counter
     int32_t *abort_flag;     // set when a bounded wait ran out
-    unsigned long long *prof; // optional: block 0 stamps %globaltimer at every phase boundary (NULL = off)
+    unsigned long long *prof; // optional: every block stamps %globaltimer at its phase boundaries (NULL = off)
 };
 
 // ------------------------------------------------------------------ PTX helpers
@@ -79,6 +85,9 @@ __device__ __forceinline__ void mbar_init(uint64_t *b, int count) {
 }
 __device__ __forceinline__ void mbar_expect_tx(uint64_t *b, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(b)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t *b) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(b)) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint64_t *b, uint32_t parity) {
     uint32_t ok;
@@ -127,6 +136,9 @@ struct Ctx {
     unsigned char *scratch;        // SCRATCH_BYTES
     unsigned char *ring;           // this warp's stages
     uint64_t *mbar;                // this warp's STAGES barriers
+    float *hand;                   // hand-over buffer of this warp pair
+    uint64_t *hand_full, *hand_empty;
+    int n_hand;                    // tiles handed over / received so far by this warp
     int32_t *row_pos, *row_tok;    // [MAX_ROWS]
     int32_t *n_rows;               // [MAX_ROWS] per sequence
     float *inv_rms;                // [MAX_ROWS]

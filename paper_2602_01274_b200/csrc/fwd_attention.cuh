@@ -10,6 +10,7 @@
 namespace fwd {
 
 constexpr int ATT_RB = 8;      // query rows handled together by a warp
+constexpr int ATT_WARPS = 8;   // warps that walk the keys (their partials are merged through shared memory)
 
 template <int EPL>             // channels per lane: hd = 32 * EPL
 __device__ __forceinline__ void load_kv_row(const bf16 *p, float (&out)[EPL]) {
@@ -38,7 +39,7 @@ __device__ __forceinline__ void attention_item(Ctx &c, const Args &a, int layer,
     float *qs = reinterpret_cast<float *>(c.scratch);                       // [MAX_ROWS][hd]
     bf16 *kn = reinterpret_cast<bf16 *>(qs + MAX_ROWS * hd);                // [MAX_ROWS][hd]
     bf16 *vn = kn + MAX_ROWS * hd;
-    float *red = reinterpret_cast<float *>(vn + MAX_ROWS * hd);             // [WARPS][ATT_RB][PW]
+    float *red = reinterpret_cast<float *>(vn + MAX_ROWS * hd);             // [ATT_WARPS][ATT_RB][PW]
     const size_t cbase = (((size_t)layer * d.max_batch + seq) * Hkv + kh) * (size_t)d.max_ctx * hd;
     const bool writer = split == 0 && h == kh * group;
     const float scale = rsqrtf((float)hd);
@@ -99,14 +100,15 @@ __device__ __forceinline__ void attention_item(Ctx &c, const Args &a, int layer,
                 }
             }
         };
-        for (int p = lo + c.warp; p < hi; p += WARPS) {          // cached keys: every new row sees them
+        const bool walker = c.warp < ATT_WARPS;
+        for (int p = lo + c.warp; walker && p < hi; p += ATT_WARPS) {   // cached keys: every new row sees them
             float kk[EPL], vv[EPL];
             load_kv_row<EPL>(kc + (size_t)p * hd, kk);
             load_kv_row<EPL>(vc + (size_t)p * hd, vv);
             one_key(kk, vv, 0);
         }
-        if (with_new) {                                          // new keys: row j sees new keys 0..j
-            for (int jn = c.warp; jn < n_r; jn += WARPS) {
+        if (with_new && walker) {                                // new keys: row j sees new keys 0..j
+            for (int jn = c.warp; jn < n_r; jn += ATT_WARPS) {
                 float kk[EPL], vv[EPL];
                 load_kv_row<EPL>(kn + jn * hd + c.lane * EPL, kk);
                 load_kv_row<EPL>(vn + jn * hd + c.lane * EPL, vv);
@@ -115,7 +117,7 @@ __device__ __forceinline__ void attention_item(Ctx &c, const Args &a, int layer,
         }
         // merge the warps' partials of this row block
 #pragma unroll
-        for (int jj = 0; jj < ATT_RB; ++jj) {
+        for (int jj = 0; walker && jj < ATT_RB; ++jj) {
             float *rw = red + ((size_t)c.warp * ATT_RB + jj) * PW;
 #pragma unroll
             for (int e = 0; e < EPL; ++e) rw[c.lane * EPL + e] = acc[jj][e];
@@ -126,10 +128,10 @@ __device__ __forceinline__ void attention_item(Ctx &c, const Args &a, int layer,
             const int jj = i / hd, ch = i - jj * hd;
             float M = -INFINITY;
 #pragma unroll
-            for (int w = 0; w < WARPS; ++w) M = fmaxf(M, red[((size_t)w * ATT_RB + jj) * PW + hd]);
+            for (int w = 0; w < ATT_WARPS; ++w) M = fmaxf(M, red[((size_t)w * ATT_RB + jj) * PW + hd]);
             float L = 0.f, o = 0.f;
 #pragma unroll
-            for (int w = 0; w < WARPS; ++w) {
+            for (int w = 0; w < ATT_WARPS; ++w) {
                 const float *rw = red + ((size_t)w * ATT_RB + jj) * PW;
                 const float f = rw[hd] == -INFINITY ? 0.f : __expf(rw[hd] - M);
                 L += rw[hd + 1] * f;

@@ -115,10 +115,15 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
     extern __shared__ __align__(1024) unsigned char smem[];
     Ctx c;
     c.warp = threadIdx.x >> 5; c.lane = threadIdx.x & 31; c.cta = blockIdx.x; c.ncta = gridDim.x;
+    const int pw = c.warp & (MMA_WARPS - 1);                                 // index of the warp pair
     c.scratch = smem;
-    c.ring = smem + SCRATCH_BYTES + c.warp * (STAGES * STAGE_BYTES);
+    c.hand = reinterpret_cast<float *>(smem + XBUF_BYTES + pw * (HAND_BYTES / MMA_WARPS));
+    c.ring = smem + SCRATCH_BYTES + pw * (STAGES * STAGE_BYTES);
     unsigned char *misc = smem + SCRATCH_BYTES + RING_BYTES;
-    c.mbar = reinterpret_cast<uint64_t *>(misc) + c.warp * STAGES;           // 8 * STAGES * 8 bytes
+    c.mbar = reinterpret_cast<uint64_t *>(misc) + pw * STAGES;               // 8 * STAGES * 8 bytes
+    c.hand_full = reinterpret_cast<uint64_t *>(misc + 128) + pw;             // 8 * 8 bytes
+    c.hand_empty = reinterpret_cast<uint64_t *>(misc + 192) + pw;
+    c.n_hand = 0;
     c.row_pos = reinterpret_cast<int32_t *>(misc + 256);
     c.row_tok = c.row_pos + MAX_ROWS;
     c.n_rows = c.row_tok + MAX_ROWS;
@@ -180,8 +185,11 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
         const unsigned long long v = ld_acquire_u64(a.fb.bar);
         c.bar_target = v / (unsigned long long)c.ncta * (unsigned long long)c.ncta;
     }
-    if (c.lane == 0)
+    if (c.lane == 0 && c.warp < MMA_WARPS) {
         for (int i = 0; i < STAGES; ++i) mbar_init(c.mbar + i, 1);
+        mbar_init(c.hand_full, 1);
+        mbar_init(c.hand_empty, 1);
+    }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_proxy_async();
     __syncthreads();
@@ -190,14 +198,19 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
     Stream st;
     st.cu.q = st.cu.m = st.cu.j = st.cu.u = 0; st.cu.done = 0;
     st.pn = st.cn = 0;
-    settle(st.cu, a.P, c.cta, c.ncta, c.warp);
-    for (int i = 0; i < STAGES; ++i) issue_unit(c, st, a.P);
+    if (c.warp < MMA_WARPS) {
+        settle(st.cu, a.P, c.cta, c.ncta, c.warp);
+        for (int i = 0; i < STAGES; ++i) issue_unit(c, st, a.P);
+    } else {
+        st.cu.done = 1;
+    }
 
     constexpr int RPAD = NT * 8;
     const int dm = m.cfg.d_model;
     int n_stamp = 0;
     auto stamp = [&]() {
-        if (a.fb.prof && c.cta == 0 && threadIdx.x == 0 && n_stamp < PROF_STAMPS) a.fb.prof[n_stamp++] = globaltimer_ns();
+        if (a.fb.prof && threadIdx.x == 0 && n_stamp < PROF_STAMPS)
+            a.fb.prof[(size_t)c.cta * PROF_STAMPS + n_stamp++] = globaltimer_ns();
     };
     stamp();
     phase_begin(c, a, RPAD);
@@ -294,7 +307,7 @@ static inline void plan_op(GemmOp &op, int ncta, int NT, int rot) {
                     const int s = i % S, g = i / S;
                     const int tiles = std::min(TPG, MT - g * TPG), len = std::min(ksc, chunks - s * ksc);
                     // bytes in units of one tile x one 32-chunk, plus the price of loading the item's activations
-                    load[(i + rot) % ncta] += (long long)((tiles + WARPS - 1) / WARPS) * WARPS * len / 2 +
+                    load[(i + rot) % ncta] += (long long)((tiles + MMA_WARPS - 1) / MMA_WARPS) * MMA_WARPS * len / 2 +
                                               (long long)tiles * len / 2 + 3 * len;
                 }
                 const long long mk = *std::max_element(load.begin(), load.end());

@@ -109,12 +109,13 @@ __device__ __forceinline__ void compute_inv(Ctx &c, const Args &a) {
     const int dm = a.m.cfg.d_model, ntiles = dm >> 4;
     const int r = threadIdx.x >> 3, sub = threadIdx.x & 7;
     float s = 0.f;
-    for (int t = sub; t < ntiles; t += 8) s += __ldcg(a.fb.ssq + t * MAX_ROWS + r);
+    if (r < MAX_ROWS)
+        for (int t = sub; t < ntiles; t += 8) s += __ldcg(a.fb.ssq + t * MAX_ROWS + r);
     s += __shfl_xor_sync(0xffffffffu, s, 1);
     s += __shfl_xor_sync(0xffffffffu, s, 2);
     s += __shfl_xor_sync(0xffffffffu, s, 4);
     __syncthreads();                            // earlier readers of inv_rms are done
-    if (sub == 0) c.inv_rms[r] = rsqrtf(s / (float)dm + a.m.cfg.rms_eps);
+    if (sub == 0 && r < MAX_ROWS) c.inv_rms[r] = rsqrtf(s / (float)dm + a.m.cfg.rms_eps);
     __syncthreads();
 }
 

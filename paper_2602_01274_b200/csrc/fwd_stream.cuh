@@ -32,7 +32,7 @@ __device__ __forceinline__ bool settle(Cursor &cu, const Plan &P, int cta, int n
         if (idx >= op.items) { ++cu.q; cu.m = cu.j = cu.u = 0; continue; }
         const int s = idx % op.S, g = idx / op.S;
         const int t_lo = g * op.TPG, t_hi = min(op.MT, t_lo + op.TPG);
-        const int tile = t_lo + warp + WARPS * cu.j;
+        const int tile = t_lo + warp + MMA_WARPS * cu.j;
         if (tile >= t_hi) { ++cu.m; cu.j = cu.u = 0; continue; }
         const int k_lo = s * op.KS, k_hi = min(op.K, k_lo + op.KS);
         const int k = k_lo + cu.u * KC;
@@ -78,17 +78,45 @@ __device__ __forceinline__ void issue_unit(Ctx &c, Stream &st, const Plan &P) {
     settle(st.cu, P, c.cta, c.ncta, c.warp);
 }
 
-// Bounded wait for the stage that holds unit number n of this warp.
-__device__ __forceinline__ void wait_unit(Ctx &c, const FwdBufs &fb, int n) {
-    uint64_t *bar = c.mbar + (n % STAGES);
-    const uint32_t parity = (uint32_t)(n / STAGES) & 1u;
+// Bounded wait on a shared-memory barrier phase.
+__device__ __forceinline__ void wait_bar(Ctx &c, const FwdBufs &fb, uint64_t *bar, uint32_t parity, int code) {
     unsigned it = 0;
     while (!mbar_try_wait(bar, parity)) {
         if (++it > SPIN_LIMIT) {
-            if (c.lane == 0) atomicExch(fb.abort_flag, 2);
+            if (c.lane == 0) atomicExch(fb.abort_flag, code);
             break;
         }
     }
+}
+
+// Bounded wait for the stage that holds unit number n of this warp.
+__device__ __forceinline__ void wait_unit(Ctx &c, const FwdBufs &fb, int n) {
+    wait_bar(c, fb, c.mbar + (n % STAGES), (uint32_t)(n / STAGES) & 1u, 2);
+}
+
+// Streaming warp -> its epilogue partner: the accumulators of a finished tile,
+// through shared memory in lane order (conflict free), one tile at a time.
+template <int NT>
+__device__ __forceinline__ void hand_over(Ctx &c, const FwdBufs &fb, const float (&acc)[NT][4]) {
+    wait_bar(c, fb, c.hand_empty, ((uint32_t)c.n_hand & 1u) ^ 1u, 3);      // the partner took the previous tile
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) c.hand[(nt * 4 + i) * 32 + c.lane] = acc[nt][i];
+    __syncwarp();
+    if (c.lane == 0) mbar_arrive(c.hand_full);
+    ++c.n_hand;
+}
+template <int NT>
+__device__ __forceinline__ void receive(Ctx &c, const FwdBufs &fb, float (&acc)[NT][4]) {
+    wait_bar(c, fb, c.hand_full, (uint32_t)c.n_hand & 1u, 4);
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) acc[nt][i] = c.hand[(nt * 4 + i) * 32 + c.lane];
+    __syncwarp();
+    if (c.lane == 0) mbar_arrive(c.hand_empty);
+    ++c.n_hand;
 }
 
 // acc[nt] += W(16 rows x 32*nchunks k) * X over one stage.  Lane (g, t) reads the
@@ -170,14 +198,17 @@ __device__ __forceinline__ bool tile_reduce(Ctx &c, const FwdBufs &fb, const Gem
 }
 
 // One projection: for every item of this block load the activation slice, then
-// every warp streams its tiles through its pipeline.  xload(k_lo, k_hi) fills the
-// scratch with the slice in fragment order (all threads call it); epi(tile, acc)
-// runs in the warp that completed the tile.
+// every streaming warp runs its tiles through its pipeline and hands each
+// finished tile to its partner.  xload(k_lo, k_hi) fills the scratch with the
+// slice in fragment order (all threads call it); epi(tile, acc) runs in the
+// epilogue warp that completed the tile (last k slice to arrive).
 template <int NT, class XLoad, class Epi>
 __device__ __forceinline__ void gemm_op(Ctx &c, const FwdBufs &fb, const Plan &P, int opi, Stream &st, XLoad xload,
                                         Epi epi) {
     const GemmOp &op = P.op[opi];
     const uint4 *xs = reinterpret_cast<const uint4 *>(c.scratch);
+    const bool streamer = c.warp < MMA_WARPS;
+    const int w = c.warp & (MMA_WARPS - 1);
     for (int idx = first_item(op, c.cta, c.ncta); idx < op.items; idx += c.ncta) {
         const int s = idx % op.S, g = idx / op.S;
         const int k_lo = s * op.KS, k_hi = min(op.K, k_lo + op.KS);
@@ -185,20 +216,25 @@ __device__ __forceinline__ void gemm_op(Ctx &c, const FwdBufs &fb, const Plan &P
         __syncthreads();                       // the scratch is free
         xload(k_lo, k_hi);
         __syncthreads();
-        for (int tile = t_lo + c.warp; tile < t_hi; tile += WARPS) {
+        for (int tile = t_lo + w; tile < t_hi; tile += MMA_WARPS) {
             float acc[NT][4];
+            if (streamer) {
 #pragma unroll
-            for (int nt = 0; nt < NT; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
-            for (int k = k_lo; k < k_hi; k += KC) {
-                const int kc = min(KC, k_hi - k);
-                wait_unit(c, fb, st.cn);
-                consume_unit<NT>(c.ring + (st.cn % STAGES) * STAGE_BYTES, xs, (k - k_lo) >> 5, kc >> 5, acc, c.lane);
-                ++st.cn;
-                __syncwarp();
-                fence_proxy_async();
-                issue_unit(c, st, P);          // refill the freed stage with the next unit of the static list
+                for (int nt = 0; nt < NT; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
+                for (int k = k_lo; k < k_hi; k += KC) {
+                    const int kc = min(KC, k_hi - k);
+                    wait_unit(c, fb, st.cn);
+                    consume_unit<NT>(c.ring + (st.cn % STAGES) * STAGE_BYTES, xs, (k - k_lo) >> 5, kc >> 5, acc, c.lane);
+                    ++st.cn;
+                    __syncwarp();
+                    fence_proxy_async();
+                    issue_unit(c, st, P);      // refill the freed stage with the next unit of the static list
+                }
+                hand_over<NT>(c, fb, acc);
+            } else {
+                receive<NT>(c, fb, acc);
+                if (tile_reduce<NT>(c, fb, op, tile, s, acc)) epi(tile, acc);
             }
-            if (tile_reduce<NT>(c, fb, op, tile, s, acc)) epi(tile, acc);
         }
     }
 }

@@ -189,7 +189,7 @@ static Layout make_layout(const pacer_cfg &c) {
     L.att_cnt = cv.take(sizeof(int32_t) * (size_t)B * h_max);
     L.bar = cv.take(sizeof(unsigned long long));
     L.abort_flag = cv.take(sizeof(int32_t));
-    L.prof = cv.take(sizeof(unsigned long long) * fwd::PROF_STAMPS);
+    L.prof = cv.take(sizeof(unsigned long long) * fwd::PROF_STAMPS * fwd::PROF_BLOCKS);
     L.state_bytes = cv.off;                                   // zeroed at create
     L.hpend = cv.take(sizeof(float) * B * (c.block_b + 1) * c.draft.d_model);
     L.verify_logits = cv.take(sizeof(float) * B * (gc + 1) * V);
@@ -309,7 +309,7 @@ extern "C" int pacer_create(const pacer_cfg *cfg, void *dev_workspace, size_t wo
     reg(PACER_BUF_HPEND, d.hpend, sizeof(float) * B * (cfg->block_b + 1) * cfg->draft.d_model);
     reg(PACER_BUF_DRAFT_LEN, d.draft_len, sizeof(int32_t) * B * L.max_steps);
     reg(PACER_BUF_ACCEPT_LEN, d.accept_len, sizeof(int32_t) * B * L.max_steps);
-    reg(PACER_BUF_PHASE_NS, c->prof_stamps, sizeof(unsigned long long) * fwd::PROF_STAMPS);
+    reg(PACER_BUF_PHASE_NS, c->prof_stamps, sizeof(unsigned long long) * fwd::PROF_STAMPS * fwd::PROF_BLOCKS);
     for (int i = 0; i < 3; ++i) {
         reg(PACER_BUF_KCACHE_T + 2 * i, c->model[i].kcache, L.kv_bytes[i]);
         reg(PACER_BUF_VCACHE_T + 2 * i, c->model[i].vcache, L.kv_bytes[i]);
@@ -407,7 +407,7 @@ static int run_forward(pacer_ctx *c, int which, const Geom &g, int kind, int aux
     }
     fwd::Args a;
     a.d = c->d; a.m = m; a.g = g; a.P = it->second; a.fb = c->fb; a.kind = kind; a.aux = aux;
-    a.fb.prof = (c->prof_on && which == PACER_TARGET) ? c->prof_stamps : nullptr;
+    a.fb.prof = (c->prof_on && which == PACER_TARGET && c->ncta <= fwd::PROF_BLOCKS) ? c->prof_stamps : nullptr;
     const bool prof = c->prof_on && which == PACER_TARGET && c->prof_used + 2 <= c->prof_ev.size();
     if (prof) CK(cudaEventRecord(c->prof_ev[c->prof_used], c->stream));
     CK(fwd::launch(a, which, c->ncta, c->stream));
