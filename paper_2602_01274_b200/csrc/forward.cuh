@@ -1,42 +1,46 @@
 // One decoder forward as ONE persistent cooperative kernel (one block per SM).
 //
 // The forward is bound by streaming the weights from HBM once, so the kernel is
-// built around an uninterrupted weight stream:
-//   - every warp owns a private pipeline of shared-memory stages that it fills
-//     itself with bulk async copies (cp.async.bulk + mbarrier) of 16 weight rows
-//     x 256 k each; the list of (projection, tile, k-range) units a warp will
-//     need is static, so a warp keeps issuing copies for the NEXT projection
-//     while the block sits in a grid barrier or in a small phase (attention,
-//     tail): the HBM queue never drains between projections;
-//   - the few activation rows of a projection live in shared memory in MMA
-//     fragment order; tensor cores (mma.m16n8k16, bf16 in / fp32 accumulate,
-//     weights as the 16-row operand) do the contraction, so the math is invisible;
-//   - a projection is cut into (k-slice, column-group) items spread over the
-//     blocks; the warp that delivers the last k-slice of a 16-column tile sums
-//     the slices in slice order (deterministic) and applies the row-wise step
-//     that follows the projection in the decoder (residual add + RMS statistics,
-//     SwiGLU, bias/arg-max of the LM head), so no separate row kernels exist;
-//   - the streaming warps never wait on global-memory round trips: each hands
-//     its finished accumulators through shared memory to a partner "epilogue"
-//     warp, which does the stores, fences, arrival counting and row-wise steps;
+// built around an uninterrupted weight stream and a critical path with as few
+// dependent global-memory round trips as possible:
+//   - a producer warp walks the static list of weight units (16 rows x 256 k)
+//     of the block for the WHOLE forward and keeps a shared-memory ring full
+//     with bulk async copies (cp.async.bulk + mbarrier); it runs ahead into the
+//     next projection while the block sits in a grid barrier or in a small
+//     phase, so the HBM queue never drains between projections;
+//   - a block owns whole 16-row tiles of a projection over the full k extent
+//     (no split-k: no partial sums, no atomics, no fences), the eight MMA warps
+//     advance over k in lockstep, and the activation rows of each 256-wide k
+//     step arrive through a second small ring, copied by a second producer warp
+//     from a bf16 buffer that already has MMA fragment order;
+//   - tensor cores (mma.m16n8k16, bf16 in / fp32 accumulate, weights as the
+//     16-row operand) do the contraction, so the math is invisible;
+//   - the row-wise step that follows a projection in the decoder (residual add,
+//     RMSNorm input of the next projection, SwiGLU, bias/arg-max of the LM head)
+//     is the epilogue of the warp that owns the tile; RMSNorm's 1/rms factor is
+//     applied to the OUTPUT rows of the next projection, so its input can be
+//     written before the row's sum of squares is complete;
 //   - phases are separated by grid barriers with bounded waits.
 #pragma once
 #include "common.cuh"
 
 namespace fwd {
 
-constexpr int THREADS = 512, WARPS = 16;         // warps 0..7 stream weights and do the MMAs, warps 8..15 are their epilogue partners
-constexpr int MMA_WARPS = 8;
+constexpr int MMA_WARPS = 8, MMA_THREADS = 256;  // warps 0..7: MMAs, epilogues and all block-wide phases
+constexpr int W_PRODUCER = 8, X_PRODUCER = 9;    // warp 8 streams weights, warp 9 activations (and RMS statistics)
+constexpr int THREADS = 320;
 constexpr int KC = 256;                         // k columns of one weight unit
 constexpr int PITCH = KC * 2 + 64;              // bytes between the rows of a stage (bank-conflict free)
 constexpr int STAGE_BYTES = 16 * PITCH;         // 9216
-constexpr int STAGES = 2;
-constexpr int RING_BYTES = MMA_WARPS * STAGES * STAGE_BYTES;   // 147456
-constexpr int XBUF_BYTES = 64 * 1024;           // activation slice of a projection item
-constexpr int HAND_BYTES = MMA_WARPS * 2048;    // accumulator hand-over buffers (4 row tiles x 4 x 32 lanes x fp32 each)
-constexpr int SCRATCH_BYTES = XBUF_BYTES + HAND_BYTES;   // the attention phase and the tails use both, contiguously
+constexpr int NS = 16;                          // weight stages in the ring
+constexpr int RING_BYTES = NS * STAGE_BYTES;    // 147456
+constexpr int XS = 3;                           // activation stages
+constexpr int XSTAGE_BYTES = 4 * 4096;          // up to 4 row tiles x 8 chunks x 512 bytes
+constexpr int SCRATCH_BYTES = 80 * 1024;        // the activation ring lives in its first 48 KB; the attention
+                                                // phase and the tails use all of it (no activations in flight then)
 constexpr int MISC_BYTES = 2048;
 constexpr int SMEM_BYTES = SCRATCH_BYTES + RING_BYTES + MISC_BYTES;
+constexpr int MAX_TILES = 16;                   // tiles of one pass of a block (two per MMA warp)
 constexpr int MAX_ROWS = 32;                    // rows of one forward (all sequences together)
 constexpr int MAX_SPLIT = 16;                   // key-range splits of one attention head
 constexpr unsigned SPIN_LIMIT = 1u << 22;
@@ -45,15 +49,16 @@ constexpr int PROF_BLOCKS = 256;              // blocks the stamp buffer has roo
 
 enum OpKind { OP_QKV = 0, OP_O = 1, OP_GU = 2, OP_DOWN = 3, OP_HEAD = 4, N_OPS = 5 };
 
-// One weight-streaming projection, cut into items = (k slice s, tile group g).
+// One weight-streaming projection.  Block c owns the contiguous tiles
+// [t0, t0 + T) given by tile_range(); it runs them in passes of MAX_TILES.
 struct GemmOp {
     const bf16 *W1, *W2;     // layer-0 base; W2 only for the interleaved gate/up projection
+    const bf16 *X;           // activations, bf16 in fragment order [K/32][row tiles][32 lanes][8]
     long long lstride;       // elements between layers
     int32_t N;               // weight rows in all (gate/up: 2F)
     int32_t MT;              // 16-row tiles
-    int32_t K, S, KS;        // k extent, slices, slice length (multiple of 32)
-    int32_t G, TPG;          // tile groups, tiles per group
-    int32_t items, rot;      // S*G; block that gets item 0
+    int32_t K;
+    int32_t rot;             // block that gets the first tile range (spreads the one-tile imbalance)
     int32_t interleave;      // 1: tile t = gate rows 8t..8t+7 then up rows 8t..8t+7
 };
 
@@ -64,12 +69,11 @@ struct Plan {
 
 // Device buffers of the forward kernel beyond DevPtrs (all in the workspace).
 struct FwdBufs {
-    float *qkv;              // [MAX_ROWS][qrows] fp32, complete sums
-    float *part;             // split-k partial tiles [S][MT][rpad][16]
-    int32_t *tile_cnt;       // [MT max] arrivals per tile, zero between projections
+    float *qkv;              // [MAX_ROWS][qrows] fp32
+    bf16 *xg;                // x * gain of the next RMSNorm, bf16 in fragment order (its 1/rms comes later)
     float *ssq;              // [d/16][MAX_ROWS] sum of squares of x over the 16 columns of a tile
     float *tile_top;         // [MT(head)][MAX_ROWS][4]: max, argmax (int bits), runner-up, unused
-    float *attp;             // attention partials [item][MAX_ROWS][hd + 2]
+    float *attp;             // attention partials [seq*H + h][split][row][hd + 2]
     int32_t *att_cnt;        // [batch * H]
     unsigned long long *bar; // grid barrier counter
     int32_t *abort_flag;     // set when a bounded wait ran out
@@ -133,40 +137,54 @@ __device__ __forceinline__ void mma16816(float (&c)[4], uint32_t a0, uint32_t a1
 
 struct Ctx {
     // shared memory
-    unsigned char *scratch;        // SCRATCH_BYTES
-    unsigned char *ring;           // this warp's stages
-    uint64_t *mbar;                // this warp's STAGES barriers
-    float *hand;                   // hand-over buffer of this warp pair
-    uint64_t *hand_full, *hand_empty;
-    int n_hand;                    // tiles handed over / received so far by this warp
+    unsigned char *scratch;        // SCRATCH_BYTES (activation ring in front)
+    unsigned char *ring;           // weight ring
+    uint64_t *wfull, *wempty;      // [NS]
+    uint64_t *xfull, *xempty;      // [XS]
     int32_t *row_pos, *row_tok;    // [MAX_ROWS]
     int32_t *n_rows;               // [MAX_ROWS] per sequence
     float *inv_rms;                // [MAX_ROWS]
+    volatile int32_t *ready_op;    // [0] projections whose inputs are complete; [1] projections whose inv_rms is ready
     int32_t *flag;                 // block-wide scratch word
     // registers
     unsigned long long bar_target; // used by thread 0
     int warp, lane, cta, ncta;
     uint64_t policy;
+    int wn, xn;                    // weight units / activation chunks of this block consumed (or produced) so far
 };
 
-// Grid barrier: every block arrives once; waits are bounded.  A wait that runs
+// Barrier of the eight MMA warps (the producer warps never join it).
+__device__ __forceinline__ void bsync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+
+// Tile range of block `cta` for a projection with MT tiles.
+__device__ __host__ __forceinline__ void tile_range(int MT, int rot, int cta, int ncta, int &t0, int &T) {
+    int ci = cta - rot;
+    if (ci < 0) ci += ncta;
+    const int base = MT / ncta, rem = MT % ncta;
+    T = base + (ci < rem ? 1 : 0);
+    t0 = ci * base + (ci < rem ? ci : rem);
+}
+
+// Grid barrier (MMA warps only): every block arrives once; waits are bounded.  A wait that runs
 // out raises the abort flag, after which all later barriers fall through.
 __device__ __forceinline__ void grid_barrier(Ctx &c, const FwdBufs &fb) {
-    __syncthreads();
+    asm volatile("fence.proxy.async;" ::: "memory");   // this thread's global writes, for bulk copies issued later
+    bsync();
     if (threadIdx.x == 0) {
         c.bar_target += (unsigned long long)c.ncta;
         __threadfence();
         atomicAdd(fb.bar, 1ULL);
         unsigned it = 0;
         while (ld_acquire_u64(fb.bar) < c.bar_target) {
-            if (++it > SPIN_LIMIT || *(volatile int32_t *)fb.abort_flag) {
-                atomicExch(fb.abort_flag, 1);
+            ++it;
+            if ((it & 255u) == 0 && (it > SPIN_LIMIT || *(volatile int32_t *)fb.abort_flag)) {
+                atomicCAS(fb.abort_flag, 0, 1);
                 break;
             }
         }
         __threadfence();
     }
-    __syncthreads();
+    bsync();
 }
 
 }  // namespace fwd

@@ -10,7 +10,7 @@
 namespace fwd {
 
 constexpr int ATT_RB = 8;      // query rows handled together by a warp
-constexpr int ATT_WARPS = 8;   // warps that walk the keys (their partials are merged through shared memory)
+constexpr int ATT_WARPS = MMA_WARPS;
 
 template <int EPL>             // channels per lane: hd = 32 * EPL
 __device__ __forceinline__ void load_kv_row(const bf16 *p, float (&out)[EPL]) {
@@ -45,7 +45,7 @@ __device__ __forceinline__ void attention_item(Ctx &c, const Args &a, int layer,
     const float scale = rsqrtf((float)hd);
 
     // rotary embedding of the new rows (rotate-half pairs (i, i + hd/2)); k and v rounded to bf16 as cached
-    for (int i = threadIdx.x; i < n_r * half; i += THREADS) {
+    for (int i = threadIdx.x; i < n_r * half; i += MMA_THREADS) {
         const int j = i / half, ii = i - j * half, pos = pos0 + j;
         const float *row = a.fb.qkv + (size_t)(r_base + j) * qrows;
         const float2 cs = m.rope[(size_t)pos * half + ii];
@@ -64,7 +64,7 @@ __device__ __forceinline__ void attention_item(Ctx &c, const Args &a, int layer,
             vc[ii] = v0; vc[ii + half] = v1;
         }
     }
-    __syncthreads();
+    bsync();
 
     const int lo = (int)((long long)pos0 * split / nsplit), hi = (int)((long long)pos0 * (split + 1) / nsplit);
     const bool with_new = split == nsplit - 1;
@@ -100,7 +100,7 @@ __device__ __forceinline__ void attention_item(Ctx &c, const Args &a, int layer,
                 }
             }
         };
-        const bool walker = c.warp < ATT_WARPS;
+        const bool walker = true;
         for (int p = lo + c.warp; walker && p < hi; p += ATT_WARPS) {   // cached keys: every new row sees them
             float kk[EPL], vv[EPL];
             load_kv_row<EPL>(kc + (size_t)p * hd, kk);
@@ -123,8 +123,8 @@ __device__ __forceinline__ void attention_item(Ctx &c, const Args &a, int layer,
             for (int e = 0; e < EPL; ++e) rw[c.lane * EPL + e] = acc[jj][e];
             if (c.lane == 0) { rw[hd] = mx[jj]; rw[hd + 1] = den[jj]; }
         }
-        __syncthreads();
-        for (int i = threadIdx.x; i < nrb * hd; i += THREADS) {
+        bsync();
+        for (int i = threadIdx.x; i < nrb * hd; i += MMA_THREADS) {
             const int jj = i / hd, ch = i - jj * hd;
             float M = -INFINITY;
 #pragma unroll
@@ -141,22 +141,22 @@ __device__ __forceinline__ void attention_item(Ctx &c, const Args &a, int layer,
             op[ch] = o;
             if (ch == 0) { op[hd] = M; op[hd + 1] = L; }
         }
-        __syncthreads();
+        bsync();
     }
 
     // the item that finishes last for (seq, h) merges the splits
     __threadfence();
-    __syncthreads();
+    bsync();
     if (threadIdx.x == 0) {
         const int old = atomicAdd(a.fb.att_cnt + seq * H + h, 1);
         c.flag[0] = old == nsplit - 1;
         if (old == nsplit - 1) a.fb.att_cnt[seq * H + h] = 0;
     }
-    __syncthreads();
+    bsync();
     if (c.flag[0]) {
         __threadfence();
         const float *base = a.fb.attp + ((size_t)(seq * H + h) * MAX_SPLIT) * a.g.rps * PW;
-        for (int i = threadIdx.x; i < n_r * hd; i += THREADS) {
+        for (int i = threadIdx.x; i < n_r * hd; i += MMA_THREADS) {
             const int j = i / hd, ch = i - j * hd;
             float M = -INFINITY;
             for (int sp = 0; sp < nsplit; ++sp) M = fmaxf(M, __ldcg(base + ((size_t)sp * a.g.rps + j) * PW + hd));
@@ -171,7 +171,7 @@ __device__ __forceinline__ void attention_item(Ctx &c, const Args &a, int layer,
             d.att[xfrag_index(r_base + j, h * hd + ch, nt_total)] = __float2bfloat16(o / L);
         }
     }
-    __syncthreads();
+    bsync();
 }
 
 // All blocks: the attention of one layer.

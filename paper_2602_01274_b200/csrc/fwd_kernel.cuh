@@ -1,5 +1,5 @@
-// The forward kernel itself, the tails that take the loop's decisions, the host
-// planner that cuts the projections into items, and the cooperative launch.
+// The forward kernel itself, the tails that take the loop's decisions (Eq. 6 /
+// Eq. 7 / Algorithm 1) on the device, the host-side plan and the cooperative launch.
 #pragma once
 #include <algorithm>
 #include <vector>
@@ -23,9 +23,9 @@ __device__ __forceinline__ void tail_draft(Ctx &c, const Args &a, int s) {
     const int gamma = st.gamma, n_pend = st.n_pend, r_last = s * a.g.rps + n_in - 1;
     for (int jj = 0; jj < n_in; ++jj) {
         float *dst = d.hpend + ((size_t)s * (d.block_b + 1) + n_pend + jj) * dm;
-        for (int i = threadIdx.x; i < dm; i += THREADS) dst[i] = hidden_at(a, c, s * a.g.rps + jj, i);
+        for (int i = threadIdx.x; i < dm; i += MMA_THREADS) dst[i] = hidden_at(a, c, s * a.g.rps + jj, i);
     }
-    __syncthreads();
+    bsync();
     if (threadIdx.x == 0) {
         for (int jj = 0; jj < n_in; ++jj)
             d.hpend_e[s * (d.block_b + 1) + n_pend + jj] = (jj == n_in - 1) ? gamma + 1 : 0;
@@ -48,16 +48,16 @@ __device__ __forceinline__ void tail_mb(Ctx &c, const Args &a, int s) {
         const int r = s * a.g.rps + j, e = c.row_tok[r];
         if (e == 0) continue;
         float z0 = 0.f, z1 = 0.f;
-        for (int i = threadIdx.x; i < dm; i += THREADS) {
+        for (int i = threadIdx.x; i < dm; i += MMA_THREADS) {
             const float hv = hidden_at(a, c, r, i);
             z0 += hv * __bfloat162float(a.m.head_b[i]);
             z1 += hv * __bfloat162float(a.m.head_b[dm + i]);
         }
-        z0 = block_sum(z0, red);
-        z1 = block_sum(z1, red);
+        z0 = mma_block_sum(z0, red);
+        z1 = mma_block_sum(z1, red);
         if (threadIdx.x == 0) d.alpha[(size_t)s * d.gamma_cap + e - 1] = 1.f / (1.f + expf(z0 - z1));
     }
-    __syncthreads();
+    bsync();
     if (threadIdx.x == 0) {
         const int b = d.block_b, gamma = st.gamma;
         const float *ab = d.alpha + (size_t)s * d.gamma_cap + (gamma - b);
@@ -85,7 +85,7 @@ __device__ __forceinline__ void tail_prefill(Ctx &c, const Args &a, int s, int w
     if (which == PACER_DRAFT)
         for (int j = 0; j < n; ++j) {
             const int r = s * a.g.rps + j;
-            for (int i = threadIdx.x; i < dm; i += THREADS) d.hidden[(size_t)r * dm + i] = hidden_at(a, c, r, i);
+            for (int i = threadIdx.x; i < dm; i += MMA_THREADS) d.hidden[(size_t)r * dm + i] = hidden_at(a, c, r, i);
         }
     if (threadIdx.x == 0) {
         SeqState &st = d.st[s];
@@ -115,24 +115,24 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
     extern __shared__ __align__(1024) unsigned char smem[];
     Ctx c;
     c.warp = threadIdx.x >> 5; c.lane = threadIdx.x & 31; c.cta = blockIdx.x; c.ncta = gridDim.x;
-    const int pw = c.warp & (MMA_WARPS - 1);                                 // index of the warp pair
     c.scratch = smem;
-    c.hand = reinterpret_cast<float *>(smem + XBUF_BYTES + pw * (HAND_BYTES / MMA_WARPS));
-    c.ring = smem + SCRATCH_BYTES + pw * (STAGES * STAGE_BYTES);
+    c.ring = smem + SCRATCH_BYTES;
     unsigned char *misc = smem + SCRATCH_BYTES + RING_BYTES;
-    c.mbar = reinterpret_cast<uint64_t *>(misc) + pw * STAGES;               // 8 * STAGES * 8 bytes
-    c.hand_full = reinterpret_cast<uint64_t *>(misc + 128) + pw;             // 8 * 8 bytes
-    c.hand_empty = reinterpret_cast<uint64_t *>(misc + 192) + pw;
-    c.n_hand = 0;
-    c.row_pos = reinterpret_cast<int32_t *>(misc + 256);
+    c.wfull = reinterpret_cast<uint64_t *>(misc);                            // NS
+    c.wempty = c.wfull + NS;                                                 // NS
+    c.xfull = c.wempty + NS;                                                 // XS
+    c.xempty = c.xfull + XS;                                                 // XS  (ends at 8 * (2*NS + 2*XS) = 304)
+    c.row_pos = reinterpret_cast<int32_t *>(misc + 320);
     c.row_tok = c.row_pos + MAX_ROWS;
     c.n_rows = c.row_tok + MAX_ROWS;
     c.inv_rms = reinterpret_cast<float *>(c.n_rows + MAX_ROWS);
-    c.flag = reinterpret_cast<int32_t *>(c.inv_rms + MAX_ROWS);              // 4 words
+    c.ready_op = reinterpret_cast<volatile int32_t *>(c.inv_rms + MAX_ROWS); // 2 words
+    c.flag = reinterpret_cast<int32_t *>(misc + 320 + 4 * 128 + 16);         // 4 words
     float **row_dst = reinterpret_cast<float **>(misc + 1024);               // [MAX_ROWS]
     int32_t *bias_at = reinterpret_cast<int32_t *>(misc + 1024 + 256);       // [MAX_ROWS]
-    Top2 *top_sm = reinterpret_cast<Top2 *>(misc + 1024 + 384);              // [32]
+    Top2 *top_sm = reinterpret_cast<Top2 *>(misc + 1024 + 384);              // [8]
     c.bar_target = 0;
+    c.wn = c.xn = 0;
     c.policy = policy_evict_first();
     const DevPtrs &d = a.d;
     const ModelDev &m = a.m;
@@ -184,28 +184,23 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
     if (threadIdx.x == 0) {
         const unsigned long long v = ld_acquire_u64(a.fb.bar);
         c.bar_target = v / (unsigned long long)c.ncta * (unsigned long long)c.ncta;
+        for (int i = 0; i < NS; ++i) { mbar_init(c.wfull + i, 1); mbar_init(c.wempty + i, 1); }
+        for (int i = 0; i < XS; ++i) { mbar_init(c.xfull + i, 1); mbar_init(c.xempty + i, MMA_WARPS); }
+        c.ready_op[0] = 0; c.ready_op[1] = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (c.lane == 0 && c.warp < MMA_WARPS) {
-        for (int i = 0; i < STAGES; ++i) mbar_init(c.mbar + i, 1);
-        mbar_init(c.hand_full, 1);
-        mbar_init(c.hand_empty, 1);
-    }
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_proxy_async();
     __syncthreads();
 
-    // start the weight stream: it runs ahead of the phases from here on
-    Stream st;
-    st.cu.q = st.cu.m = st.cu.j = st.cu.u = 0; st.cu.done = 0;
-    st.pn = st.cn = 0;
-    if (c.warp < MMA_WARPS) {
-        settle(st.cu, a.P, c.cta, c.ncta, c.warp);
-        for (int i = 0; i < STAGES; ++i) issue_unit(c, st, a.P);
-    } else {
-        st.cu.done = 1;
+    // the two producer warps live in their streams until the forward's last unit
+    if (c.warp == W_PRODUCER) { weight_producer(c, a.fb, a.P); return; }
+    if (c.warp == X_PRODUCER) {
+        uint64_t keep;
+        asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(keep));
+        activation_producer(c, a.fb, a.P, NT, m.cfg.d_model, m.cfg.rms_eps, keep);
+        return;
     }
 
-    constexpr int RPAD = NT * 8;
     const int dm = m.cfg.d_model;
     int n_stamp = 0;
     auto stamp = [&]() {
@@ -213,16 +208,14 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
             a.fb.prof[(size_t)c.cta * PROF_STAMPS + n_stamp++] = globaltimer_ns();
     };
     stamp();
-    phase_begin(c, a, RPAD);
+    phase_begin(c, a, NT);
     stamp();
     grid_barrier(c, a.fb);
     stamp();
 
-    for (int l = 0; l < a.P.n_layers; ++l) {
-        compute_inv(c, a);
-        gemm_op<NT>(c, a.fb, a.P, OP_QKV, st,
-                    [&](int k_lo, int k_hi) { xload_normed<NT>(c, a, m.norm1 + (size_t)l * dm, k_lo, k_hi); },
-                    [&](int tile, float (&acc)[NT][4]) { epi_qkv<NT>(c, a, tile, acc); });
+    const int L = a.P.n_layers;
+    for (int l = 0; l < L; ++l) {
+        gemm_op<NT>(c, a.fb, a.P, 4 * l + OP_QKV, [&](int tile, float (&acc)[NT][4]) { epi_qkv<NT>(c, a, tile, acc); });
         stamp();
         grid_barrier(c, a.fb);
         stamp();
@@ -230,30 +223,24 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
         stamp();
         grid_barrier(c, a.fb);
         stamp();
-        gemm_op<NT>(c, a.fb, a.P, OP_O, st,
-                    [&](int k_lo, int k_hi) { xload_frag<NT>(c, d.att, k_lo, k_hi); },
-                    [&](int tile, float (&acc)[NT][4]) { epi_residual<NT>(c, a, tile, acc); });
+        gemm_op<NT>(c, a.fb, a.P, 4 * l + OP_O,
+                    [&](int tile, float (&acc)[NT][4]) { epi_residual<NT>(c, a, m.norm2 + (size_t)l * dm, tile, acc); });
         stamp();
         grid_barrier(c, a.fb);
         stamp();
-        compute_inv(c, a);
-        gemm_op<NT>(c, a.fb, a.P, OP_GU, st,
-                    [&](int k_lo, int k_hi) { xload_normed<NT>(c, a, m.norm2 + (size_t)l * dm, k_lo, k_hi); },
-                    [&](int tile, float (&acc)[NT][4]) { epi_swiglu<NT>(c, a, tile, acc); });
+        gemm_op<NT>(c, a.fb, a.P, 4 * l + OP_GU, [&](int tile, float (&acc)[NT][4]) { epi_swiglu<NT>(c, a, tile, acc); });
         stamp();
         grid_barrier(c, a.fb);
         stamp();
-        gemm_op<NT>(c, a.fb, a.P, OP_DOWN, st,
-                    [&](int k_lo, int k_hi) { xload_frag<NT>(c, d.act, k_lo, k_hi); },
-                    [&](int tile, float (&acc)[NT][4]) { epi_residual<NT>(c, a, tile, acc); });
+        const bf16 *gain_next = l + 1 < L ? m.norm1 + (size_t)(l + 1) * dm : m.normf;
+        gemm_op<NT>(c, a.fb, a.P, 4 * l + OP_DOWN,
+                    [&](int tile, float (&acc)[NT][4]) { epi_residual<NT>(c, a, gain_next, tile, acc); });
         stamp();
         grid_barrier(c, a.fb);
         stamp();
     }
-    compute_inv(c, a);                      // final RMSNorm statistics (LM head and tails)
     if (a.P.has_head) {
-        gemm_op<NT>(c, a.fb, a.P, OP_HEAD, st,
-                    [&](int k_lo, int k_hi) { xload_normed<NT>(c, a, m.normf, k_lo, k_hi); },
+        gemm_op<NT>(c, a.fb, a.P, 4 * L,
                     [&](int tile, float (&acc)[NT][4]) { epi_head<NT>(c, a, row_dst, bias_at, tile, acc); });
         stamp();
         grid_barrier(c, a.fb);
@@ -264,94 +251,44 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
             head_row_argmax(a, c.cta * g.rps + c.n_rows[c.cta] - 1, top_sm);
         }
     }
-    if (c.cta < g.batch) {
+    if (c.cta < g.batch && kind != KIND_VERIFY) {
+        // final RMSNorm statistics for the hidden rows the tails need
+        if (c.warp == 0) compute_inv(c, a.fb, dm, m.cfg.rms_eps);
+        bsync();
         if (kind == KIND_DRAFT) tail_draft(c, a, c.cta);
         else if (kind == KIND_MB) tail_mb(c, a, c.cta);
         else if (kind == KIND_AR) tail_ar(c, a, c.cta);
         else if (kind == KIND_PREFILL || kind == KIND_PREFILL_B) tail_prefill(c, a, c.cta, which);
     }
     stamp();
-    // nothing of this warp's stream may still be in flight at exit
-    while (st.cn < st.pn) { wait_unit(c, a.fb, st.cn); ++st.cn; }
 }
 
 }  // namespace fwd
 
-// ------------------------------------------------------------------ host: planning and launch
+// ------------------------------------------------------------------ host: plan and launch
 
 namespace fwd {
 
-// Cuts one projection into S k-slices x G tile groups.  The slice must fit the
-// activation buffer; among the admissible cuts the one with the smallest
-// per-block maximum of streamed bytes wins (more slices cost a little: their
-// partial sums travel through L2).
-static inline void plan_op(GemmOp &op, int ncta, int NT, int rot) {
-    const int chunks = op.K / 32, MT = op.MT;
-    const int maxchunks = std::max(1, XBUF_BYTES / (NT * 512));
-    const int s_min = (chunks + maxchunks - 1) / maxchunks;
-    double best = 1e300;
-    int bS = s_min, bKS = 0, bG = 1, bTPG = MT;
-    std::vector<long long> load(ncta);
-    for (int S0 = s_min; S0 <= std::min(chunks, s_min + 24); ++S0) {
-        const int ksc = (chunks + S0 - 1) / S0, S = (chunks + ksc - 1) / ksc;
-        if (S != S0) continue;
-        for (int mlt = 1; mlt <= 6; ++mlt) {
-            for (int dg = 0; dg < 2; ++dg) {
-                int G = (int)((long long)ncta * mlt / S) + dg;
-                G = std::max(1, std::min(G, MT));
-                const int TPG = (MT + G - 1) / G;
-                G = (MT + TPG - 1) / TPG;
-                std::fill(load.begin(), load.end(), 0LL);
-                const int items = S * G;
-                for (int i = 0; i < items; ++i) {
-                    const int s = i % S, g = i / S;
-                    const int tiles = std::min(TPG, MT - g * TPG), len = std::min(ksc, chunks - s * ksc);
-                    // bytes in units of one tile x one 32-chunk, plus the price of loading the item's activations
-                    load[(i + rot) % ncta] += (long long)((tiles + MMA_WARPS - 1) / MMA_WARPS) * MMA_WARPS * len / 2 +
-                                              (long long)tiles * len / 2 + 3 * len;
-                }
-                const long long mk = *std::max_element(load.begin(), load.end());
-                const double score = (double)mk * (1.0 + 0.01 * (S - 1));
-                if (score < best) { best = score; bS = S; bKS = ksc * 32; bG = G; bTPG = TPG; }
-            }
-        }
-    }
-    op.S = bS; op.KS = bKS; op.G = bG; op.TPG = bTPG; op.items = bS * bG; op.rot = rot;
-}
-
-static inline Plan make_plan(const ModelDev &m, int ncta, int NT, bool has_head) {
+static inline Plan make_plan(const ModelDev &m, const DevPtrs &d, const FwdBufs &fb, int ncta, bool has_head) {
     Plan P;
     memset(&P, 0, sizeof P);
     const pacer_model_cfg &k = m.cfg;
     const long long dm = k.d_model, F = k.d_ffn, hh = (long long)k.n_heads * m.hd;
-    auto set = [&](int i, const bf16 *w1, const bf16 *w2, long long lstride, int N, int K, int MT, int inter) {
-        GemmOp &o = P.op[i];
-        o.W1 = w1; o.W2 = w2 ? w2 : w1; o.lstride = lstride; o.N = N; o.K = K; o.MT = MT; o.interleave = inter;
-    };
-    set(OP_QKV, m.wqkv, nullptr, (long long)m.qrows * dm, m.qrows, (int)dm, (m.qrows + 15) / 16, 0);
-    set(OP_O, m.wo, nullptr, dm * hh, (int)dm, (int)hh, ((int)dm + 15) / 16, 0);
-    set(OP_GU, m.wgate, m.wup, F * dm, (int)(2 * F), (int)dm, ((int)F + 7) / 8, 1);
-    set(OP_DOWN, m.wdown, nullptr, dm * F, (int)dm, (int)F, ((int)dm + 15) / 16, 0);
-    set(OP_HEAD, m.head, nullptr, 0, k.vocab, (int)dm, (k.vocab + 15) / 16, 0);
     int rot = 0;
-    for (int i = 0; i < N_OPS; ++i) {
-        if (i == OP_HEAD && !has_head) { P.op[i].S = 1; P.op[i].KS = 32; P.op[i].G = 0; P.op[i].TPG = 1; P.op[i].items = 0; continue; }
-        plan_op(P.op[i], ncta, NT, rot);
-        rot = (rot + P.op[i].items) % ncta;
-    }
+    auto set = [&](int i, const bf16 *w1, const bf16 *w2, const bf16 *x, long long lstride, int N, int K, int MT, int inter) {
+        GemmOp &o = P.op[i];
+        o.W1 = w1; o.W2 = w2 ? w2 : w1; o.X = x; o.lstride = lstride; o.N = N; o.K = K; o.MT = MT; o.interleave = inter;
+        o.rot = rot;
+        rot = (rot + MT % ncta) % ncta;       // the next projection's extra tiles go to other blocks
+    };
+    set(OP_QKV, m.wqkv, nullptr, fb.xg, (long long)m.qrows * dm, m.qrows, (int)dm, (m.qrows + 15) / 16, 0);
+    set(OP_O, m.wo, nullptr, d.att, dm * hh, (int)dm, (int)hh, ((int)dm + 15) / 16, 0);
+    set(OP_GU, m.wgate, m.wup, fb.xg, F * dm, (int)(2 * F), (int)dm, ((int)F + 7) / 8, 1);
+    set(OP_DOWN, m.wdown, nullptr, d.act, dm * F, (int)dm, (int)F, ((int)dm + 15) / 16, 0);
+    set(OP_HEAD, m.head, nullptr, fb.xg, 0, k.vocab, (int)dm, (k.vocab + 15) / 16, 0);
     P.n_layers = k.n_layers;
     P.has_head = has_head ? 1 : 0;
     return P;
-}
-
-// Floats of split-k partials the plan needs.
-static inline size_t plan_part_floats(const Plan &P, int NT) {
-    size_t mx = 0;
-    for (int i = 0; i < N_OPS; ++i) {
-        if (P.op[i].items == 0 || P.op[i].S == 1) continue;
-        mx = std::max(mx, (size_t)P.op[i].S * P.op[i].MT * (size_t)NT * 8 * 16);
-    }
-    return mx;
 }
 
 template <int NT>

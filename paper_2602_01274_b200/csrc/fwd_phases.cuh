@@ -1,7 +1,6 @@
-// Phases of the forward kernel other than the weight stream itself: row set-up,
-// input rows, activation-slice loaders (with RMSNorm applied on the fly),
-// per-tile epilogues of the projections, and the tails that take the loop's
-// decisions (Eq. 6 / Eq. 7 / Algorithm 1) on the device.
+// Phases of the forward kernel other than the streams themselves: row set-up,
+// input rows, and the per-tile epilogues of the projections (which also prepare
+// the input of the projection that follows).
 #pragma once
 #include "control.cuh"
 #include "fwd_stream.cuh"
@@ -69,21 +68,27 @@ __device__ __forceinline__ RowDesc row_desc(int kind, const DevPtrs &d, int s, i
 
 // ------------------------------------------------------------------ input rows
 
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t *>(&v);
+}
+
 // x = embedding row (or h + e for the pre-verification model, or the draft's
-// hidden row during its prefill), spread over all warps of the grid by 16-column
-// tiles; also the per-tile sums of squares the first RMSNorm needs.
-__device__ __forceinline__ void phase_begin(Ctx &c, const Args &a, int rpad) {
+// hidden row during its prefill), spread over the MMA warps of the grid by
+// 16-column tiles.  Leaves x (fp32), x * gain of the first RMSNorm (bf16,
+// fragment order) and the per-tile sums of squares.
+__device__ __forceinline__ void phase_begin(Ctx &c, const Args &a, int nt_total) {
     const DevPtrs &d = a.d;
     const ModelDev &m = a.m;
-    const int dm = m.cfg.d_model, ntiles = dm >> 4;
+    const int dm = m.cfg.d_model, ntiles = dm >> 4, rpad = nt_total * 8;
     const int half = c.lane >> 4, col16 = c.lane & 15;
-    for (int tile = c.cta * WARPS + c.warp; tile < ntiles; tile += c.ncta * WARPS) {
+    for (int tile = c.cta * MMA_WARPS + c.warp; tile < ntiles; tile += c.ncta * MMA_WARPS) {
         const int col = tile * 16 + col16;
+        const float gain = __bfloat162float(m.norm1[col]);
         for (int rr = 0; rr < rpad; rr += 2) {
             const int r = rr + half;
             float v = 0.f;
-            const bool act = r < a.g.rtot && c.row_pos[r] >= 0;
-            if (act) {
+            if (r < a.g.rtot && c.row_pos[r] >= 0) {
                 const int s = r / a.g.rps, j = r - s * a.g.rps;
                 if (a.kind == KIND_MB) {
                     v = d.hpend[((size_t)s * (d.block_b + 1) + j) * dm + col];
@@ -96,75 +101,19 @@ __device__ __forceinline__ void phase_begin(Ctx &c, const Args &a, int rpad) {
                 }
                 d.xres[(size_t)r * dm + col] = v;
             }
+            a.fb.xg[xfrag_index(r, col, nt_total)] = __float2bfloat16(v * gain);
             float ss = v * v;
 #pragma unroll
             for (int o = 8; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-            if (col16 == 0 && r < MAX_ROWS) a.fb.ssq[tile * MAX_ROWS + r] = ss;
+            if (col16 == 0) a.fb.ssq[tile * MAX_ROWS + r] = ss;
         }
     }
-}
-
-// inv_rms[r] = 1 / sqrt(mean(x_r^2) + eps) from the per-tile sums, in a fixed order.
-__device__ __forceinline__ void compute_inv(Ctx &c, const Args &a) {
-    const int dm = a.m.cfg.d_model, ntiles = dm >> 4;
-    const int r = threadIdx.x >> 3, sub = threadIdx.x & 7;
-    float s = 0.f;
-    if (r < MAX_ROWS)
-        for (int t = sub; t < ntiles; t += 8) s += __ldcg(a.fb.ssq + t * MAX_ROWS + r);
-    s += __shfl_xor_sync(0xffffffffu, s, 1);
-    s += __shfl_xor_sync(0xffffffffu, s, 2);
-    s += __shfl_xor_sync(0xffffffffu, s, 4);
-    __syncthreads();                            // earlier readers of inv_rms are done
-    if (sub == 0 && r < MAX_ROWS) c.inv_rms[r] = rsqrtf(s / (float)dm + a.m.cfg.rms_eps);
-    __syncthreads();
-}
-
-// ------------------------------------------------------------------ activation slices
-
-__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
-    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-    return *reinterpret_cast<uint32_t *>(&v);
-}
-
-// Slice [k_lo, k_hi) of RMSNorm(x) * gain as bf16 in fragment order:
-// [chunk of 32 k][row tile][lane = (r % 8) * 4 + (k % 32) / 8] x 8 values.
-template <int NT>
-__device__ __forceinline__ void xload_normed(Ctx &c, const Args &a, const bf16 *gain, int k_lo, int k_hi) {
-    uint4 *xs = reinterpret_cast<uint4 *>(c.scratch);
-    const int dm = a.m.cfg.d_model;
-    const int npieces = (k_hi - k_lo) >> 3;
-    for (int i = threadIdx.x; i < NT * 8 * npieces; i += THREADS) {
-        const int r = i / npieces, p = i - r * npieces, k = k_lo + p * 8;
-        uint4 out = make_uint4(0u, 0u, 0u, 0u);
-        if (r < a.g.rtot && c.row_pos[r] >= 0) {
-            const float4 x0 = __ldcg(reinterpret_cast<const float4 *>(a.d.xres + (size_t)r * dm + k));
-            const float4 x1 = __ldcg(reinterpret_cast<const float4 *>(a.d.xres + (size_t)r * dm + k + 4));
-            const uint4 gw = *reinterpret_cast<const uint4 *>(gain + k);
-            const __nv_bfloat162 *g2 = reinterpret_cast<const __nv_bfloat162 *>(&gw);
-            const float inv = c.inv_rms[r];
-            const float2 ga = __bfloat1622float2(g2[0]), gb = __bfloat1622float2(g2[1]);
-            const float2 gc = __bfloat1622float2(g2[2]), gd = __bfloat1622float2(g2[3]);
-            out.x = pack_bf16x2(x0.x * inv * ga.x, x0.y * inv * ga.y);
-            out.y = pack_bf16x2(x0.z * inv * gb.x, x0.w * inv * gb.y);
-            out.z = pack_bf16x2(x1.x * inv * gc.x, x1.y * inv * gc.y);
-            out.w = pack_bf16x2(x1.z * inv * gd.x, x1.w * inv * gd.y);
-        }
-        xs[((p >> 2) * NT + (r >> 3)) * 32 + ((r & 7) << 2) + (p & 3)] = out;
-    }
-}
-
-// Slice of a bf16 buffer that already is in fragment order in global memory.
-template <int NT>
-__device__ __forceinline__ void xload_frag(Ctx &c, const bf16 *src, int k_lo, int k_hi) {
-    uint4 *xs = reinterpret_cast<uint4 *>(c.scratch);
-    const uint4 *s4 = reinterpret_cast<const uint4 *>(src) + (size_t)(k_lo >> 5) * (NT * 32);
-    const int n = ((k_hi - k_lo) >> 5) * (NT * 32);
-    for (int i = threadIdx.x; i < n; i += THREADS) xs[i] = __ldcg(s4 + i);
 }
 
 // ------------------------------------------------------------------ tile epilogues
+// acc element (nt, i): token row nt*8 + 2t + (i & 1), tile column g + 8*(i >> 1), with g = lane / 4, t = lane % 4.
 
-// Complete q/k/v sums of a tile -> qkv[row][column].
+// q/k/v tile: the deferred 1/rms of the input RMSNorm, then qkv[row][column].
 template <int NT>
 __device__ __forceinline__ void epi_qkv(Ctx &c, const Args &a, int tile, float (&acc)[NT][4]) {
     const int g = c.lane >> 2, t = c.lane & 3, N = a.m.qrows;
@@ -172,18 +121,32 @@ __device__ __forceinline__ void epi_qkv(Ctx &c, const Args &a, int tile, float (
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
         const int r0 = nt * 8 + 2 * t;
+        const float i0 = c.inv_rms[r0], i1 = c.inv_rms[r0 + 1];
         float *q0 = a.fb.qkv + (size_t)r0 * N, *q1 = q0 + N;
-        if (n0 < N) { q0[n0] = acc[nt][0]; q1[n0] = acc[nt][1]; }
-        if (n1 < N) { q0[n1] = acc[nt][2]; q1[n1] = acc[nt][3]; }
+        if (n0 < N) { q0[n0] = acc[nt][0] * i0; q1[n0] = acc[nt][1] * i1; }
+        if (n1 < N) { q0[n1] = acc[nt][2] * i0; q1[n1] = acc[nt][3] * i1; }
     }
 }
 
-// Residual add of a tile of the attention-output / down projection, and the
-// tile's share of sum(x^2) per row for the RMSNorm that follows.
+// Tile of the attention-output / down projection: residual add; x * gain of the
+// RMSNorm that follows, as bf16 in fragment order (the next projection's input);
+// the tile's share of sum(x^2) per row.
 template <int NT>
-__device__ __forceinline__ void epi_residual(Ctx &c, const Args &a, int tile, float (&acc)[NT][4]) {
+__device__ __forceinline__ void epi_residual(Ctx &c, const Args &a, const bf16 *gain_next, int tile, float (&acc)[NT][4]) {
     const int g = c.lane >> 2, t = c.lane & 3, dm = a.m.cfg.d_model;
     const int n0 = tile * 16 + g, n1 = n0 + 8;
+    const float g0 = n0 < dm ? __bfloat162float(gain_next[n0]) : 0.f, g1 = n1 < dm ? __bfloat162float(gain_next[n1]) : 0.f;
+    float xo[NT][4];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)                      // all loads first: one round trip
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const int r = nt * 8 + 2 * t + i;
+            const bool act = r < a.g.rtot && c.row_pos[r] >= 0;
+            const float *x = a.d.xres + (size_t)r * dm;
+            xo[nt][i] = act && n0 < dm ? __ldcg(x + n0) : 0.f;
+            xo[nt][2 + i] = act && n1 < dm ? __ldcg(x + n1) : 0.f;
+        }
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
         float ss[2] = {0.f, 0.f};
@@ -192,8 +155,16 @@ __device__ __forceinline__ void epi_residual(Ctx &c, const Args &a, int tile, fl
             const int r = nt * 8 + 2 * t + i;
             if (r < a.g.rtot && c.row_pos[r] >= 0) {
                 float *x = a.d.xres + (size_t)r * dm;
-                if (n0 < dm) { const float v = __ldcg(x + n0) + acc[nt][i]; x[n0] = v; ss[i] += v * v; }
-                if (n1 < dm) { const float v = __ldcg(x + n1) + acc[nt][2 + i]; x[n1] = v; ss[i] += v * v; }
+                if (n0 < dm) {
+                    const float v = xo[nt][i] + acc[nt][i];
+                    x[n0] = v; ss[i] += v * v;
+                    a.fb.xg[xfrag_index(r, n0, NT)] = __float2bfloat16(v * g0);
+                }
+                if (n1 < dm) {
+                    const float v = xo[nt][2 + i] + acc[nt][2 + i];
+                    x[n1] = v; ss[i] += v * v;
+                    a.fb.xg[xfrag_index(r, n1, NT)] = __float2bfloat16(v * g1);
+                }
             }
         }
 #pragma unroll
@@ -209,8 +180,8 @@ __device__ __forceinline__ void epi_residual(Ctx &c, const Args &a, int tile, fl
 }
 
 // Interleaved gate/up tile: rows 0..7 are gate rows f = 8*tile + g, rows 8..15 the
-// up rows of the same f, so a lane holds both and writes silu(gate) * up as bf16
-// in the fragment order the down projection reads.
+// up rows of the same f, so a lane holds both; 1/rms of the input RMSNorm, then
+// silu(gate) * up as bf16 in the fragment order the down projection reads.
 template <int NT>
 __device__ __forceinline__ void epi_swiglu(Ctx &c, const Args &a, int tile, float (&acc)[NT][4]) {
     const int g = c.lane >> 2, t = c.lane & 3, F = a.m.cfg.d_ffn;
@@ -221,15 +192,16 @@ __device__ __forceinline__ void epi_swiglu(Ctx &c, const Args &a, int tile, floa
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
             const int r = nt * 8 + 2 * t + i;
-            const float gt = acc[nt][i], up = acc[nt][2 + i];
-            const float v = gt / (1.f + expf(-gt)) * up;
+            const float inv = c.inv_rms[r];
+            const float gt = acc[nt][i] * inv, up = acc[nt][2 + i] * inv;
+            const float v = (r < a.g.rtot && c.row_pos[r] >= 0) ? gt / (1.f + expf(-gt)) * up : 0.f;
             a.d.act[xfrag_index(r, f, NT)] = __float2bfloat16(v);
         }
     }
 }
 
-// LM-head tile: logits (+ planted bias) to their destination rows, and the
-// tile's (max, argmax, runner-up) per row.
+// LM-head tile: 1/rms of the final RMSNorm, planted bias, logits to their
+// destination rows, and the tile's (max, argmax, runner-up) per row.
 template <int NT>
 __device__ __forceinline__ void epi_head(Ctx &c, const Args &a, float *const *row_dst, const int *bias_at, int tile,
                                          float (&acc)[NT][4]) {
@@ -244,13 +216,14 @@ __device__ __forceinline__ void epi_head(Ctx &c, const Args &a, float *const *ro
             Top2 tp{-INFINITY, 0x7fffffff, -INFINITY};
             if (dst) {
                 const int b = bias_at[r];
+                const float inv = c.inv_rms[r];
                 if (n0 < V) {
-                    const float v = acc[nt][i] + (n0 == b ? a.d.succ_bias : 0.f);
+                    const float v = acc[nt][i] * inv + (n0 == b ? a.d.succ_bias : 0.f);
                     dst[n0] = v;
                     tp.v1 = v; tp.i1 = n0;
                 }
                 if (n1 < V) {
-                    const float v = acc[nt][2 + i] + (n1 == b ? a.d.succ_bias : 0.f);
+                    const float v = acc[nt][2 + i] * inv + (n1 == b ? a.d.succ_bias : 0.f);
                     dst[n1] = v;
                     tp = top2_merge(tp, Top2{v, n1, -INFINITY});
                 }
@@ -270,19 +243,50 @@ __device__ __forceinline__ void epi_head(Ctx &c, const Args &a, float *const *ro
     }
 }
 
+// Top-2 over the eight MMA warps; every thread gets the result.  sm: 8 entries.
+__device__ __forceinline__ Top2 mma_block_top2(Top2 t, Top2 *sm) {
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        Top2 u;
+        u.v1 = __shfl_xor_sync(0xffffffffu, t.v1, o);
+        u.i1 = __shfl_xor_sync(0xffffffffu, t.i1, o);
+        u.v2 = __shfl_xor_sync(0xffffffffu, t.v2, o);
+        t = top2_merge(t, u);
+    }
+    bsync();
+    if (lane == 0) sm[w] = t;
+    bsync();
+    Top2 r = sm[0];
+#pragma unroll
+    for (int i = 1; i < MMA_WARPS; ++i) r = top2_merge(r, sm[i]);
+    return r;
+}
+
+// Sum over the eight MMA warps; every thread gets the result.  red: 8 floats.
+__device__ __forceinline__ float mma_block_sum(float v, float *red) {
+    v = warp_sum(v);
+    bsync();
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+    bsync();
+    float s = 0.f;
+#pragma unroll
+    for (int i = 0; i < MMA_WARPS; ++i) s += red[i];
+    return s;
+}
+
 // Arg-max (lowest index on ties) and gap to the runner-up of LM-head row r from
-// the per-tile results; the whole block works on one row.
+// the per-tile results; the MMA warps of the block work on one row.
 __device__ __forceinline__ void head_row_argmax(const Args &a, int r, Top2 *sm) {
     const int MT = a.P.op[OP_HEAD].MT;
     Top2 t{-INFINITY, 0x7fffffff, -INFINITY};
-    for (int tile = threadIdx.x; tile < MT; tile += THREADS) {
+    for (int tile = threadIdx.x; tile < MT; tile += MMA_THREADS) {
         const float4 v = __ldcg(reinterpret_cast<const float4 *>(a.fb.tile_top) + (size_t)tile * MAX_ROWS + r);
         t = top2_merge(t, Top2{v.x, __float_as_int(v.y), v.z});
     }
-    __syncthreads();
-    t = block_top2(t, sm);
+    t = mma_block_top2(t, sm);
     if (threadIdx.x == 0) { a.d.row_arg[r] = t.i1; a.d.row_margin[r] = t.v1 - t.v2; }
-    __syncthreads();
+    bsync();
 }
 
 }  // namespace fwd

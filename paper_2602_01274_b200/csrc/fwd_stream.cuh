@@ -1,122 +1,142 @@
-// Weight stream of the forward kernel: the static list of weight units of one
-// warp, the bulk-copy producer that walks it, and the projection loop that
-// consumes it with tensor cores.
+// Weight and activation streams of the forward kernel: the two producer warps
+// and the projection loop of the MMA warps.
+//
+// Order of everything, identical on both sides: projections q = 0, 1, ... of the
+// forward (four per layer, then the LM head); inside a projection the passes of
+// this block (at most MAX_TILES tiles each); inside a pass the k steps of KC
+// columns; inside a k step the tiles of the pass.  Weight unit number n of the
+// block lives in ring stage n % NS, activation chunk number m in stage m % XS.
 #pragma once
 #include "forward.cuh"
 
 namespace fwd {
 
-// Position in the static unit list of (block, warp): projection q (layer-major:
-// 4 per layer, then the LM head), item ordinal m of this block, tile ordinal j of
-// this warp, unit ordinal u inside the k slice.
-struct Cursor {
-    int q, m, j, u;
-    int done;
-    // derived by settle()
-    int opi, layer, tile, k, kc;
-};
-
-__device__ __forceinline__ int first_item(const GemmOp &op, int cta, int ncta) {
-    int f = cta - op.rot;
-    return f < 0 ? f + ncta : f;
-}
-
-// Moves the cursor to the next existing unit at or after its position.
-__device__ __forceinline__ bool settle(Cursor &cu, const Plan &P, int cta, int ncta, int warp) {
-    const int nq = 4 * P.n_layers + (P.has_head ? 1 : 0);
-    while (true) {
-        if (cu.q >= nq) { cu.done = 1; return false; }
-        const int opi = cu.q < 4 * P.n_layers ? (cu.q & 3) : OP_HEAD;
-        const GemmOp &op = P.op[opi];
-        const int idx = first_item(op, cta, ncta) + cu.m * ncta;
-        if (idx >= op.items) { ++cu.q; cu.m = cu.j = cu.u = 0; continue; }
-        const int s = idx % op.S, g = idx / op.S;
-        const int t_lo = g * op.TPG, t_hi = min(op.MT, t_lo + op.TPG);
-        const int tile = t_lo + warp + MMA_WARPS * cu.j;
-        if (tile >= t_hi) { ++cu.m; cu.j = cu.u = 0; continue; }
-        const int k_lo = s * op.KS, k_hi = min(op.K, k_lo + op.KS);
-        const int k = k_lo + cu.u * KC;
-        if (k >= k_hi) { ++cu.j; cu.u = 0; continue; }
-        cu.opi = opi;
-        cu.layer = cu.q < 4 * P.n_layers ? (cu.q >> 2) : 0;
-        cu.tile = tile;
-        cu.k = k;
-        cu.kc = min(KC, k_hi - k);
-        return true;
-    }
-}
-
-struct Stream {
-    Cursor cu;
-    int pn, cn;            // units issued / consumed by this warp
-};
-
-// Issues the bulk copies of the cursor's unit into the next stage and advances the cursor.
-__device__ __forceinline__ void issue_unit(Ctx &c, Stream &st, const Plan &P) {
-    if (st.cu.done) return;
-    const int slot = st.pn % STAGES;
-    unsigned char *stage = c.ring + slot * STAGE_BYTES;
-    uint64_t *bar = c.mbar + slot;
-    const GemmOp &op = P.op[st.cu.opi];
-    const uint32_t bytes = (uint32_t)st.cu.kc * 2u;
-    if (c.lane == 0) mbar_expect_tx(bar, 16u * bytes);
-    __syncwarp();
-    if (c.lane < 16) {
-        const bf16 *src;
-        if (op.interleave) {
-            const int F = op.N >> 1;
-            const int f = min(st.cu.tile * 8 + (c.lane & 7), F - 1);
-            src = (c.lane < 8 ? op.W1 : op.W2) + (size_t)st.cu.layer * op.lstride + (size_t)f * op.K + st.cu.k;
-        } else {
-            const int n = min(st.cu.tile * 16 + c.lane, op.N - 1);
-            src = op.W1 + (size_t)st.cu.layer * op.lstride + (size_t)n * op.K + st.cu.k;
-        }
-        bulk_g2s(stage + c.lane * PITCH, src, bytes, bar, c.policy);
-    }
-    ++st.pn;
-    ++st.cu.u;
-    settle(st.cu, P, c.cta, c.ncta, c.warp);
-}
-
 // Bounded wait on a shared-memory barrier phase.
-__device__ __forceinline__ void wait_bar(Ctx &c, const FwdBufs &fb, uint64_t *bar, uint32_t parity, int code) {
+__device__ __forceinline__ void wait_bar(const FwdBufs &fb, uint64_t *bar, uint32_t parity, int code) {
     unsigned it = 0;
     while (!mbar_try_wait(bar, parity)) {
-        if (++it > SPIN_LIMIT) {
-            if (c.lane == 0) atomicExch(fb.abort_flag, code);
+        ++it;
+        if ((it & 1023u) == 0 && (it > SPIN_LIMIT || *(volatile int32_t *)fb.abort_flag)) {
+            atomicCAS(fb.abort_flag, 0, code);
             break;
         }
     }
 }
 
-// Bounded wait for the stage that holds unit number n of this warp.
-__device__ __forceinline__ void wait_unit(Ctx &c, const FwdBufs &fb, int n) {
-    wait_bar(c, fb, c.mbar + (n % STAGES), (uint32_t)(n / STAGES) & 1u, 2);
+// Bounded wait until a shared-memory counter written by another warp reaches `want`.
+__device__ __forceinline__ void wait_count(const FwdBufs &fb, volatile int32_t *p, int want, int code) {
+    unsigned it = 0;
+    while (*p < want) {
+        ++it;
+        if ((it & 1023u) == 0 && (it > SPIN_LIMIT * 4u || *(volatile int32_t *)fb.abort_flag)) {
+            atomicCAS(fb.abort_flag, 0, code);
+            break;
+        }
+    }
 }
 
-// Streaming warp -> its epilogue partner: the accumulators of a finished tile,
-// through shared memory in lane order (conflict free), one tile at a time.
-template <int NT>
-__device__ __forceinline__ void hand_over(Ctx &c, const FwdBufs &fb, const float (&acc)[NT][4]) {
-    wait_bar(c, fb, c.hand_empty, ((uint32_t)c.n_hand & 1u) ^ 1u, 3);      // the partner took the previous tile
-#pragma unroll
-    for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-        for (int i = 0; i < 4; ++i) c.hand[(nt * 4 + i) * 32 + c.lane] = acc[nt][i];
-    __syncwarp();
-    if (c.lane == 0) mbar_arrive(c.hand_full);
-    ++c.n_hand;
+__device__ __forceinline__ int n_ops(const Plan &P) { return 4 * P.n_layers + (P.has_head ? 1 : 0); }
+__device__ __forceinline__ int op_index(const Plan &P, int q) { return q < 4 * P.n_layers ? (q & 3) : OP_HEAD; }
+__device__ __forceinline__ int op_layer(const Plan &P, int q) { return q < 4 * P.n_layers ? (q >> 2) : 0; }
+
+// Warp W_PRODUCER: every weight unit of the block, for the whole forward, in order.
+__device__ __forceinline__ void weight_producer(Ctx &c, const FwdBufs &fb, const Plan &P) {
+    int n = 0;
+    for (int q = 0; q < n_ops(P); ++q) {
+        const GemmOp &op = P.op[op_index(P, q)];
+        const size_t lbase = (size_t)op_layer(P, q) * op.lstride;
+        int t0, T;
+        tile_range(op.MT, op.rot, c.cta, c.ncta, t0, T);
+        for (int p0 = 0; p0 < T; p0 += MAX_TILES) {
+            const int Tp = min(MAX_TILES, T - p0);
+            for (int k = 0; k < op.K; k += KC) {
+                const uint32_t bytes = (uint32_t)min(KC, op.K - k) * 2u;
+                for (int i = 0; i < Tp; ++i, ++n) {
+                    const int slot = n % NS, tile = t0 + p0 + i;
+                    wait_bar(fb, c.wempty + slot, (((uint32_t)(n / NS)) & 1u) ^ 1u, 5);
+                    if (*(volatile int32_t *)fb.abort_flag) return;      // a wait ran out somewhere: stop feeding
+                    if (c.lane == 0) mbar_expect_tx(c.wfull + slot, 16u * bytes);
+                    __syncwarp();
+                    if (c.lane < 16) {
+                        const bf16 *src;
+                        if (op.interleave) {
+                            const int f = min(tile * 8 + (c.lane & 7), (op.N >> 1) - 1);
+                            src = (c.lane < 8 ? op.W1 : op.W2) + lbase + (size_t)f * op.K + k;
+                        } else {
+                            const int nrow = min(tile * 16 + c.lane, op.N - 1);
+                            src = op.W1 + lbase + (size_t)nrow * op.K + k;
+                        }
+                        bulk_g2s(c.ring + slot * STAGE_BYTES + c.lane * PITCH, src, bytes, c.wfull + slot, c.policy);
+                    }
+                }
+            }
+        }
+    }
 }
-template <int NT>
-__device__ __forceinline__ void receive(Ctx &c, const FwdBufs &fb, float (&acc)[NT][4]) {
-    wait_bar(c, fb, c.hand_full, (uint32_t)c.n_hand & 1u, 4);
-#pragma unroll
-    for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-        for (int i = 0; i < 4; ++i) acc[nt][i] = c.hand[(nt * 4 + i) * 32 + c.lane];
+
+// inv_rms[r] = 1 / sqrt(mean(x_r^2) + eps) from the per-tile sums ssq[tile][row], in a fixed
+// order (one warp, lane = row; four running sums keep the loads independent).
+__device__ __forceinline__ void compute_inv(Ctx &c, const FwdBufs &fb, int dm, float eps) {
+    const int ntiles = dm >> 4;
+    const float *p = fb.ssq + c.lane;
+    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+    int t = 0;
+    for (; t + 4 <= ntiles; t += 4) {
+        s0 += __ldcg(p + (t + 0) * MAX_ROWS);
+        s1 += __ldcg(p + (t + 1) * MAX_ROWS);
+        s2 += __ldcg(p + (t + 2) * MAX_ROWS);
+        s3 += __ldcg(p + (t + 3) * MAX_ROWS);
+    }
+    for (; t < ntiles; ++t) s0 += __ldcg(p + t * MAX_ROWS);
+    c.inv_rms[c.lane] = rsqrtf(((s0 + s1) + (s2 + s3)) / (float)dm + eps);
     __syncwarp();
-    if (c.lane == 0) mbar_arrive(c.hand_empty);
-    ++c.n_hand;
+}
+
+// Warp X_PRODUCER: the activation chunk of every k step once the projection's
+// inputs are complete (the MMA warps raise ready_op[0] after the grid barrier),
+// and the RMS statistics the projection's epilogue applies.
+__device__ __forceinline__ void activation_producer(Ctx &c, const FwdBufs &fb, const Plan &P, int NT, int dm, float eps,
+                                                    uint64_t keep_policy) {
+    int m = 0;
+    for (int q = 0; q < n_ops(P); ++q) {
+        const int opi = op_index(P, q);
+        const GemmOp &op = P.op[opi];
+        const bool normed = opi == OP_QKV || opi == OP_GU || opi == OP_HEAD;
+        int t0, T;
+        tile_range(op.MT, op.rot, c.cta, c.ncta, t0, T);
+        wait_count(fb, c.ready_op, q + 1, 6);
+        __threadfence_block();
+        asm volatile("fence.proxy.async;" ::: "memory");
+        bool inv_done = !normed;
+        int issued = 0;
+        for (int p0 = 0; p0 < T; p0 += MAX_TILES) {
+            for (int k = 0; k < op.K; k += KC, ++m, ++issued) {
+                if (!inv_done && issued == XS) {          // the ring is full: a good moment for the statistics
+                    compute_inv(c, fb, dm, eps);
+                    __threadfence_block();
+                    if (c.lane == 0) c.ready_op[1] = q + 1;
+                    inv_done = true;
+                }
+                const int slot = m % XS;
+                wait_bar(fb, c.xempty + slot, (((uint32_t)(m / XS)) & 1u) ^ 1u, 7);
+                if (c.lane == 0) {
+                    const uint32_t bytes = (uint32_t)(min(KC, op.K - k) >> 5) * (uint32_t)NT * 512u;
+                    mbar_expect_tx(c.xfull + slot, bytes);
+                    bulk_g2s(c.scratch + slot * XSTAGE_BYTES, op.X + (size_t)(k >> 5) * NT * 256, bytes, c.xfull + slot,
+                             keep_policy);
+                }
+                __syncwarp();
+            }
+        }
+        if (!inv_done) {
+            compute_inv(c, fb, dm, eps);
+            __threadfence_block();
+            if (c.lane == 0) c.ready_op[1] = q + 1;
+        } else if (!normed && c.lane == 0) {
+            c.ready_op[1] = q + 1;
+        }
+        __syncwarp();
+    }
 }
 
 // acc[nt] += W(16 rows x 32*nchunks k) * X over one stage.  Lane (g, t) reads the
@@ -124,15 +144,15 @@ __device__ __forceinline__ void receive(Ctx &c, const FwdBufs &fb, float (&acc)[
 // slots {2t, 2t+1, 2t+8, 2t+9} of two MMAs; the activation fragments are stored
 // with the same rule, so the products pair up.
 template <int NT>
-__device__ __forceinline__ void consume_unit(const unsigned char *stage, const uint4 *xs, int chunk0, int nchunks,
-                                             float (&acc)[NT][4], int lane) {
+__device__ __forceinline__ void consume_unit(const unsigned char *stage, const uint4 *xs, int nchunks, float (&acc)[NT][4],
+                                             int lane) {
     const int g = lane >> 2, t = lane & 3;
     const unsigned char *p0 = stage + g * PITCH + t * 16, *p1 = p0 + 8 * PITCH;
 #pragma unroll 2
     for (int cix = 0; cix < nchunks; ++cix) {
         const uint4 a0 = *reinterpret_cast<const uint4 *>(p0 + cix * 64);
         const uint4 a1 = *reinterpret_cast<const uint4 *>(p1 + cix * 64);
-        const uint4 *xb = xs + (size_t)(chunk0 + cix) * (NT * 32) + lane;
+        const uint4 *xb = xs + cix * (NT * 32) + lane;
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
             const uint4 b = xb[nt * 32];
@@ -142,100 +162,57 @@ __device__ __forceinline__ void consume_unit(const unsigned char *stage, const u
     }
 }
 
-// Split-k reduction of one 16-column tile.  The warp stores its slice's partial,
-// counts itself in, and the warp that arrives last adds the slices up in slice
-// order.  Returns true for that warp, with the complete sums in acc.
+// One projection, run by the eight MMA warps after the grid barrier that
+// completed its inputs.  Warp w owns tiles w and w + 8 of every pass, over the
+// full k extent; epi(tile, acc) gets the complete sums.
 // Accumulator element (nt, i): token row nt*8 + 2t + (i & 1), tile column g + 8*(i >> 1).
-template <int NT>
-__device__ __forceinline__ bool tile_reduce(Ctx &c, const FwdBufs &fb, const GemmOp &op, int tile, int s,
-                                            float (&acc)[NT][4]) {
-    if (op.S == 1) return true;
-    constexpr int RPAD = NT * 8;
-    const int g = c.lane >> 2, t = c.lane & 3;
-    float *mine = fb.part + ((size_t)s * op.MT + tile) * (RPAD * 16);
-#pragma unroll
-    for (int nt = 0; nt < NT; ++nt) {
-        const int r0 = nt * 8 + 2 * t;
-        mine[r0 * 16 + g] = acc[nt][0];
-        mine[(r0 + 1) * 16 + g] = acc[nt][1];
-        mine[r0 * 16 + g + 8] = acc[nt][2];
-        mine[(r0 + 1) * 16 + g + 8] = acc[nt][3];
+template <int NT, class Epi>
+__device__ __forceinline__ void gemm_op(Ctx &c, const FwdBufs &fb, const Plan &P, int q, Epi epi) {
+    const GemmOp &op = P.op[op_index(P, q)];
+    if (threadIdx.x == 0) {
+        __threadfence_block();
+        c.ready_op[0] = q + 1;                 // the activation producer may start on this projection
     }
-    __threadfence();
-    __syncwarp();
-    int old = 0;
-    if (c.lane == 0) old = atomicAdd(fb.tile_cnt + tile, 1);
-    old = __shfl_sync(0xffffffffu, old, 0);
-    if (old != op.S - 1) return false;
-    if (c.lane == 0) fb.tile_cnt[tile] = 0;        // the next projection starts from zero (a grid barrier lies between)
-    __threadfence();
-    float sum[NT][4];
+    int t0, T;
+    tile_range(op.MT, op.rot, c.cta, c.ncta, t0, T);
+    for (int p0 = 0; p0 < T; p0 += MAX_TILES) {
+        const int Tp = min(MAX_TILES, T - p0);
+        const bool has0 = c.warp < Tp, has1 = c.warp + MMA_WARPS < Tp;
+        float acc0[NT][4], acc1[NT][4];
 #pragma unroll
-    for (int nt = 0; nt < NT; ++nt) sum[nt][0] = sum[nt][1] = sum[nt][2] = sum[nt][3] = 0.f;
-    for (int ss = 0; ss < op.S; ++ss) {
-        if (ss == s) {
+        for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-            for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-                for (int i = 0; i < 4; ++i) sum[nt][i] += acc[nt][i];
-        } else {
-            const float *p = fb.part + ((size_t)ss * op.MT + tile) * (RPAD * 16);
-#pragma unroll
-            for (int nt = 0; nt < NT; ++nt) {
-                const int r0 = nt * 8 + 2 * t;
-                sum[nt][0] += __ldcg(p + r0 * 16 + g);
-                sum[nt][1] += __ldcg(p + (r0 + 1) * 16 + g);
-                sum[nt][2] += __ldcg(p + r0 * 16 + g + 8);
-                sum[nt][3] += __ldcg(p + (r0 + 1) * 16 + g + 8);
+            for (int i = 0; i < 4; ++i) acc0[nt][i] = acc1[nt][i] = 0.f;
+        for (int k = 0; k < op.K; k += KC) {
+            const int nch = min(KC, op.K - k) >> 5;
+            const int xslot = c.xn % XS;
+            wait_bar(fb, c.xfull + xslot, ((uint32_t)(c.xn / XS)) & 1u, 8);
+            const uint4 *xs = reinterpret_cast<const uint4 *>(c.scratch + xslot * XSTAGE_BYTES);
+            if (has0) {
+                const int n = c.wn + c.warp, slot = n % NS;
+                wait_bar(fb, c.wfull + slot, ((uint32_t)(n / NS)) & 1u, 9);
+                consume_unit<NT>(c.ring + slot * STAGE_BYTES, xs, nch, acc0, c.lane);
+                __syncwarp();
+                if (c.lane == 0) mbar_arrive(c.wempty + slot);
             }
-        }
-    }
-#pragma unroll
-    for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-        for (int i = 0; i < 4; ++i) acc[nt][i] = sum[nt][i];
-    return true;
-}
-
-// One projection: for every item of this block load the activation slice, then
-// every streaming warp runs its tiles through its pipeline and hands each
-// finished tile to its partner.  xload(k_lo, k_hi) fills the scratch with the
-// slice in fragment order (all threads call it); epi(tile, acc) runs in the
-// epilogue warp that completed the tile (last k slice to arrive).
-template <int NT, class XLoad, class Epi>
-__device__ __forceinline__ void gemm_op(Ctx &c, const FwdBufs &fb, const Plan &P, int opi, Stream &st, XLoad xload,
-                                        Epi epi) {
-    const GemmOp &op = P.op[opi];
-    const uint4 *xs = reinterpret_cast<const uint4 *>(c.scratch);
-    const bool streamer = c.warp < MMA_WARPS;
-    const int w = c.warp & (MMA_WARPS - 1);
-    for (int idx = first_item(op, c.cta, c.ncta); idx < op.items; idx += c.ncta) {
-        const int s = idx % op.S, g = idx / op.S;
-        const int k_lo = s * op.KS, k_hi = min(op.K, k_lo + op.KS);
-        const int t_lo = g * op.TPG, t_hi = min(op.MT, t_lo + op.TPG);
-        __syncthreads();                       // the scratch is free
-        xload(k_lo, k_hi);
-        __syncthreads();
-        for (int tile = t_lo + w; tile < t_hi; tile += MMA_WARPS) {
-            float acc[NT][4];
-            if (streamer) {
-#pragma unroll
-                for (int nt = 0; nt < NT; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
-                for (int k = k_lo; k < k_hi; k += KC) {
-                    const int kc = min(KC, k_hi - k);
-                    wait_unit(c, fb, st.cn);
-                    consume_unit<NT>(c.ring + (st.cn % STAGES) * STAGE_BYTES, xs, (k - k_lo) >> 5, kc >> 5, acc, c.lane);
-                    ++st.cn;
-                    __syncwarp();
-                    fence_proxy_async();
-                    issue_unit(c, st, P);      // refill the freed stage with the next unit of the static list
-                }
-                hand_over<NT>(c, fb, acc);
-            } else {
-                receive<NT>(c, fb, acc);
-                if (tile_reduce<NT>(c, fb, op, tile, s, acc)) epi(tile, acc);
+            if (has1) {
+                const int n = c.wn + c.warp + MMA_WARPS, slot = n % NS;
+                wait_bar(fb, c.wfull + slot, ((uint32_t)(n / NS)) & 1u, 9);
+                consume_unit<NT>(c.ring + slot * STAGE_BYTES, xs, nch, acc1, c.lane);
+                __syncwarp();
+                if (c.lane == 0) mbar_arrive(c.wempty + slot);
             }
+            __syncwarp();
+            if (c.lane == 0) mbar_arrive(c.xempty + xslot);
+            c.wn += Tp;
+            ++c.xn;
         }
+        if (has0 || has1) {
+            wait_count(fb, c.ready_op + 1, q + 1, 10);                 // RMS statistics of this projection's input
+            __threadfence_block();
+        }
+        if (has0) epi(t0 + p0 + c.warp, acc0);
+        if (has1) epi(t0 + p0 + c.warp + MMA_WARPS, acc1);
     }
 }
 

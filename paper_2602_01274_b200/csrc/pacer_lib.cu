@@ -26,8 +26,7 @@ struct pacer_ctx {
     Geom g_draft, g_mb, g_verify, g_ar;
     fwd::FwdBufs fb;
     int ncta;                  // blocks of the forward kernel (one per SM)
-    std::map<int, fwd::Plan> plans;   // key: which * 16 + nt * 2 + has_head
-    size_t part_floats;        // capacity of the split-k partial buffer
+    std::map<int, fwd::Plan> plans;   // key: which * 2 + has_head
     unsigned long long *prof_stamps;
     int batch;                 // sequences of the current run
     int prefilled;
@@ -116,7 +115,7 @@ struct Carver {
 struct Layout {
     size_t st, x, y, alpha, hpend, hpend_e, draft_len, accept_len, verify_logits, draft_logits;
     size_t row_pos, row_tok, n_rows, row_arg, row_margin, xres, att, act, hidden, part;
-    size_t tile_cnt, att_cnt, bar, abort_flag, qkv, ssq, tile_top, attp, prof;
+    size_t att_cnt, bar, abort_flag, qkv, xg, ssq, tile_top, attp, prof;
     size_t kc[3], vc[3], rope[3];
     size_t kv_bytes[3], rope_bytes[3];
     size_t total;
@@ -131,27 +130,6 @@ static int sm_count_or_default() {
         return n;
     cudaGetLastError();
     return 148;
-}
-
-// Split-k partial floats the forward kernel can need for this configuration (any row-tile count, any model).
-static size_t part_floats_needed(const pacer_cfg &c, int ncta) {
-    const pacer_model_cfg mb = mb_cfg(c);
-    const pacer_model_cfg *ms[3] = {&c.target, &c.draft, &mb};
-    const int rps_max = std::max(c.gamma_cap + 1, c.block_b + 1);
-    const int nt_max = std::min(4, (c.max_batch * rps_max + 7) / 8);
-    size_t mx = 0;
-    for (int i = 0; i < 3; ++i) {
-        ModelDev m;
-        memset(&m, 0, sizeof m);
-        m.cfg = *ms[i];
-        m.hd = m.cfg.d_model / m.cfg.n_heads;
-        m.qrows = (m.cfg.n_heads + 2 * m.cfg.n_kv_heads) * m.hd;
-        for (int nt = 1; nt <= nt_max; ++nt) {
-            fwd::Plan P = fwd::make_plan(m, ncta, nt, i != 2);
-            mx = std::max(mx, fwd::plan_part_floats(P, nt));
-        }
-    }
-    return mx;
 }
 
 static Layout make_layout(const pacer_cfg &c) {
@@ -185,7 +163,6 @@ static Layout make_layout(const pacer_cfg &c) {
     L.n_rows = cv.take(sizeof(int32_t) * fwd::MAX_ROWS);
     L.row_arg = cv.take(sizeof(int32_t) * fwd::MAX_ROWS);
     L.row_margin = cv.take(sizeof(float) * fwd::MAX_ROWS);
-    L.tile_cnt = cv.take(sizeof(int32_t) * ((size_t)std::max(V, 2 * f_max) / 8 + 16));
     L.att_cnt = cv.take(sizeof(int32_t) * (size_t)B * h_max);
     L.bar = cv.take(sizeof(unsigned long long));
     L.abort_flag = cv.take(sizeof(int32_t));
@@ -199,13 +176,11 @@ static Layout make_layout(const pacer_cfg &c) {
     L.att = cv.take(sizeof(bf16) * fwd::MAX_ROWS * d_max);
     L.act = cv.take(sizeof(bf16) * fwd::MAX_ROWS * f_max);
     L.qkv = cv.take(sizeof(float) * fwd::MAX_ROWS * qrows_max);
+    L.xg = cv.take(sizeof(bf16) * fwd::MAX_ROWS * d_max);
     L.ssq = cv.take(sizeof(float) * fwd::MAX_ROWS * (d_max / 16 + 1));
     L.tile_top = cv.take(sizeof(float) * 4 * fwd::MAX_ROWS * ((size_t)V / 16 + 1));
     L.attp = cv.take(sizeof(float) * (size_t)B * h_max * fwd::MAX_SPLIT * rps_max * (hd_max + 2));
-    // planned for 148 blocks and for the device's own count when one is present; twice the need, so that a
-    // device with another SM count still fits
-    size_t pf = std::max(part_floats_needed(c, 148), part_floats_needed(c, sm_count_or_default()));
-    L.part_bytes = 2 * pf * sizeof(float) + 256;
+    L.part_bytes = 256;
     L.part = cv.take(L.part_bytes);
     for (int i = 0; i < 3; ++i) {
         const int hd = ms[i]->d_model / ms[i]->n_heads;
@@ -267,13 +242,12 @@ extern "C" int pacer_create(const pacer_cfg *cfg, void *dev_workspace, size_t wo
     d.row_arg = (int32_t *)(w + L.row_arg); d.row_margin = (float *)(w + L.row_margin);
     d.xres = (float *)(w + L.xres); d.xn = nullptr; d.att = (bf16 *)(w + L.att); d.act = (bf16 *)(w + L.act);
     d.q = nullptr; d.hidden = (float *)(w + L.hidden); d.part = (float *)(w + L.part);
-    c->fb.qkv = (float *)(w + L.qkv); c->fb.part = (float *)(w + L.part); c->fb.tile_cnt = (int32_t *)(w + L.tile_cnt);
+    c->fb.qkv = (float *)(w + L.qkv); c->fb.xg = (bf16 *)(w + L.xg);
     c->fb.ssq = (float *)(w + L.ssq); c->fb.tile_top = (float *)(w + L.tile_top); c->fb.attp = (float *)(w + L.attp);
     c->fb.att_cnt = (int32_t *)(w + L.att_cnt); c->fb.bar = (unsigned long long *)(w + L.bar);
     c->fb.abort_flag = (int32_t *)(w + L.abort_flag);
     c->fb.prof = nullptr;
     c->prof_stamps = (unsigned long long *)(w + L.prof);
-    c->part_floats = L.part_bytes / sizeof(float);
     c->ncta = sm_count_or_default();
     d.max_batch = cfg->max_batch; d.max_ctx = cfg->max_ctx; d.gamma_cap = cfg->gamma_cap; d.block_b = cfg->block_b;
     d.max_steps = L.max_steps; d.rho = cfg->rho; d.succ_bias = cfg->succ_bias; d.criterion = cfg->criterion;
@@ -397,14 +371,9 @@ static double model_weight_bytes(const ModelDev &m, bool head) {
 static int run_forward(pacer_ctx *c, int which, const Geom &g, int kind, int aux, bool head) {
     ModelDev &m = c->model[which];
     if (g.rtot > fwd::MAX_ROWS || g.nt > 4) return fail(c, PACER_EUNSUPPORTED, "more than 32 rows in one forward");
-    const int key = which * 16 + g.nt * 2 + (head ? 1 : 0);
+    const int key = which * 2 + (head ? 1 : 0);
     auto it = c->plans.find(key);
-    if (it == c->plans.end()) {
-        fwd::Plan P = fwd::make_plan(m, c->ncta, g.nt, head);
-        if (fwd::plan_part_floats(P, g.nt) > c->part_floats)
-            return fail(c, PACER_ENOMEM, "split-k partial buffer too small for this device's SM count");
-        it = c->plans.emplace(key, P).first;
-    }
+    if (it == c->plans.end()) it = c->plans.emplace(key, fwd::make_plan(m, c->d, c->fb, c->ncta, head)).first;
     fwd::Args a;
     a.d = c->d; a.m = m; a.g = g; a.P = it->second; a.fb = c->fb; a.kind = kind; a.aux = aux;
     a.fb.prof = (c->prof_on && which == PACER_TARGET && c->ncta <= fwd::PROF_BLOCKS) ? c->prof_stamps : nullptr;
@@ -454,7 +423,7 @@ static int start_run(pacer_ctx *c, const int32_t *prompt, int batch, int n_promp
     }
     CK(cudaMemcpyAsync(c->d.st, hs.data(), sizeof(SeqState) * hs.size(), cudaMemcpyHostToDevice, c->stream));
     // arrival counters, grid barrier and abort flag start from zero (they are contiguous in the workspace)
-    CK(cudaMemsetAsync(c->fb.tile_cnt, 0, (char *)c->fb.abort_flag + sizeof(int32_t) - (char *)c->fb.tile_cnt, c->stream));
+    CK(cudaMemsetAsync(c->fb.att_cnt, 0, (char *)c->fb.abort_flag + sizeof(int32_t) - (char *)c->fb.att_cnt, c->stream));
     CK(cudaMemcpy2DAsync(c->d.x, sizeof(int32_t) * k.max_ctx, prompt, sizeof(int32_t) * n_prompt, sizeof(int32_t) * n_prompt,
                          batch, cudaMemcpyHostToDevice, c->stream));
     CK(cudaStreamSynchronize(c->stream));        // hs is a local
