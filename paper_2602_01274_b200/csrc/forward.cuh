@@ -27,8 +27,10 @@
 namespace fwd {
 
 constexpr int MMA_WARPS = 8, MMA_THREADS = 256;  // warps 0..7: MMAs, epilogues and all block-wide phases
-constexpr int W_PRODUCER = 8, X_PRODUCER = 9;    // warp 8 streams weights, warp 9 activations (and RMS statistics)
-constexpr int THREADS = 320;
+constexpr int W_PRODUCERS = 4;                   // warps 8..11 stream weights (unit n by producer n % 4: one warp alone
+                                                 // cannot issue bulk copies fast enough), warp 12 activations + RMS statistics
+constexpr int W_PRODUCER = 8, X_PRODUCER = W_PRODUCER + W_PRODUCERS;
+constexpr int THREADS = 32 * (X_PRODUCER + 1);
 constexpr int KC = 256;                         // k columns of one weight unit
 constexpr int PITCH = KC * 2 + 64;              // bytes between the rows of a stage (bank-conflict free)
 constexpr int STAGE_BYTES = 16 * PITCH;         // 9216
@@ -43,7 +45,8 @@ constexpr int SMEM_BYTES = SCRATCH_BYTES + RING_BYTES + MISC_BYTES;
 constexpr int MAX_TILES = 16;                   // tiles of one pass of a block (two per MMA warp)
 constexpr int MAX_ROWS = 32;                    // rows of one forward (all sequences together)
 constexpr int MAX_SPLIT = 16;                   // key-range splits of one attention head
-constexpr unsigned SPIN_LIMIT = 1u << 22;
+constexpr unsigned SPIN_LIMIT = 1u << 22;        // polls of a global word or a shared counter
+constexpr unsigned MBAR_SPIN_LIMIT = 1u << 18;   // polls of an mbarrier (each may suspend for microseconds)
 constexpr int PROF_STAMPS = 512;              // phase-boundary time stamps kept per block and forward
 constexpr int PROF_BLOCKS = 256;              // blocks the stamp buffer has room for
 
@@ -76,7 +79,7 @@ struct FwdBufs {
     float *attp;             // attention partials [seq*H + h][split][row][hd + 2]
     int32_t *att_cnt;        // [batch * H]
     unsigned long long *bar; // grid barrier counter
-    int32_t *abort_flag;     // set when a bounded wait ran out
+    int32_t *abort_flag;     // [0] code of the first bounded wait that ran out, [1..3] its block, warp, detail
     unsigned long long *prof; // optional: every block stamps %globaltimer at its phase boundaries (NULL = off)
 };
 
@@ -177,7 +180,7 @@ __device__ __forceinline__ void grid_barrier(Ctx &c, const FwdBufs &fb) {
         unsigned it = 0;
         while (ld_acquire_u64(fb.bar) < c.bar_target) {
             ++it;
-            if ((it & 255u) == 0 && (it > SPIN_LIMIT || *(volatile int32_t *)fb.abort_flag)) {
+            if ((it & 255u) == 0 && (it > 4u * SPIN_LIMIT || *(volatile int32_t *)fb.abort_flag)) {
                 atomicCAS(fb.abort_flag, 0, 1);
                 break;
             }

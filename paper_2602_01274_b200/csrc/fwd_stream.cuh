@@ -11,16 +11,20 @@
 
 namespace fwd {
 
-// Bounded wait on a shared-memory barrier phase.
-__device__ __forceinline__ void wait_bar(const FwdBufs &fb, uint64_t *bar, uint32_t parity, int code) {
+// Bounded wait on a shared-memory barrier phase.  Returns false when it gave up
+// (its own limit, or another wait of the grid gave up before).
+__device__ __forceinline__ bool wait_bar(const FwdBufs &fb, uint64_t *bar, uint32_t parity, int code, int info = 0) {
     unsigned it = 0;
     while (!mbar_try_wait(bar, parity)) {
         ++it;
-        if ((it & 1023u) == 0 && (it > SPIN_LIMIT || *(volatile int32_t *)fb.abort_flag)) {
-            atomicCAS(fb.abort_flag, 0, code);
-            break;
+        if ((it & 1023u) == 0 && (it > MBAR_SPIN_LIMIT || *(volatile int32_t *)fb.abort_flag)) {
+            if (atomicCAS(fb.abort_flag, 0, code) == 0) {      // first wait of the grid to give up: leave a note
+                fb.abort_flag[1] = blockIdx.x; fb.abort_flag[2] = threadIdx.x >> 5; fb.abort_flag[3] = info;
+            }
+            return false;
         }
     }
+    return true;
 }
 
 // Bounded wait until a shared-memory counter written by another warp reaches `want`.
@@ -29,7 +33,9 @@ __device__ __forceinline__ void wait_count(const FwdBufs &fb, volatile int32_t *
     while (*p < want) {
         ++it;
         if ((it & 1023u) == 0 && (it > SPIN_LIMIT * 4u || *(volatile int32_t *)fb.abort_flag)) {
-            atomicCAS(fb.abort_flag, 0, code);
+            if (atomicCAS(fb.abort_flag, 0, code) == 0) {
+                fb.abort_flag[1] = blockIdx.x; fb.abort_flag[2] = threadIdx.x >> 5; fb.abort_flag[3] = want;
+            }
             break;
         }
     }
@@ -39,8 +45,9 @@ __device__ __forceinline__ int n_ops(const Plan &P) { return 4 * P.n_layers + (P
 __device__ __forceinline__ int op_index(const Plan &P, int q) { return q < 4 * P.n_layers ? (q & 3) : OP_HEAD; }
 __device__ __forceinline__ int op_layer(const Plan &P, int q) { return q < 4 * P.n_layers ? (q >> 2) : 0; }
 
-// Warp W_PRODUCER: every weight unit of the block, for the whole forward, in order.
-__device__ __forceinline__ void weight_producer(Ctx &c, const FwdBufs &fb, const Plan &P) {
+// Warps W_PRODUCER ..: every weight unit of the block, for the whole forward, in
+// order; producer `me` issues the units n with n % W_PRODUCERS == me.
+__device__ __forceinline__ void weight_producer(Ctx &c, const FwdBufs &fb, const Plan &P, int me) {
     int n = 0;
     for (int q = 0; q < n_ops(P); ++q) {
         const GemmOp &op = P.op[op_index(P, q)];
@@ -52,9 +59,9 @@ __device__ __forceinline__ void weight_producer(Ctx &c, const FwdBufs &fb, const
             for (int k = 0; k < op.K; k += KC) {
                 const uint32_t bytes = (uint32_t)min(KC, op.K - k) * 2u;
                 for (int i = 0; i < Tp; ++i, ++n) {
+                    if (n % W_PRODUCERS != me) continue;
                     const int slot = n % NS, tile = t0 + p0 + i;
-                    wait_bar(fb, c.wempty + slot, (((uint32_t)(n / NS)) & 1u) ^ 1u, 5);
-                    if (*(volatile int32_t *)fb.abort_flag) return;      // a wait ran out somewhere: stop feeding
+                    if (!wait_bar(fb, c.wempty + slot, (((uint32_t)(n / NS)) & 1u) ^ 1u, 5, n)) return;   // stop feeding
                     if (c.lane == 0) mbar_expect_tx(c.wfull + slot, 16u * bytes);
                     __syncwarp();
                     if (c.lane < 16) {
@@ -118,7 +125,7 @@ __device__ __forceinline__ void activation_producer(Ctx &c, const FwdBufs &fb, c
                     inv_done = true;
                 }
                 const int slot = m % XS;
-                wait_bar(fb, c.xempty + slot, (((uint32_t)(m / XS)) & 1u) ^ 1u, 7);
+                wait_bar(fb, c.xempty + slot, (((uint32_t)(m / XS)) & 1u) ^ 1u, 7, m);
                 if (c.lane == 0) {
                     const uint32_t bytes = (uint32_t)(min(KC, op.K - k) >> 5) * (uint32_t)NT * 512u;
                     mbar_expect_tx(c.xfull + slot, bytes);
@@ -186,18 +193,18 @@ __device__ __forceinline__ void gemm_op(Ctx &c, const FwdBufs &fb, const Plan &P
         for (int k = 0; k < op.K; k += KC) {
             const int nch = min(KC, op.K - k) >> 5;
             const int xslot = c.xn % XS;
-            wait_bar(fb, c.xfull + xslot, ((uint32_t)(c.xn / XS)) & 1u, 8);
+            wait_bar(fb, c.xfull + xslot, ((uint32_t)(c.xn / XS)) & 1u, 8, c.xn);
             const uint4 *xs = reinterpret_cast<const uint4 *>(c.scratch + xslot * XSTAGE_BYTES);
             if (has0) {
                 const int n = c.wn + c.warp, slot = n % NS;
-                wait_bar(fb, c.wfull + slot, ((uint32_t)(n / NS)) & 1u, 9);
+                wait_bar(fb, c.wfull + slot, ((uint32_t)(n / NS)) & 1u, 9, n);
                 consume_unit<NT>(c.ring + slot * STAGE_BYTES, xs, nch, acc0, c.lane);
                 __syncwarp();
                 if (c.lane == 0) mbar_arrive(c.wempty + slot);
             }
             if (has1) {
                 const int n = c.wn + c.warp + MMA_WARPS, slot = n % NS;
-                wait_bar(fb, c.wfull + slot, ((uint32_t)(n / NS)) & 1u, 9);
+                wait_bar(fb, c.wfull + slot, ((uint32_t)(n / NS)) & 1u, 9, n);
                 consume_unit<NT>(c.ring + slot * STAGE_BYTES, xs, nch, acc1, c.lane);
                 __syncwarp();
                 if (c.lane == 0) mbar_arrive(c.wempty + slot);
@@ -206,6 +213,10 @@ __device__ __forceinline__ void gemm_op(Ctx &c, const FwdBufs &fb, const Plan &P
             if (c.lane == 0) mbar_arrive(c.xempty + xslot);
             c.wn += Tp;
             ++c.xn;
+            // Lockstep over k: a ring stage is shared by different warps at different times, and a parity wait
+            // is exact only while the waiter is less than one stage generation ahead.  After this barrier every
+            // unit of the k step is consumed, so the next step's waits (at most MAX_TILES <= NS units on) are exact.
+            bsync();
         }
         if (has0 || has1) {
             wait_count(fb, c.ready_op + 1, q + 1, 10);                 // RMS statistics of this projection's input

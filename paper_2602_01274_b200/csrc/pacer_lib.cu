@@ -165,7 +165,7 @@ static Layout make_layout(const pacer_cfg &c) {
     L.row_margin = cv.take(sizeof(float) * fwd::MAX_ROWS);
     L.att_cnt = cv.take(sizeof(int32_t) * (size_t)B * h_max);
     L.bar = cv.take(sizeof(unsigned long long));
-    L.abort_flag = cv.take(sizeof(int32_t));
+    L.abort_flag = cv.take(sizeof(int32_t) * 4);
     L.prof = cv.take(sizeof(unsigned long long) * fwd::PROF_STAMPS * fwd::PROF_BLOCKS);
     L.state_bytes = cv.off;                                   // zeroed at create
     L.hpend = cv.take(sizeof(float) * B * (c.block_b + 1) * c.draft.d_model);
@@ -423,7 +423,7 @@ static int start_run(pacer_ctx *c, const int32_t *prompt, int batch, int n_promp
     }
     CK(cudaMemcpyAsync(c->d.st, hs.data(), sizeof(SeqState) * hs.size(), cudaMemcpyHostToDevice, c->stream));
     // arrival counters, grid barrier and abort flag start from zero (they are contiguous in the workspace)
-    CK(cudaMemsetAsync(c->fb.att_cnt, 0, (char *)c->fb.abort_flag + sizeof(int32_t) - (char *)c->fb.att_cnt, c->stream));
+    CK(cudaMemsetAsync(c->fb.att_cnt, 0, (char *)c->fb.abort_flag + 4 * sizeof(int32_t) - (char *)c->fb.att_cnt, c->stream));
     CK(cudaMemcpy2DAsync(c->d.x, sizeof(int32_t) * k.max_ctx, prompt, sizeof(int32_t) * n_prompt, sizeof(int32_t) * n_prompt,
                          batch, cudaMemcpyHostToDevice, c->stream));
     CK(cudaStreamSynchronize(c->stream));        // hs is a local
@@ -556,9 +556,12 @@ static int collect(pacer_ctx *c, int batch, int max_new, int n_prompt, int32_t *
     CK(cudaMemcpy2DAsync(out_tokens, sizeof(int32_t) * max_new, c->d.x + n_prompt, sizeof(int32_t) * k.max_ctx,
                          sizeof(int32_t) * max_new, batch, cudaMemcpyDeviceToHost, c->stream));
     CK(cudaStreamSynchronize(c->stream));
-    int32_t aborted = 0;
-    CK(cudaMemcpy(&aborted, c->fb.abort_flag, sizeof aborted, cudaMemcpyDeviceToHost));
-    if (aborted) return fail(c, PACER_EDEVICE, "a bounded wait inside the forward kernel ran out");
+    int32_t aborted[4] = {0, 0, 0, 0};
+    CK(cudaMemcpy(aborted, c->fb.abort_flag, sizeof aborted, cudaMemcpyDeviceToHost));
+    if (aborted[0])
+        return fail(c, PACER_EDEVICE, "a bounded wait inside the forward kernel ran out (wait code " + std::to_string(aborted[0]) +
+                                          ", block " + std::to_string(aborted[1]) + ", warp " + std::to_string(aborted[2]) +
+                                          ", detail " + std::to_string(aborted[3]) + ")");
     int64_t nd = 0, nm = 0, nt = 0, ns = 0, ng = 0;
     for (int s = 0; s < batch; ++s) {
         const SeqState &a = hs[s];
