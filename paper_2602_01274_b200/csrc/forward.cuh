@@ -8,18 +8,20 @@
 //     with bulk async copies (cp.async.bulk + mbarrier); it runs ahead into the
 //     next projection while the block sits in a grid barrier or in a small
 //     phase, so the HBM queue never drains between projections;
-//   - a block owns whole 16-row tiles of a projection over the full k extent
-//     (no split-k: no partial sums, no atomics, no fences), the eight MMA warps
+//   - a block owns whole 16-row tiles of a projection over its k range (no
+//     partial-sum buffers, no arrival counters, no fences), the eight MMA warps
 //     advance over k in lockstep, and the activation rows of each 256-wide k
-//     step arrive through a second small ring, copied by a second producer warp
-//     from a bf16 buffer that already has MMA fragment order;
+//     step arrive through a second small ring, filled by activation-producer warps;
 //   - tensor cores (mma.m16n8k16, bf16 in / fp32 accumulate, weights as the
 //     16-row operand) do the contraction, so the math is invisible;
 //   - the row-wise step that follows a projection in the decoder (residual add,
-//     RMSNorm input of the next projection, SwiGLU, bias/arg-max of the LM head)
-//     is the epilogue of the warp that owns the tile; RMSNorm's 1/rms factor is
-//     applied to the OUTPUT rows of the next projection, so its input can be
-//     written before the row's sum of squares is complete;
+//     SwiGLU, bias/arg-max of the LM head) is the epilogue of the warp that owns
+//     the tile; RMSNorm is split: the activation producers multiply x by the
+//     gain while they convert it to bf16 and sum x^2 on the way, and the 1/rms
+//     factor is applied to the OUTPUT rows in the projection's epilogue;
+//   - the two projections with few output columns (attention output, MLP down)
+//     are cut along k as well, and add their partial sums straight into the
+//     fp32 residual stream with fire-and-forget atomic adds;
 //   - phases are separated by grid barriers with bounded waits.
 #pragma once
 #include "common.cuh"
@@ -27,19 +29,20 @@
 namespace fwd {
 
 constexpr int MMA_WARPS = 8, MMA_THREADS = 256;  // warps 0..7: MMAs, epilogues and all block-wide phases
-constexpr int W_PRODUCERS = 4;                   // warps 8..11 stream weights (unit n by producer n % 4: one warp alone
-                                                 // cannot issue bulk copies fast enough), warp 12 activations + RMS statistics
-constexpr int W_PRODUCER = 8, X_PRODUCER = W_PRODUCER + W_PRODUCERS;
-constexpr int THREADS = 32 * (X_PRODUCER + 1);
+constexpr int W_PRODUCERS = 4;                   // warps 8..11 stream weights: unit n by producer n % 4 (one warp alone
+                                                 // cannot issue the bulk copies fast enough)
+constexpr int X_PRODUCERS = 4;                   // warps 12..15 provide the activation chunks: chunk m by producer m % 4
+constexpr int W_PRODUCER = MMA_WARPS, X_PRODUCER = W_PRODUCER + W_PRODUCERS;
+constexpr int THREADS = 32 * (X_PRODUCER + X_PRODUCERS);
 constexpr int KC = 256;                         // k columns of one weight unit
 constexpr int PITCH = KC * 2 + 64;              // bytes between the rows of a stage (bank-conflict free)
 constexpr int STAGE_BYTES = 16 * PITCH;         // 9216
 constexpr int NS = 16;                          // weight stages in the ring
 constexpr int RING_BYTES = NS * STAGE_BYTES;    // 147456
-constexpr int XS = 3;                           // activation stages
+constexpr int XS = 4;                           // activation stages
 constexpr int XSTAGE_BYTES = 4 * 4096;          // up to 4 row tiles x 8 chunks x 512 bytes
 constexpr int SCRATCH_BYTES = 80 * 1024;        // the activation ring lives in its first 48 KB; the attention
-                                                // phase and the tails use all of it (no activations in flight then)
+                                                // phase and the tails use all of it (no activations in flight then); XS * XSTAGE_BYTES <= SCRATCH_BYTES
 constexpr int MISC_BYTES = 2048;
 constexpr int SMEM_BYTES = SCRATCH_BYTES + RING_BYTES + MISC_BYTES;
 constexpr int MAX_TILES = 16;                   // tiles of one pass of a block (two per MMA warp)
@@ -61,6 +64,8 @@ struct GemmOp {
     int32_t N;               // weight rows in all (gate/up: 2F)
     int32_t MT;              // 16-row tiles
     int32_t K;
+    int32_t S;               // k slices (1, or a divisor of the grid size for the two projections whose outputs
+                             // are ADDED to the residual stream: their partial sums go there with atomic adds)
     int32_t rot;             // block that gets the first tile range (spreads the one-tile imbalance)
     int32_t interleave;      // 1: tile t = gate rows 8t..8t+7 then up rows 8t..8t+7
 };
@@ -73,8 +78,6 @@ struct Plan {
 // Device buffers of the forward kernel beyond DevPtrs (all in the workspace).
 struct FwdBufs {
     float *qkv;              // [MAX_ROWS][qrows] fp32
-    bf16 *xg;                // x * gain of the next RMSNorm, bf16 in fragment order (its 1/rms comes later)
-    float *ssq;              // [d/16][MAX_ROWS] sum of squares of x over the 16 columns of a tile
     float *tile_top;         // [MT(head)][MAX_ROWS][4]: max, argmax (int bits), runner-up, unused
     float *attp;             // attention partials [seq*H + h][split][row][hd + 2]
     int32_t *att_cnt;        // [batch * H]
@@ -159,13 +162,21 @@ struct Ctx {
 // Barrier of the eight MMA warps (the producer warps never join it).
 __device__ __forceinline__ void bsync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
-// Tile range of block `cta` for a projection with MT tiles.
-__device__ __host__ __forceinline__ void tile_range(int MT, int rot, int cta, int ncta, int &t0, int &T) {
-    int ci = cta - rot;
+// Work of block `cta` in a projection: tiles [t0, t0 + T) over the k range [k_lo, k_hi).
+// With S slices the blocks form ncta / S groups; a group shares a tile range and its S
+// blocks take one k slice each (slices are whole KC steps).
+__device__ __host__ __forceinline__ void op_range(const GemmOp &op, int cta, int ncta, int &t0, int &T, int &k_lo, int &k_hi) {
+    int ci = cta - op.rot;
     if (ci < 0) ci += ncta;
-    const int base = MT / ncta, rem = MT % ncta;
-    T = base + (ci < rem ? 1 : 0);
-    t0 = ci * base + (ci < rem ? ci : rem);
+    const int groups = ncta / op.S, g = ci / op.S, s = ci % op.S;
+    const int base = op.MT / groups, rem = op.MT % groups;
+    T = g < groups ? base + (g < rem ? 1 : 0) : 0;
+    t0 = g * base + (g < rem ? g : rem);
+    const int nks = (op.K + KC - 1) / KC, sb = nks / op.S, sr = nks % op.S;
+    k_lo = (s * sb + (s < sr ? s : sr)) * KC;
+    k_hi = k_lo + (sb + (s < sr ? 1 : 0)) * KC;
+    if (k_hi > op.K) k_hi = op.K;
+    if (k_lo >= k_hi) T = 0;
 }
 
 // Grid barrier (MMA warps only): every block arrives once; waits are bounded.  A wait that runs

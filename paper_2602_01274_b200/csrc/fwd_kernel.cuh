@@ -14,6 +14,20 @@ __device__ __forceinline__ float hidden_at(const Args &a, const Ctx &c, int r, i
     return __ldcg(a.d.xres + (size_t)r * a.m.cfg.d_model + i) * c.inv_rms[r] * __bfloat162float(a.m.normf[i]);
 }
 
+// 1/rms of the final residual rows of sequence s, for the final RMSNorm the tails apply (MMA warps of one block).
+__device__ __forceinline__ void tail_inv_rms(Ctx &c, const Args &a, int s) {
+    const int dm = a.m.cfg.d_model;
+    float *red = reinterpret_cast<float *>(c.scratch);
+    for (int j = 0; j < c.n_rows[s]; ++j) {
+        const int r = s * a.g.rps + j;
+        float ss = 0.f;
+        for (int i = threadIdx.x; i < dm; i += MMA_THREADS) { const float v = __ldcg(a.d.xres + (size_t)r * dm + i); ss += v * v; }
+        ss = mma_block_sum(ss, red);
+        if (threadIdx.x == 0) c.inv_rms[r] = rsqrtf(ss / (float)dm + a.m.cfg.rms_eps);
+    }
+    bsync();
+}
+
 // End of one draft forward (Eq. 6): y_i, h_i queued for the pre-verification model, cache length.
 __device__ __forceinline__ void tail_draft(Ctx &c, const Args &a, int s) {
     const DevPtrs &d = a.d;
@@ -194,26 +208,30 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
 
     // the two producer warps live in their streams until the forward's last unit
     if (c.warp >= W_PRODUCER && c.warp < X_PRODUCER) { weight_producer(c, a.fb, a.P, c.warp - W_PRODUCER); return; }
-    if (c.warp == X_PRODUCER) {
+    if (c.warp >= X_PRODUCER) {
         uint64_t keep;
         asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(keep));
-        activation_producer(c, a.fb, a.P, NT, m.cfg.d_model, m.cfg.rms_eps, keep);
+        XSrc xs;
+        xs.xres = d.xres; xs.norm1 = m.norm1; xs.norm2 = m.norm2; xs.normf = m.normf;
+        xs.dm = m.cfg.d_model; xs.rtot = g.rtot; xs.eps = m.cfg.rms_eps;
+        xs.xss = reinterpret_cast<float *>(misc + 1536);                     // [X_PRODUCERS][MAX_ROWS]
+        activation_producer<NT>(c, a.fb, a.P, xs, c.warp - X_PRODUCER, keep);
         return;
     }
 
-    const int dm = m.cfg.d_model;
     int n_stamp = 0;
     auto stamp = [&]() {
         if (a.fb.prof && threadIdx.x == 0 && n_stamp < PROF_STAMPS)
             a.fb.prof[(size_t)c.cta * PROF_STAMPS + n_stamp++] = globaltimer_ns();
     };
     stamp();
-    phase_begin(c, a, NT);
+    phase_begin(c, a);
     stamp();
     grid_barrier(c, a.fb);
     stamp();
 
     const int L = a.P.n_layers;
+    (void)m;
     for (int l = 0; l < L; ++l) {
         gemm_op<NT>(c, a.fb, a.P, 4 * l + OP_QKV, [&](int tile, float (&acc)[NT][4]) { epi_qkv<NT>(c, a, tile, acc); });
         stamp();
@@ -223,8 +241,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
         stamp();
         grid_barrier(c, a.fb);
         stamp();
-        gemm_op<NT>(c, a.fb, a.P, 4 * l + OP_O,
-                    [&](int tile, float (&acc)[NT][4]) { epi_residual<NT>(c, a, m.norm2 + (size_t)l * dm, tile, acc); });
+        gemm_op<NT>(c, a.fb, a.P, 4 * l + OP_O, [&](int tile, float (&acc)[NT][4]) { epi_residual<NT>(c, a, tile, acc); });
         stamp();
         grid_barrier(c, a.fb);
         stamp();
@@ -232,9 +249,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
         stamp();
         grid_barrier(c, a.fb);
         stamp();
-        const bf16 *gain_next = l + 1 < L ? m.norm1 + (size_t)(l + 1) * dm : m.normf;
-        gemm_op<NT>(c, a.fb, a.P, 4 * l + OP_DOWN,
-                    [&](int tile, float (&acc)[NT][4]) { epi_residual<NT>(c, a, gain_next, tile, acc); });
+        gemm_op<NT>(c, a.fb, a.P, 4 * l + OP_DOWN, [&](int tile, float (&acc)[NT][4]) { epi_residual<NT>(c, a, tile, acc); });
         stamp();
         grid_barrier(c, a.fb);
         stamp();
@@ -252,9 +267,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
         }
     }
     if (c.cta < g.batch && kind != KIND_VERIFY) {
-        // final RMSNorm statistics for the hidden rows the tails need
-        if (c.warp == 0) compute_inv(c, a.fb, dm, m.cfg.rms_eps);
-        bsync();
+        if (kind != KIND_AR) tail_inv_rms(c, a, c.cta);     // the tails below apply the final RMSNorm themselves
         if (kind == KIND_DRAFT) tail_draft(c, a, c.cta);
         else if (kind == KIND_MB) tail_mb(c, a, c.cta);
         else if (kind == KIND_AR) tail_ar(c, a, c.cta);
@@ -278,14 +291,21 @@ static inline Plan make_plan(const ModelDev &m, const DevPtrs &d, const FwdBufs 
     auto set = [&](int i, const bf16 *w1, const bf16 *w2, const bf16 *x, long long lstride, int N, int K, int MT, int inter) {
         GemmOp &o = P.op[i];
         o.W1 = w1; o.W2 = w2 ? w2 : w1; o.X = x; o.lstride = lstride; o.N = N; o.K = K; o.MT = MT; o.interleave = inter;
+        // the projections that add into the residual stream are also cut along k when they have few tiles
+        o.S = 1;
+        if (i == OP_O || i == OP_DOWN) {
+            const int nks = (K + KC - 1) / KC;
+            for (int sdiv = 2; sdiv <= 8; ++sdiv)
+                if (ncta % sdiv == 0 && sdiv <= nks && MT * (sdiv / 2) < 4 * ncta) o.S = sdiv;
+        }
         o.rot = rot;
-        rot = (rot + MT % ncta) % ncta;       // the next projection's extra tiles go to other blocks
+        rot = (rot + (MT % (ncta / o.S)) * o.S) % ncta;       // the next projection's extra tiles go to other blocks
     };
-    set(OP_QKV, m.wqkv, nullptr, fb.xg, (long long)m.qrows * dm, m.qrows, (int)dm, (m.qrows + 15) / 16, 0);
+    set(OP_QKV, m.wqkv, nullptr, nullptr, (long long)m.qrows * dm, m.qrows, (int)dm, (m.qrows + 15) / 16, 0);
     set(OP_O, m.wo, nullptr, d.att, dm * hh, (int)dm, (int)hh, ((int)dm + 15) / 16, 0);
-    set(OP_GU, m.wgate, m.wup, fb.xg, F * dm, (int)(2 * F), (int)dm, ((int)F + 7) / 8, 1);
+    set(OP_GU, m.wgate, m.wup, nullptr, F * dm, (int)(2 * F), (int)dm, ((int)F + 7) / 8, 1);
     set(OP_DOWN, m.wdown, nullptr, d.act, dm * F, (int)dm, (int)F, ((int)dm + 15) / 16, 0);
-    set(OP_HEAD, m.head, nullptr, fb.xg, 0, k.vocab, (int)dm, (k.vocab + 15) / 16, 0);
+    set(OP_HEAD, m.head, nullptr, nullptr, 0, k.vocab, (int)dm, (k.vocab + 15) / 16, 0);
     P.n_layers = k.n_layers;
     P.has_head = has_head ? 1 : 0;
     return P;

@@ -52,12 +52,12 @@ __device__ __forceinline__ void weight_producer(Ctx &c, const FwdBufs &fb, const
     for (int q = 0; q < n_ops(P); ++q) {
         const GemmOp &op = P.op[op_index(P, q)];
         const size_t lbase = (size_t)op_layer(P, q) * op.lstride;
-        int t0, T;
-        tile_range(op.MT, op.rot, c.cta, c.ncta, t0, T);
+        int t0, T, k_lo, k_hi;
+        op_range(op, c.cta, c.ncta, t0, T, k_lo, k_hi);
         for (int p0 = 0; p0 < T; p0 += MAX_TILES) {
             const int Tp = min(MAX_TILES, T - p0);
-            for (int k = 0; k < op.K; k += KC) {
-                const uint32_t bytes = (uint32_t)min(KC, op.K - k) * 2u;
+            for (int k = k_lo; k < k_hi; k += KC) {
+                const uint32_t bytes = (uint32_t)min(KC, k_hi - k) * 2u;
                 for (int i = 0; i < Tp; ++i, ++n) {
                     if (n % W_PRODUCERS != me) continue;
                     const int slot = n % NS, tile = t0 + p0 + i;
@@ -81,68 +81,132 @@ __device__ __forceinline__ void weight_producer(Ctx &c, const FwdBufs &fb, const
     }
 }
 
-// inv_rms[r] = 1 / sqrt(mean(x_r^2) + eps) from the per-tile sums ssq[tile][row], in a fixed
-// order (one warp, lane = row; four running sums keep the loads independent).
-__device__ __forceinline__ void compute_inv(Ctx &c, const FwdBufs &fb, int dm, float eps) {
-    const int ntiles = dm >> 4;
-    const float *p = fb.ssq + c.lane;
-    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-    int t = 0;
-    for (; t + 4 <= ntiles; t += 4) {
-        s0 += __ldcg(p + (t + 0) * MAX_ROWS);
-        s1 += __ldcg(p + (t + 1) * MAX_ROWS);
-        s2 += __ldcg(p + (t + 2) * MAX_ROWS);
-        s3 += __ldcg(p + (t + 3) * MAX_ROWS);
-    }
-    for (; t < ntiles; ++t) s0 += __ldcg(p + t * MAX_ROWS);
-    c.inv_rms[c.lane] = rsqrtf(((s0 + s1) + (s2 + s3)) / (float)dm + eps);
-    __syncwarp();
+// What the activation producers read.
+struct XSrc {
+    const float *xres;                       // fp32 residual stream [row][d]
+    const bf16 *norm1, *norm2, *normf;       // RMSNorm gains
+    int32_t dm, rtot;
+    float eps;
+    float *xss;                              // shared: [X_PRODUCERS][MAX_ROWS] partial sums of x^2
+};
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t *>(&v);
 }
 
-// Warp X_PRODUCER: the activation chunk of every k step once the projection's
-// inputs are complete (the MMA warps raise ready_op[0] after the grid barrier),
-// and the RMS statistics the projection's epilogue applies.
-__device__ __forceinline__ void activation_producer(Ctx &c, const FwdBufs &fb, const Plan &P, int NT, int dm, float eps,
+// One k step of RMSNorm's input side: x * gain as bf16 in fragment order
+// [chunk of 32 k][row tile][lane = (r % 8) * 4 + (k % 32) / 8] x 8 values, written
+// into an activation stage by one warp; ss[r] gathers this lane's share of sum(x_r^2).
+template <int NT>
+__device__ __forceinline__ void convert_chunk(Ctx &c, const XSrc &xs, const bf16 *gain, int k0, int nch, uint4 *stage,
+                                              float (&ss)[NT * 8], bool sum) {
+    const int p = c.lane;                    // 16-byte piece (8 k) of the k step
+    if (p < nch * 4) {
+        const int k = k0 + p * 8;
+        const uint4 gw = *reinterpret_cast<const uint4 *>(gain + k);
+        const __nv_bfloat162 *g2 = reinterpret_cast<const __nv_bfloat162 *>(&gw);
+        const float2 ga = __bfloat1622float2(g2[0]), gb = __bfloat1622float2(g2[1]);
+        const float2 gc = __bfloat1622float2(g2[2]), gd = __bfloat1622float2(g2[3]);
+        constexpr int RB = 8;                // rows whose loads are issued together (one round trip per group)
+#pragma unroll
+        for (int r0 = 0; r0 < NT * 8; r0 += RB) {
+            float4 xa[RB], xb[RB];
+            bool act[RB];
+#pragma unroll
+            for (int j = 0; j < RB; ++j) {
+                const int r = r0 + j;
+                act[j] = r < xs.rtot && c.row_pos[r] >= 0;                             // the same in every lane
+                if (act[j]) {
+                    const float *src = xs.xres + (size_t)r * xs.dm + k;
+                    xa[j] = __ldcg(reinterpret_cast<const float4 *>(src));
+                    xb[j] = __ldcg(reinterpret_cast<const float4 *>(src + 4));
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < RB; ++j) {
+                const int r = r0 + j;
+                uint4 out = make_uint4(0u, 0u, 0u, 0u);
+                if (act[j]) {
+                    const float4 x0 = xa[j], x1 = xb[j];
+                    out.x = pack_bf16x2(x0.x * ga.x, x0.y * ga.y);
+                    out.y = pack_bf16x2(x0.z * gb.x, x0.w * gb.y);
+                    out.z = pack_bf16x2(x1.x * gc.x, x1.y * gc.y);
+                    out.w = pack_bf16x2(x1.z * gd.x, x1.w * gd.y);
+                    if (sum)
+                        ss[r] += (x0.x * x0.x + x0.y * x0.y) + (x0.z * x0.z + x0.w * x0.w) + (x1.x * x1.x + x1.y * x1.y) +
+                                 (x1.z * x1.z + x1.w * x1.w);
+                }
+                stage[((p >> 2) * NT + (r >> 3)) * 32 + ((r & 7) << 2) + (p & 3)] = out;
+            }
+        }
+    }
+}
+
+// Warps X_PRODUCER ..: the activation chunk of every k step, once the projection's
+// inputs are complete (the MMA warps raise ready_op[0] after the grid barrier).
+// Projections that follow an RMSNorm get x * gain converted on the fly, and the
+// producers leave 1/rms per row for the epilogues (ready_op[1]); the others get a
+// bulk copy of a bf16 buffer that already has fragment order.
+template <int NT>
+__device__ __forceinline__ void activation_producer(Ctx &c, const FwdBufs &fb, const Plan &P, const XSrc &xs, int me,
                                                     uint64_t keep_policy) {
     int m = 0;
+    bool dead = false;                       // a wait gave up: keep walking (the barriers below must be met), do nothing
     for (int q = 0; q < n_ops(P); ++q) {
-        const int opi = op_index(P, q);
+        const int opi = op_index(P, q), layer = op_layer(P, q);
         const GemmOp &op = P.op[opi];
         const bool normed = opi == OP_QKV || opi == OP_GU || opi == OP_HEAD;
-        int t0, T;
-        tile_range(op.MT, op.rot, c.cta, c.ncta, t0, T);
+        const bf16 *gain = opi == OP_QKV ? xs.norm1 + (size_t)layer * xs.dm : opi == OP_GU ? xs.norm2 + (size_t)layer * xs.dm : xs.normf;
+        int t0, T, k_lo, k_hi;
+        op_range(op, c.cta, c.ncta, t0, T, k_lo, k_hi);
+        if (T == 0) continue;
         wait_count(fb, c.ready_op, q + 1, 6);
         __threadfence_block();
         asm volatile("fence.proxy.async;" ::: "memory");
-        bool inv_done = !normed;
-        int issued = 0;
+        float ss[NT * 8];
+#pragma unroll
+        for (int r = 0; r < NT * 8; ++r) ss[r] = 0.f;
         for (int p0 = 0; p0 < T; p0 += MAX_TILES) {
-            for (int k = 0; k < op.K; k += KC, ++m, ++issued) {
-                if (!inv_done && issued == XS) {          // the ring is full: a good moment for the statistics
-                    compute_inv(c, fb, dm, eps);
-                    __threadfence_block();
-                    if (c.lane == 0) c.ready_op[1] = q + 1;
-                    inv_done = true;
-                }
-                const int slot = m % XS;
-                wait_bar(fb, c.xempty + slot, (((uint32_t)(m / XS)) & 1u) ^ 1u, 7, m);
-                if (c.lane == 0) {
-                    const uint32_t bytes = (uint32_t)(min(KC, op.K - k) >> 5) * (uint32_t)NT * 512u;
+            for (int k = k_lo; k < k_hi; k += KC, ++m) {
+                if (m % X_PRODUCERS != me || dead) continue;
+                const int slot = m % XS, nch = min(KC, k_hi - k) >> 5;
+                if (!wait_bar(fb, c.xempty + slot, (((uint32_t)(m / XS)) & 1u) ^ 1u, 7, m)) { dead = true; continue; }
+                if (normed) {
+                    convert_chunk<NT>(c, xs, gain, k, nch, reinterpret_cast<uint4 *>(c.scratch + slot * XSTAGE_BYTES), ss, p0 == 0);
+                    __syncwarp();
+                    if (c.lane == 0) mbar_arrive(c.xfull + slot);
+                } else if (c.lane == 0) {
+                    const uint32_t bytes = (uint32_t)nch * (uint32_t)NT * 512u;
                     mbar_expect_tx(c.xfull + slot, bytes);
                     bulk_g2s(c.scratch + slot * XSTAGE_BYTES, op.X + (size_t)(k >> 5) * NT * 256, bytes, c.xfull + slot,
                              keep_policy);
                 }
                 __syncwarp();
             }
+            if (normed && p0 == 0) {         // 1/rms per row from the four producers' shares, in a fixed order
+#pragma unroll
+                for (int r = 0; r < NT * 8; ++r) {
+                    float v = ss[r];
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+                    if (c.lane == 0) xs.xss[me * MAX_ROWS + r] = v;
+                }
+                asm volatile("bar.sync 2, 128;" ::: "memory");
+                if (me == 0) {
+                    if (c.lane < NT * 8) {
+                        float v = 0.f;
+#pragma unroll
+                        for (int j = 0; j < X_PRODUCERS; ++j) v += xs.xss[j * MAX_ROWS + c.lane];
+                        c.inv_rms[c.lane] = rsqrtf(v / (float)xs.dm + xs.eps);
+                    }
+                    __syncwarp();
+                    __threadfence_block();
+                    if (c.lane == 0) c.ready_op[1] = q + 1;
+                }
+                asm volatile("bar.sync 2, 128;" ::: "memory");
+            }
         }
-        if (!inv_done) {
-            compute_inv(c, fb, dm, eps);
-            __threadfence_block();
-            if (c.lane == 0) c.ready_op[1] = q + 1;
-        } else if (!normed && c.lane == 0) {
-            c.ready_op[1] = q + 1;
-        }
-        __syncwarp();
     }
 }
 
@@ -180,8 +244,10 @@ __device__ __forceinline__ void gemm_op(Ctx &c, const FwdBufs &fb, const Plan &P
         __threadfence_block();
         c.ready_op[0] = q + 1;                 // the activation producer may start on this projection
     }
-    int t0, T;
-    tile_range(op.MT, op.rot, c.cta, c.ncta, t0, T);
+    const int opi = op_index(P, q);
+    const bool normed = opi == OP_QKV || opi == OP_GU || opi == OP_HEAD;
+    int t0, T, k_lo, k_hi;
+    op_range(op, c.cta, c.ncta, t0, T, k_lo, k_hi);
     for (int p0 = 0; p0 < T; p0 += MAX_TILES) {
         const int Tp = min(MAX_TILES, T - p0);
         const bool has0 = c.warp < Tp, has1 = c.warp + MMA_WARPS < Tp;
@@ -190,8 +256,8 @@ __device__ __forceinline__ void gemm_op(Ctx &c, const FwdBufs &fb, const Plan &P
         for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
             for (int i = 0; i < 4; ++i) acc0[nt][i] = acc1[nt][i] = 0.f;
-        for (int k = 0; k < op.K; k += KC) {
-            const int nch = min(KC, op.K - k) >> 5;
+        for (int k = k_lo; k < k_hi; k += KC) {
+            const int nch = min(KC, k_hi - k) >> 5;
             const int xslot = c.xn % XS;
             wait_bar(fb, c.xfull + xslot, ((uint32_t)(c.xn / XS)) & 1u, 8, c.xn);
             const uint4 *xs = reinterpret_cast<const uint4 *>(c.scratch + xslot * XSTAGE_BYTES);
@@ -218,8 +284,8 @@ __device__ __forceinline__ void gemm_op(Ctx &c, const FwdBufs &fb, const Plan &P
             // unit of the k step is consumed, so the next step's waits (at most MAX_TILES <= NS units on) are exact.
             bsync();
         }
-        if (has0 || has1) {
-            wait_count(fb, c.ready_op + 1, q + 1, 10);                 // RMS statistics of this projection's input
+        if (normed && (has0 || has1)) {
+            wait_count(fb, c.ready_op + 1, q + 1, 10);                 // 1/rms of this projection's input rows
             __threadfence_block();
         }
         if (has0) epi(t0 + p0 + c.warp, acc0);
