@@ -1,7 +1,10 @@
 // Attention phase of the forward kernel: rotary embedding of the new q/k rows,
 // append of k/v to the bf16 cache, and causal attention of the new rows over the
-// cache.  Work items are (sequence, head, key-range split); every item leaves an
-// un-normalised partial (running max, sum, weighted values) and the item that
+// cache, on tensor cores.  Work items are (sequence, head, key-range split).
+// Inside an item the eight MMA warps split the keys in steps of 16 (and the two
+// 16-row query tiles when there are more than 16 rows); every warp keeps a
+// running (max, sum, output) per row, FlashAttention style.  The warps' results
+// are merged through shared memory into the item's partial, and the item that
 // finishes last for a (sequence, head) merges the splits and writes the bf16
 // attention output in the fragment order the output projection reads.
 #pragma once
@@ -9,139 +12,226 @@
 
 namespace fwd {
 
-constexpr int ATT_RB = 8;      // query rows handled together by a warp
-constexpr int ATT_WARPS = MMA_WARPS;
+__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gsrc) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(smem_dst)), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], const void *smem_row) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(smem_u32(smem_row)));
+}
 
-template <int EPL>             // channels per lane: hd = 32 * EPL
-__device__ __forceinline__ void load_kv_row(const bf16 *p, float (&out)[EPL]) {
-    if constexpr (EPL == 4) {
-        const uint2 raw = *reinterpret_cast<const uint2 *>(p);
-        const __nv_bfloat162 *h2 = reinterpret_cast<const __nv_bfloat162 *>(&raw);
-        const float2 a = __bfloat1622float2(h2[0]), b = __bfloat1622float2(h2[1]);
-        out[0] = a.x; out[1] = a.y; out[2] = b.x; out[3] = b.y;
-    } else if constexpr (EPL == 2) {
-        const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(p));
-        out[0] = a.x; out[1] = a.y;
-    } else {
-        out[0] = __bfloat162float(p[0]);
+// Geometry of the shared-memory scratch during an attention item.
+template <int HD>
+struct AttSmem {
+    static constexpr int QP = HD * 2 + 64;   // bytes between query rows (conflict-free 16-byte reads of rows g, g+8)
+    static constexpr int VP = HD * 2 + 16;   // bytes between the rows of a V step (conflict-free ldmatrix)
+    static constexpr int PW = HD + 2;        // floats of a partial row: values, running max, running sum
+    static constexpr int Q_OFF = 0;                       // [32][QP] bf16 q, scaled and rotated
+    static constexpr int KN_OFF = 32 * QP;                // [32][HD] bf16 new keys as cached
+    static constexpr int VN_OFF = KN_OFF + 32 * HD * 2;   // [32][HD] bf16 new values as cached
+    static constexpr int VS_OFF = VN_OFF + 32 * HD * 2;   // [8 warps][16][VP] V rows of the current step
+    static constexpr int END = VS_OFF + MMA_WARPS * 16 * VP;
+    static_assert(END <= SCRATCH_BYTES, "attention staging does not fit the scratch");
+    static_assert(MMA_WARPS * 16 * PW * 4 <= SCRATCH_BYTES, "attention merge buffer does not fit the scratch");
+};
+
+// Rotary embedding of the new rows of (seq, head h): q (scaled) to shared memory
+// as bf16; k, v of the kv head rounded to bf16 as the cache holds them, to shared
+// memory and, by one item per kv head, to the cache.
+template <int HD>
+__device__ __forceinline__ void attention_rows(Ctx &c, const Args &a, int layer, int seq, int h, bool writer) {
+    using SM = AttSmem<HD>;
+    constexpr int half = HD / 2;
+    const DevPtrs &d = a.d;
+    const ModelDev &m = a.m;
+    const int H = m.cfg.n_heads, Hkv = m.cfg.n_kv_heads, kh = h / (H / Hkv), qrows = m.qrows;
+    const int n_r = c.n_rows[seq], r_base = seq * a.g.rps, pos0 = c.row_pos[r_base];
+    bf16 *kn = reinterpret_cast<bf16 *>(c.scratch + SM::KN_OFF), *vn = reinterpret_cast<bf16 *>(c.scratch + SM::VN_OFF);
+    const size_t cbase = (((size_t)layer * d.max_batch + seq) * Hkv + kh) * (size_t)d.max_ctx * HD;
+    const float scale = rsqrtf((float)HD);
+    for (int i = threadIdx.x; i < 32 * half; i += MMA_THREADS) {
+        const int j = i / half, ii = i - j * half;
+        bf16 *qrow = reinterpret_cast<bf16 *>(c.scratch + SM::Q_OFF + j * SM::QP);
+        if (j < n_r) {
+            const int pos = pos0 + j;
+            const float *row = a.fb.qkv + (size_t)(r_base + j) * qrows;
+            const float2 cs = m.rope[(size_t)pos * half + ii];
+            const float qa = __ldcg(row + h * HD + ii), qb = __ldcg(row + h * HD + ii + half);
+            qrow[ii] = __float2bfloat16((qa * cs.x - qb * cs.y) * scale);
+            qrow[ii + half] = __float2bfloat16((qb * cs.x + qa * cs.y) * scale);
+            const float ka = __ldcg(row + (H + kh) * HD + ii), kb = __ldcg(row + (H + kh) * HD + ii + half);
+            const bf16 k0 = __float2bfloat16(ka * cs.x - kb * cs.y), k1 = __float2bfloat16(kb * cs.x + ka * cs.y);
+            const bf16 v0 = __float2bfloat16(__ldcg(row + (H + Hkv + kh) * HD + ii));
+            const bf16 v1 = __float2bfloat16(__ldcg(row + (H + Hkv + kh) * HD + ii + half));
+            kn[j * HD + ii] = k0; kn[j * HD + ii + half] = k1;
+            vn[j * HD + ii] = v0; vn[j * HD + ii + half] = v1;
+            if (writer) {
+                bf16 *kc = m.kcache + cbase + (size_t)pos * HD, *vc = m.vcache + cbase + (size_t)pos * HD;
+                kc[ii] = k0; kc[ii + half] = k1;
+                vc[ii] = v0; vc[ii + half] = v1;
+            }
+        } else {
+            qrow[ii] = __float2bfloat16(0.f);
+            qrow[ii + half] = __float2bfloat16(0.f);
+        }
     }
 }
 
-template <int EPL>
+// The key loop of one warp: keys in steps of 16 (step st, st + KW, ...), first the
+// cached keys [lo, hi), then (last split only) the n_r keys of this forward, which
+// row j sees up to key j.  mt: the warp's 16-row query tile.  Leaves running max,
+// sum (this lane's share) and un-normalised output of rows g and g+8 of the tile.
+template <int HD>
+__device__ __forceinline__ void attention_keys(Ctx &c, const bf16 *kcache, const bf16 *vcache, int lo, int hi, int n_new,
+                                               int n_r, int mt, int kw, int KW, float (&mx)[2], float (&lsum)[2],
+                                               float (&o)[HD / 8][4]) {
+    using SM = AttSmem<HD>;
+    constexpr int NCH = HD / 32, NOT = HD / 8, QP = SM::QP, VP = SM::VP;
+    const int g = c.lane >> 2, t = c.lane & 3;
+    const bf16 *kn = reinterpret_cast<const bf16 *>(c.scratch + SM::KN_OFF), *vn = reinterpret_cast<const bf16 *>(c.scratch + SM::VN_OFF);
+    unsigned char *vslot = c.scratch + SM::VS_OFF + c.warp * (16 * VP);
+    const unsigned char *q0 = c.scratch + SM::Q_OFF + (mt * 16 + g) * QP + t * 16, *q1 = q0 + 8 * QP;
+    const int steps_c = (hi - lo + 15) >> 4, steps_n = (n_new + 15) >> 4;
+    for (int st = kw; st < steps_c + steps_n; st += KW) {
+        const bool fresh = st >= steps_c;                // keys of this forward (from shared memory), else cached keys
+        const int key0 = fresh ? (st - steps_c) * 16 : lo + st * 16;
+        const int kend = fresh ? n_r : hi;               // first invalid key index
+        const bf16 *kb = fresh ? kn : kcache, *vb = fresh ? vn : vcache;
+        // V rows of the step into this warp's slot (rows past the end repeat the last valid row: finite, and masked)
+        for (int i = c.lane; i < 16 * (HD / 8); i += 32) {
+            const int kr = i / (HD / 8), piece = i - kr * (HD / 8);
+            const bf16 *src = vb + (size_t)min(key0 + kr, kend - 1) * HD + piece * 8;
+            if (fresh) *reinterpret_cast<uint4 *>(vslot + kr * VP + piece * 16) = *reinterpret_cast<const uint4 *>(src);
+            else cp_async16(vslot + kr * VP + piece * 16, src);
+        }
+        // scores S = Q K^T for 16 keys: lane (g, t) reads 8 consecutive channels of key g of each 8-key tile and
+        // uses them as the k slots {2t, 2t+1, 2t+8, 2t+9} of two MMAs; q is read with the same rule
+        float s[2][4];
+#pragma unroll
+        for (int nb = 0; nb < 2; ++nb) {
+            s[nb][0] = s[nb][1] = s[nb][2] = s[nb][3] = 0.f;
+            const bf16 *krow = kb + (size_t)min(key0 + nb * 8 + g, kend - 1) * HD + t * 8;
+            uint4 kf[NCH];
+#pragma unroll
+            for (int cc = 0; cc < NCH; ++cc) kf[cc] = *reinterpret_cast<const uint4 *>(krow + cc * 32);
+#pragma unroll
+            for (int cc = 0; cc < NCH; ++cc) {
+                const uint4 qa = *reinterpret_cast<const uint4 *>(q0 + cc * 64), qb = *reinterpret_cast<const uint4 *>(q1 + cc * 64);
+                mma16816(s[nb], qa.x, qb.x, qa.y, qb.y, kf[cc].x, kf[cc].y);
+                mma16816(s[nb], qa.z, qb.z, qa.w, qb.w, kf[cc].z, kf[cc].w);
+            }
+        }
+        // mask: keys past the end; among the keys of this forward, row j sees keys 0..j
+        float rmax[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+        for (int nb = 0; nb < 2; ++nb)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int key = key0 + nb * 8 + 2 * t + (i & 1), row = mt * 16 + g + 8 * (i >> 1);
+                const bool ok = key < kend && (!fresh || key <= row);
+                if (!ok) s[nb][i] = -INFINITY;
+                rmax[i >> 1] = fmaxf(rmax[i >> 1], s[nb][i]);
+            }
+        float corr[2];
+#pragma unroll
+        for (int hr = 0; hr < 2; ++hr) {
+            rmax[hr] = fmaxf(rmax[hr], __shfl_xor_sync(0xffffffffu, rmax[hr], 1));
+            rmax[hr] = fmaxf(rmax[hr], __shfl_xor_sync(0xffffffffu, rmax[hr], 2));
+            const float mnew = fmaxf(mx[hr], rmax[hr]);
+            corr[hr] = mnew == -INFINITY ? 1.f : __expf(mx[hr] - mnew);
+            mx[hr] = mnew;
+            lsum[hr] *= corr[hr];
+        }
+        uint32_t pa[4];
+        {
+            float p[2][4];
+#pragma unroll
+            for (int nb = 0; nb < 2; ++nb)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const float mm = mx[i >> 1];
+                    p[nb][i] = mm == -INFINITY ? 0.f : __expf(s[nb][i] - mm);
+                    lsum[i >> 1] += p[nb][i];
+                }
+            pa[0] = pack_bf16x2(p[0][0], p[0][1]); pa[1] = pack_bf16x2(p[0][2], p[0][3]);
+            pa[2] = pack_bf16x2(p[1][0], p[1][1]); pa[3] = pack_bf16x2(p[1][2], p[1][3]);
+        }
+#pragma unroll
+        for (int i = 0; i < NOT; ++i) { o[i][0] *= corr[0]; o[i][1] *= corr[0]; o[i][2] *= corr[1]; o[i][3] *= corr[1]; }
+        // O += P V: V^T fragments through ldmatrix.trans from the slot.  Lane l gives the row address of
+        // matrix l / 8: keys 0..7 or 8..15 (bit 3 of l), channel tile 0 or 1 of the pair (bit 4 of l).
+        cp_async_wait_all();
+        __syncwarp();
+        const unsigned char *vrow = vslot + ((c.lane & 7) + ((c.lane >> 3) & 1) * 8) * VP + (c.lane >> 4) * 16;
+#pragma unroll
+        for (int np = 0; np < NOT / 2; ++np) {
+            uint32_t vf[4];
+            ldmatrix_x4_trans(vf, vrow + np * 32);
+            mma16816(o[2 * np], pa[0], pa[1], pa[2], pa[3], vf[0], vf[1]);
+            mma16816(o[2 * np + 1], pa[0], pa[1], pa[2], pa[3], vf[2], vf[3]);
+        }
+        __syncwarp();                                    // the slot is read; the next step may overwrite it
+    }
+#pragma unroll
+    for (int hr = 0; hr < 2; ++hr) {
+        lsum[hr] += __shfl_xor_sync(0xffffffffu, lsum[hr], 1);
+        lsum[hr] += __shfl_xor_sync(0xffffffffu, lsum[hr], 2);
+    }
+}
+
+template <int HD>
 __device__ __forceinline__ void attention_item(Ctx &c, const Args &a, int layer, int seq, int h, int split, int nsplit,
                                                int nt_total) {
-    constexpr int hd = 32 * EPL, half = hd / 2, PW = hd + 2;
+    using SM = AttSmem<HD>;
+    constexpr int PW = SM::PW, NOT = HD / 8;
     const DevPtrs &d = a.d;
     const ModelDev &m = a.m;
-    const int H = m.cfg.n_heads, Hkv = m.cfg.n_kv_heads, group = H / Hkv, kh = h / group, qrows = m.qrows;
-    const int n_r = c.n_rows[seq], r_base = seq * a.g.rps;
-    const int pos0 = c.row_pos[r_base];
-    float *qs = reinterpret_cast<float *>(c.scratch);                       // [MAX_ROWS][hd]
-    bf16 *kn = reinterpret_cast<bf16 *>(qs + MAX_ROWS * hd);                // [MAX_ROWS][hd]
-    bf16 *vn = kn + MAX_ROWS * hd;
-    float *red = reinterpret_cast<float *>(vn + MAX_ROWS * hd);             // [ATT_WARPS][ATT_RB][PW]
-    const size_t cbase = (((size_t)layer * d.max_batch + seq) * Hkv + kh) * (size_t)d.max_ctx * hd;
-    const bool writer = split == 0 && h == kh * group;
-    const float scale = rsqrtf((float)hd);
-
-    // rotary embedding of the new rows (rotate-half pairs (i, i + hd/2)); k and v rounded to bf16 as cached
-    for (int i = threadIdx.x; i < n_r * half; i += MMA_THREADS) {
-        const int j = i / half, ii = i - j * half, pos = pos0 + j;
-        const float *row = a.fb.qkv + (size_t)(r_base + j) * qrows;
-        const float2 cs = m.rope[(size_t)pos * half + ii];
-        const float qa = __ldcg(row + h * hd + ii), qb = __ldcg(row + h * hd + ii + half);
-        qs[j * hd + ii] = (qa * cs.x - qb * cs.y) * scale;
-        qs[j * hd + ii + half] = (qb * cs.x + qa * cs.y) * scale;
-        const float ka = __ldcg(row + (H + kh) * hd + ii), kb = __ldcg(row + (H + kh) * hd + ii + half);
-        const bf16 k0 = __float2bfloat16(ka * cs.x - kb * cs.y), k1 = __float2bfloat16(kb * cs.x + ka * cs.y);
-        const bf16 v0 = __float2bfloat16(__ldcg(row + (H + Hkv + kh) * hd + ii));
-        const bf16 v1 = __float2bfloat16(__ldcg(row + (H + Hkv + kh) * hd + ii + half));
-        kn[j * hd + ii] = k0; kn[j * hd + ii + half] = k1;
-        vn[j * hd + ii] = v0; vn[j * hd + ii + half] = v1;
-        if (writer) {
-            bf16 *kc = m.kcache + cbase + (size_t)pos * hd, *vc = m.vcache + cbase + (size_t)pos * hd;
-            kc[ii] = k0; kc[ii + half] = k1;
-            vc[ii] = v0; vc[ii + half] = v1;
-        }
-    }
+    const int H = m.cfg.n_heads, Hkv = m.cfg.n_kv_heads, group = H / Hkv, kh = h / group;
+    const int n_r = c.n_rows[seq], r_base = seq * a.g.rps, pos0 = c.row_pos[r_base];
+    const size_t cbase = (((size_t)layer * d.max_batch + seq) * Hkv + kh) * (size_t)d.max_ctx * HD;
+    attention_rows<HD>(c, a, layer, seq, h, split == 0 && h == kh * group);
     bsync();
 
     const int lo = (int)((long long)pos0 * split / nsplit), hi = (int)((long long)pos0 * (split + 1) / nsplit);
-    const bool with_new = split == nsplit - 1;
-    const bf16 *kc = m.kcache + cbase + c.lane * EPL, *vc = m.vcache + cbase + c.lane * EPL;
-    float *outp = a.fb.attp + (((size_t)(seq * H + h) * MAX_SPLIT + split) * a.g.rps) * PW;
+    const int two = n_r > 16 ? 1 : 0;                    // two query tiles: warps 0..3 take rows 0..15, warps 4..7 rows 16..31
+    const int mt = two ? (c.warp >> 2) : 0, kw = two ? (c.warp & 3) : c.warp, KW = two ? 4 : 8;
+    const int g = c.lane >> 2, t = c.lane & 3;
+    float mx[2] = {-INFINITY, -INFINITY}, lsum[2] = {0.f, 0.f};
+    float o[NOT][4];
+#pragma unroll
+    for (int i = 0; i < NOT; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+    attention_keys<HD>(c, m.kcache + cbase, m.vcache + cbase, lo, hi, split == nsplit - 1 ? n_r : 0, n_r, mt, kw, KW, mx, lsum, o);
 
-    for (int j0 = 0; j0 < n_r; j0 += ATT_RB) {
-        const int nrb = min(ATT_RB, n_r - j0);
-        float mx[ATT_RB], den[ATT_RB], acc[ATT_RB][EPL], qv[ATT_RB][EPL];
+    bsync();                                             // every warp is done with q, the new rows and the slots
+    float *red = reinterpret_cast<float *>(c.scratch);   // [8 warps][16 rows][PW]
+    {
+        float *rw0 = red + ((size_t)c.warp * 16 + g) * PW, *rw1 = rw0 + 8 * PW;
 #pragma unroll
-        for (int jj = 0; jj < ATT_RB; ++jj) {
-            mx[jj] = -INFINITY; den[jj] = 0.f;
-#pragma unroll
-            for (int e = 0; e < EPL; ++e) {
-                acc[jj][e] = 0.f;
-                qv[jj][e] = jj < nrb ? qs[(j0 + jj) * hd + c.lane * EPL + e] : 0.f;
-            }
+        for (int i = 0; i < NOT; ++i) {
+            rw0[i * 8 + 2 * t] = o[i][0]; rw0[i * 8 + 2 * t + 1] = o[i][1];
+            rw1[i * 8 + 2 * t] = o[i][2]; rw1[i * 8 + 2 * t + 1] = o[i][3];
         }
-        auto one_key = [&](const float (&kk)[EPL], const float (&vv)[EPL], int first_row) {
-#pragma unroll
-            for (int jj = 0; jj < ATT_RB; ++jj) {
-                if (jj < nrb && j0 + jj >= first_row) {
-                    float sc = 0.f;
-#pragma unroll
-                    for (int e = 0; e < EPL; ++e) sc += qv[jj][e] * kk[e];
-                    sc = warp_sum(sc);
-                    const float mnew = fmaxf(mx[jj], sc);
-                    const float corr = __expf(mx[jj] - mnew), w = __expf(sc - mnew);
-                    den[jj] = den[jj] * corr + w;
-#pragma unroll
-                    for (int e = 0; e < EPL; ++e) acc[jj][e] = acc[jj][e] * corr + w * vv[e];
-                    mx[jj] = mnew;
-                }
-            }
-        };
-        const bool walker = true;
-        for (int p = lo + c.warp; walker && p < hi; p += ATT_WARPS) {   // cached keys: every new row sees them
-            float kk[EPL], vv[EPL];
-            load_kv_row<EPL>(kc + (size_t)p * hd, kk);
-            load_kv_row<EPL>(vc + (size_t)p * hd, vv);
-            one_key(kk, vv, 0);
+        if (t == 0) { rw0[HD] = mx[0]; rw0[HD + 1] = lsum[0]; rw1[HD] = mx[1]; rw1[HD + 1] = lsum[1]; }
+    }
+    bsync();
+    // merge the warps of each query tile -> the item's partial in global memory
+    float *outp = a.fb.attp + (((size_t)(seq * H + h) * MAX_SPLIT + split) * a.g.rps) * PW;
+    for (int i = threadIdx.x; i < n_r * HD; i += MMA_THREADS) {
+        const int j = i / HD, ch = i - j * HD;
+        const int w0 = two ? (j >> 4) * 4 : 0, rr = j & 15;
+        float M = -INFINITY;
+        for (int w = 0; w < KW; ++w) M = fmaxf(M, red[((size_t)(w0 + w) * 16 + rr) * PW + HD]);
+        float L = 0.f, ov = 0.f;
+        for (int w = 0; w < KW; ++w) {
+            const float *rw = red + ((size_t)(w0 + w) * 16 + rr) * PW;
+            const float f = rw[HD] == -INFINITY ? 0.f : __expf(rw[HD] - M);
+            L += rw[HD + 1] * f;
+            ov += rw[ch] * f;
         }
-        if (with_new && walker) {                                // new keys: row j sees new keys 0..j
-            for (int jn = c.warp; jn < n_r; jn += ATT_WARPS) {
-                float kk[EPL], vv[EPL];
-                load_kv_row<EPL>(kn + jn * hd + c.lane * EPL, kk);
-                load_kv_row<EPL>(vn + jn * hd + c.lane * EPL, vv);
-                one_key(kk, vv, jn);
-            }
-        }
-        // merge the warps' partials of this row block
-#pragma unroll
-        for (int jj = 0; walker && jj < ATT_RB; ++jj) {
-            float *rw = red + ((size_t)c.warp * ATT_RB + jj) * PW;
-#pragma unroll
-            for (int e = 0; e < EPL; ++e) rw[c.lane * EPL + e] = acc[jj][e];
-            if (c.lane == 0) { rw[hd] = mx[jj]; rw[hd + 1] = den[jj]; }
-        }
-        bsync();
-        for (int i = threadIdx.x; i < nrb * hd; i += MMA_THREADS) {
-            const int jj = i / hd, ch = i - jj * hd;
-            float M = -INFINITY;
-#pragma unroll
-            for (int w = 0; w < ATT_WARPS; ++w) M = fmaxf(M, red[((size_t)w * ATT_RB + jj) * PW + hd]);
-            float L = 0.f, o = 0.f;
-#pragma unroll
-            for (int w = 0; w < ATT_WARPS; ++w) {
-                const float *rw = red + ((size_t)w * ATT_RB + jj) * PW;
-                const float f = rw[hd] == -INFINITY ? 0.f : __expf(rw[hd] - M);
-                L += rw[hd + 1] * f;
-                o += rw[ch] * f;
-            }
-            float *op = outp + (size_t)(j0 + jj) * PW;
-            op[ch] = o;
-            if (ch == 0) { op[hd] = M; op[hd + 1] = L; }
-        }
-        bsync();
+        float *op = outp + (size_t)j * PW;
+        op[ch] = ov;
+        if (ch == 0) { op[HD] = M; op[HD + 1] = L; }
     }
 
     // the item that finishes last for (seq, h) merges the splits
@@ -156,19 +246,19 @@ __device__ __forceinline__ void attention_item(Ctx &c, const Args &a, int layer,
     if (c.flag[0]) {
         __threadfence();
         const float *base = a.fb.attp + ((size_t)(seq * H + h) * MAX_SPLIT) * a.g.rps * PW;
-        for (int i = threadIdx.x; i < n_r * hd; i += MMA_THREADS) {
-            const int j = i / hd, ch = i - j * hd;
+        for (int i = threadIdx.x; i < n_r * HD; i += MMA_THREADS) {
+            const int j = i / HD, ch = i - j * HD;
             float M = -INFINITY;
-            for (int sp = 0; sp < nsplit; ++sp) M = fmaxf(M, __ldcg(base + ((size_t)sp * a.g.rps + j) * PW + hd));
-            float L = 0.f, o = 0.f;
+            for (int sp = 0; sp < nsplit; ++sp) M = fmaxf(M, __ldcg(base + ((size_t)sp * a.g.rps + j) * PW + HD));
+            float L = 0.f, ov = 0.f;
             for (int sp = 0; sp < nsplit; ++sp) {
                 const float *pp = base + ((size_t)sp * a.g.rps + j) * PW;
-                const float ms = __ldcg(pp + hd);
+                const float ms = __ldcg(pp + HD);
                 const float f = ms == -INFINITY ? 0.f : __expf(ms - M);
-                L += __ldcg(pp + hd + 1) * f;
-                o += __ldcg(pp + ch) * f;
+                L += __ldcg(pp + HD + 1) * f;
+                ov += __ldcg(pp + ch) * f;
             }
-            d.att[xfrag_index(r_base + j, h * hd + ch, nt_total)] = __float2bfloat16(o / L);
+            d.att[xfrag_index(r_base + j, h * HD + ch, nt_total)] = __float2bfloat16(ov / L);
         }
     }
     bsync();
@@ -186,11 +276,8 @@ __device__ __forceinline__ void phase_attention(Ctx &c, const Args &a, int layer
     for (int it = c.cta; it < items; it += c.ncta) {
         const int split = it % nsplit, sh = it / nsplit, h = sh % H, seq = sh / H;
         if (c.n_rows[seq] == 0) continue;
-        switch (a.m.hd) {
-            case 32: attention_item<1>(c, a, layer, seq, h, split, nsplit, nt_total); break;
-            case 64: attention_item<2>(c, a, layer, seq, h, split, nsplit, nt_total); break;
-            default: attention_item<4>(c, a, layer, seq, h, split, nsplit, nt_total); break;
-        }
+        if (a.m.hd == 64) attention_item<64>(c, a, layer, seq, h, split, nsplit, nt_total);
+        else attention_item<128>(c, a, layer, seq, h, split, nsplit, nt_total);
     }
 }
 

@@ -79,7 +79,7 @@ static bool model_cfg_ok(const pacer_model_cfg &m) {
     if (m.n_layers < 1 || m.d_model < 32 || m.n_heads < 1 || m.n_kv_heads < 1 || m.d_ffn < 32 || m.vocab < 2) return false;
     if (m.d_model % m.n_heads) return false;
     const int hd = m.d_model / m.n_heads;
-    if (hd != 32 && hd != 64 && hd != 128) return false;
+    if (hd != 64 && hd != 128) return false;
     if (m.n_heads % m.n_kv_heads) return false;
     if (m.d_model % 32 || m.d_ffn % 32) return false;
     return true;
