@@ -31,18 +31,19 @@ namespace fwd {
 constexpr int MMA_WARPS = 8, MMA_THREADS = 256;  // warps 0..7: MMAs, epilogues and all block-wide phases
 constexpr int W_PRODUCERS = 4;                   // warps 8..11 stream weights: unit n by producer n % 4 (one warp alone
                                                  // cannot issue the bulk copies fast enough)
-constexpr int X_PRODUCERS = 4;                   // warps 12..15 provide the activation chunks: chunk m by producer m % 4
+constexpr int X_PRODUCERS = 4;                   // warps 12..15 provide the activation chunks: stage s by producer s
 constexpr int W_PRODUCER = MMA_WARPS, X_PRODUCER = W_PRODUCER + W_PRODUCERS;
 constexpr int THREADS = 32 * (X_PRODUCER + X_PRODUCERS);
-constexpr int KC = 256;                         // k columns of one weight unit
+constexpr int KC = 512;                         // k columns of one weight unit: 1 KB per row and copy (DRAM likes long runs)
 constexpr int PITCH = KC * 2 + 64;              // bytes between the rows of a stage (bank-conflict free)
-constexpr int STAGE_BYTES = 16 * PITCH;         // 9216
-constexpr int NS = 16;                          // weight stages in the ring
-constexpr int RING_BYTES = NS * STAGE_BYTES;    // 147456
-constexpr int XS = 4;                           // activation stages
-constexpr int XSTAGE_BYTES = 4 * 4096;          // up to 4 row tiles x 8 chunks x 512 bytes
+constexpr int STAGE_BYTES = 16 * PITCH;         // 17408
+constexpr int NS = 8;                           // weight stages in the ring: one wave of the eight MMA warps
+constexpr int RING_BYTES = NS * STAGE_BYTES;    // 139264
+constexpr int XS_MAX = 4;                       // activation stages: as many as fit the scratch, at most 4
+__host__ __device__ constexpr int xstage_bytes(int NT) { return NT * (KC / 32) * 512; }   // row tiles x chunks x 512 B
+__host__ __device__ constexpr int x_stages(int NT) { return (80 * 1024) / xstage_bytes(NT) < XS_MAX ? (80 * 1024) / xstage_bytes(NT) : XS_MAX; }
 constexpr int SCRATCH_BYTES = 80 * 1024;        // the activation ring lives in its first 48 KB; the attention
-                                                // phase and the tails use all of it (no activations in flight then); XS * XSTAGE_BYTES <= SCRATCH_BYTES
+                                                // phase and the tails use all of it (no activations in flight then)
 constexpr int MISC_BYTES = 2048;
 constexpr int SMEM_BYTES = SCRATCH_BYTES + RING_BYTES + MISC_BYTES;
 constexpr int MAX_TILES = 16;                   // tiles of one pass of a block (two per MMA warp)
@@ -146,7 +147,7 @@ struct Ctx {
     unsigned char *scratch;        // SCRATCH_BYTES (activation ring in front)
     unsigned char *ring;           // weight ring
     uint64_t *wfull, *wempty;      // [NS]
-    uint64_t *xfull, *xempty;      // [XS]
+    uint64_t *xfull, *xempty;      // [XS_MAX]
     int32_t *row_pos, *row_tok;    // [MAX_ROWS]
     int32_t *n_rows;               // [MAX_ROWS] per sequence
     float *inv_rms;                // [MAX_ROWS]

@@ -134,8 +134,8 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
     unsigned char *misc = smem + SCRATCH_BYTES + RING_BYTES;
     c.wfull = reinterpret_cast<uint64_t *>(misc);                            // NS
     c.wempty = c.wfull + NS;                                                 // NS
-    c.xfull = c.wempty + NS;                                                 // XS
-    c.xempty = c.xfull + XS;                                                 // XS  (ends at 8 * (2*NS + 2*XS) = 304)
+    c.xfull = c.wempty + NS;                                                 // XS_MAX
+    c.xempty = c.xfull + XS_MAX;                                             // XS_MAX  (ends at 8 * (2*NS + 2*XS_MAX) <= 320)
     c.row_pos = reinterpret_cast<int32_t *>(misc + 320);
     c.row_tok = c.row_pos + MAX_ROWS;
     c.n_rows = c.row_tok + MAX_ROWS;
@@ -199,7 +199,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
         const unsigned long long v = ld_acquire_u64(a.fb.bar);
         c.bar_target = v / (unsigned long long)c.ncta * (unsigned long long)c.ncta;
         for (int i = 0; i < NS; ++i) { mbar_init(c.wfull + i, 1); mbar_init(c.wempty + i, 1); }
-        for (int i = 0; i < XS; ++i) { mbar_init(c.xfull + i, 1); mbar_init(c.xempty + i, MMA_WARPS); }
+        for (int i = 0; i < XS_MAX; ++i) { mbar_init(c.xfull + i, 1); mbar_init(c.xempty + i, MMA_WARPS); }
         c.ready_op[0] = 0; c.ready_op[1] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }

@@ -101,8 +101,7 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 template <int NT>
 __device__ __forceinline__ void convert_chunk(Ctx &c, const XSrc &xs, const bf16 *gain, int k0, int nch, uint4 *stage,
                                               float (&ss)[NT * 8], bool sum) {
-    const int p = c.lane;                    // 16-byte piece (8 k) of the k step
-    if (p < nch * 4) {
+    for (int p = c.lane; p < nch * 4; p += 32) {            // 16-byte pieces (8 k) of the k step
         const int k = k0 + p * 8;
         const uint4 gw = *reinterpret_cast<const uint4 *>(gain + k);
         const __nv_bfloat162 *g2 = reinterpret_cast<const __nv_bfloat162 *>(&gw);
@@ -151,6 +150,7 @@ __device__ __forceinline__ void convert_chunk(Ctx &c, const XSrc &xs, const bf16
 template <int NT>
 __device__ __forceinline__ void activation_producer(Ctx &c, const FwdBufs &fb, const Plan &P, const XSrc &xs, int me,
                                                     uint64_t keep_policy) {
+    constexpr int XS = x_stages(NT), XSTAGE_BYTES = xstage_bytes(NT);
     int m = 0;
     bool dead = false;                       // a wait gave up: keep walking (the barriers below must be met), do nothing
     for (int q = 0; q < n_ops(P); ++q) {
@@ -169,7 +169,7 @@ __device__ __forceinline__ void activation_producer(Ctx &c, const FwdBufs &fb, c
         for (int r = 0; r < NT * 8; ++r) ss[r] = 0.f;
         for (int p0 = 0; p0 < T; p0 += MAX_TILES) {
             for (int k = k_lo; k < k_hi; k += KC, ++m) {
-                if (m % X_PRODUCERS != me || dead) continue;
+                if (m % XS != me || dead) continue;      // one producer per stage: its generations stay in order
                 const int slot = m % XS, nch = min(KC, k_hi - k) >> 5;
                 if (!wait_bar(fb, c.xempty + slot, (((uint32_t)(m / XS)) & 1u) ^ 1u, 7, m)) { dead = true; continue; }
                 if (normed) {
@@ -248,6 +248,7 @@ __device__ __forceinline__ void gemm_op(Ctx &c, const FwdBufs &fb, const Plan &P
     const bool normed = opi == OP_QKV || opi == OP_GU || opi == OP_HEAD;
     int t0, T, k_lo, k_hi;
     op_range(op, c.cta, c.ncta, t0, T, k_lo, k_hi);
+    constexpr int XS = x_stages(NT), XSTAGE_BYTES = xstage_bytes(NT);
     for (int p0 = 0; p0 < T; p0 += MAX_TILES) {
         const int Tp = min(MAX_TILES, T - p0);
         const bool has0 = c.warp < Tp, has1 = c.warp + MMA_WARPS < Tp;
@@ -261,6 +262,10 @@ __device__ __forceinline__ void gemm_op(Ctx &c, const FwdBufs &fb, const Plan &P
             const int xslot = c.xn % XS;
             wait_bar(fb, c.xfull + xslot, ((uint32_t)(c.xn / XS)) & 1u, 8, c.xn);
             const uint4 *xs = reinterpret_cast<const uint4 *>(c.scratch + xslot * XSTAGE_BYTES);
+            // The units of a k step are consumed in waves of eight (one per MMA warp) with a barrier after each
+            // wave.  A ring stage is shared by different warps over time, and a parity wait is exact only while
+            // the waiter is less than one stage generation ahead: with NS >= 8, unit n - NS lies in an earlier
+            // wave, which the barrier has seen consumed.
             if (has0) {
                 const int n = c.wn + c.warp, slot = n % NS;
                 wait_bar(fb, c.wfull + slot, ((uint32_t)(n / NS)) & 1u, 9, n);
@@ -268,21 +273,20 @@ __device__ __forceinline__ void gemm_op(Ctx &c, const FwdBufs &fb, const Plan &P
                 __syncwarp();
                 if (c.lane == 0) mbar_arrive(c.wempty + slot);
             }
-            if (has1) {
-                const int n = c.wn + c.warp + MMA_WARPS, slot = n % NS;
-                wait_bar(fb, c.wfull + slot, ((uint32_t)(n / NS)) & 1u, 9, n);
-                consume_unit<NT>(c.ring + slot * STAGE_BYTES, xs, nch, acc1, c.lane);
-                __syncwarp();
-                if (c.lane == 0) mbar_arrive(c.wempty + slot);
+            bsync();
+            if (Tp > MMA_WARPS) {
+                if (has1) {
+                    const int n = c.wn + c.warp + MMA_WARPS, slot = n % NS;
+                    wait_bar(fb, c.wfull + slot, ((uint32_t)(n / NS)) & 1u, 9, n);
+                    consume_unit<NT>(c.ring + slot * STAGE_BYTES, xs, nch, acc1, c.lane);
+                    __syncwarp();
+                    if (c.lane == 0) mbar_arrive(c.wempty + slot);
+                }
+                bsync();
             }
-            __syncwarp();
             if (c.lane == 0) mbar_arrive(c.xempty + xslot);
             c.wn += Tp;
             ++c.xn;
-            // Lockstep over k: a ring stage is shared by different warps at different times, and a parity wait
-            // is exact only while the waiter is less than one stage generation ahead.  After this barrier every
-            // unit of the k step is consumed, so the next step's waits (at most MAX_TILES <= NS units on) are exact.
-            bsync();
         }
         if (normed && (has0 || has1)) {
             wait_count(fb, c.ready_op + 1, q + 1, 10);                 // 1/rms of this projection's input rows
