@@ -16,12 +16,10 @@
 //     16-row operand) do the contraction, so the math is invisible;
 //   - the row-wise step that follows a projection in the decoder (residual add,
 //     SwiGLU, bias/arg-max of the LM head) is the epilogue of the warp that owns
-//     the tile; RMSNorm is split: the activation producers multiply x by the
-//     gain while they convert it to bf16 and sum x^2 on the way, and the 1/rms
-//     factor is applied to the OUTPUT rows in the projection's epilogue;
-//   - the two projections with few output columns (attention output, MLP down)
-//     are cut along k as well, and add their partial sums straight into the
-//     fp32 residual stream with fire-and-forget atomic adds;
+//     the tile; RMSNorm is split: the residual epilogue also writes x * gain as
+//     bf16 in fragment order (the next projection's input) and the tile's share
+//     of sum(x^2), and the 1/rms factor is applied to the OUTPUT rows of the
+//     next projection in its epilogue, so no normalisation pass exists;
 //   - phases are separated by grid barriers with bounded waits.
 #pragma once
 #include "common.cuh"
@@ -65,8 +63,7 @@ struct GemmOp {
     int32_t N;               // weight rows in all (gate/up: 2F)
     int32_t MT;              // 16-row tiles
     int32_t K;
-    int32_t S;               // k slices (1, or a divisor of the grid size for the two projections whose outputs
-                             // are ADDED to the residual stream: their partial sums go there with atomic adds)
+    int32_t S;               // k slices (1: every block covers the full k extent of its tiles)
     int32_t rot;             // block that gets the first tile range (spreads the one-tile imbalance)
     int32_t interleave;      // 1: tile t = gate rows 8t..8t+7 then up rows 8t..8t+7
 };
@@ -79,6 +76,8 @@ struct Plan {
 // Device buffers of the forward kernel beyond DevPtrs (all in the workspace).
 struct FwdBufs {
     float *qkv;              // [MAX_ROWS][qrows] fp32
+    bf16 *xg;                // x * gain of the next RMSNorm, bf16 in fragment order (its 1/rms comes later)
+    float *ssq;              // [d/16][MAX_ROWS] sum of squares of x over the 16 columns of a tile
     float *tile_top;         // [MT(head)][MAX_ROWS][4]: max, argmax (int bits), runner-up, unused
     float *attp;             // attention partials [seq*H + h][split][row][hd + 2]
     int32_t *att_cnt;        // [batch * H]

@@ -211,29 +211,25 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
     if (c.warp >= X_PRODUCER) {
         uint64_t keep;
         asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(keep));
-        XSrc xs;
-        xs.xres = d.xres; xs.norm1 = m.norm1; xs.norm2 = m.norm2; xs.normf = m.normf;
-        xs.dm = m.cfg.d_model; xs.rtot = g.rtot; xs.eps = m.cfg.rms_eps;
-        xs.xss = reinterpret_cast<float *>(misc + 1536);                     // [X_PRODUCERS][MAX_ROWS]
-        activation_producer<NT>(c, a.fb, a.P, xs, c.warp - X_PRODUCER, keep);
+        activation_producer<NT>(c, a.fb, a.P, m.cfg.d_model, m.cfg.rms_eps, c.warp - X_PRODUCER, keep);
         return;
     }
 
+    const int dm = m.cfg.d_model;
     int n_stamp = 0;
     auto stamp = [&]() {
         if (a.fb.prof && threadIdx.x == 0 && n_stamp < PROF_STAMPS)
             a.fb.prof[(size_t)c.cta * PROF_STAMPS + n_stamp++] = globaltimer_ns();
     };
     stamp();
-    phase_begin(c, a);
+    phase_begin(c, a, NT);
     stamp();
     grid_barrier(c, a.fb);
     stamp();
 
     const int L = a.P.n_layers;
-    (void)m;
     for (int l = 0; l < L; ++l) {
-        gemm_op<NT>(c, a.fb, a.P, 4 * l + OP_QKV, [&](int tile, float (&acc)[NT][4]) { epi_qkv<NT>(c, a, tile, acc); });
+        gemm_op<NT>(c, a.fb, a.P, 4 * l + OP_QKV, nullptr, 0, [&](int tile, float (&acc)[NT][4]) { epi_qkv<NT>(c, a, tile, acc); });
         stamp();
         grid_barrier(c, a.fb);
         stamp();
@@ -241,21 +237,24 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
         stamp();
         grid_barrier(c, a.fb);
         stamp();
-        gemm_op<NT>(c, a.fb, a.P, 4 * l + OP_O, [&](int tile, float (&acc)[NT][4]) { epi_residual<NT>(c, a, tile, acc); });
+        gemm_op<NT>(c, a.fb, a.P, 4 * l + OP_O, d.xres, dm,
+                    [&](int tile, float (&acc)[NT][4]) { epi_residual<NT>(c, a, m.norm2 + (size_t)l * dm, tile, acc); });
         stamp();
         grid_barrier(c, a.fb);
         stamp();
-        gemm_op<NT>(c, a.fb, a.P, 4 * l + OP_GU, [&](int tile, float (&acc)[NT][4]) { epi_swiglu<NT>(c, a, tile, acc); });
+        gemm_op<NT>(c, a.fb, a.P, 4 * l + OP_GU, nullptr, 0, [&](int tile, float (&acc)[NT][4]) { epi_swiglu<NT>(c, a, tile, acc); });
         stamp();
         grid_barrier(c, a.fb);
         stamp();
-        gemm_op<NT>(c, a.fb, a.P, 4 * l + OP_DOWN, [&](int tile, float (&acc)[NT][4]) { epi_residual<NT>(c, a, tile, acc); });
+        const bf16 *gain_next = l + 1 < L ? m.norm1 + (size_t)(l + 1) * dm : m.normf;
+        gemm_op<NT>(c, a.fb, a.P, 4 * l + OP_DOWN, d.xres, dm,
+                    [&](int tile, float (&acc)[NT][4]) { epi_residual<NT>(c, a, gain_next, tile, acc); });
         stamp();
         grid_barrier(c, a.fb);
         stamp();
     }
     if (a.P.has_head) {
-        gemm_op<NT>(c, a.fb, a.P, 4 * L,
+        gemm_op<NT>(c, a.fb, a.P, 4 * L, nullptr, 0,
                     [&](int tile, float (&acc)[NT][4]) { epi_head<NT>(c, a, row_dst, bias_at, tile, acc); });
         stamp();
         grid_barrier(c, a.fb);
@@ -291,21 +290,15 @@ static inline Plan make_plan(const ModelDev &m, const DevPtrs &d, const FwdBufs 
     auto set = [&](int i, const bf16 *w1, const bf16 *w2, const bf16 *x, long long lstride, int N, int K, int MT, int inter) {
         GemmOp &o = P.op[i];
         o.W1 = w1; o.W2 = w2 ? w2 : w1; o.X = x; o.lstride = lstride; o.N = N; o.K = K; o.MT = MT; o.interleave = inter;
-        // the projections that add into the residual stream are also cut along k when they have few tiles
         o.S = 1;
-        if (i == OP_O || i == OP_DOWN) {
-            const int nks = (K + KC - 1) / KC;
-            for (int sdiv = 2; sdiv <= 8; ++sdiv)
-                if (ncta % sdiv == 0 && sdiv <= nks && MT * (sdiv / 2) < 4 * ncta) o.S = sdiv;
-        }
         o.rot = rot;
         rot = (rot + (MT % (ncta / o.S)) * o.S) % ncta;       // the next projection's extra tiles go to other blocks
     };
-    set(OP_QKV, m.wqkv, nullptr, nullptr, (long long)m.qrows * dm, m.qrows, (int)dm, (m.qrows + 15) / 16, 0);
+    set(OP_QKV, m.wqkv, nullptr, fb.xg, (long long)m.qrows * dm, m.qrows, (int)dm, (m.qrows + 15) / 16, 0);
     set(OP_O, m.wo, nullptr, d.att, dm * hh, (int)dm, (int)hh, ((int)dm + 15) / 16, 0);
-    set(OP_GU, m.wgate, m.wup, nullptr, F * dm, (int)(2 * F), (int)dm, ((int)F + 7) / 8, 1);
+    set(OP_GU, m.wgate, m.wup, fb.xg, F * dm, (int)(2 * F), (int)dm, ((int)F + 7) / 8, 1);
     set(OP_DOWN, m.wdown, nullptr, d.act, dm * F, (int)dm, (int)F, ((int)dm + 15) / 16, 0);
-    set(OP_HEAD, m.head, nullptr, nullptr, 0, k.vocab, (int)dm, (k.vocab + 15) / 16, 0);
+    set(OP_HEAD, m.head, nullptr, fb.xg, 0, k.vocab, (int)dm, (k.vocab + 15) / 16, 0);
     P.n_layers = k.n_layers;
     P.has_head = has_head ? 1 : 0;
     return P;

@@ -69,26 +69,39 @@ __device__ __forceinline__ RowDesc row_desc(int kind, const DevPtrs &d, int s, i
 // ------------------------------------------------------------------ input rows
 
 // x = embedding row (or h + e for the pre-verification model, or the draft's
-// hidden row during its prefill), spread over the MMA warps of the grid.
-__device__ __forceinline__ void phase_begin(Ctx &c, const Args &a) {
+// hidden row during its prefill), spread over the MMA warps of the grid by
+// 16-column tiles.  Leaves x (fp32), x * gain of the first RMSNorm (bf16,
+// fragment order) and the per-tile sums of squares.
+__device__ __forceinline__ void phase_begin(Ctx &c, const Args &a, int nt_total) {
     const DevPtrs &d = a.d;
     const ModelDev &m = a.m;
-    const int dm = m.cfg.d_model, per_row = dm >> 5;           // 32 columns per warp task
-    for (int task = c.cta * MMA_WARPS + c.warp; task < a.g.rtot * per_row; task += c.ncta * MMA_WARPS) {
-        const int r = task / per_row, col = (task - r * per_row) * 32 + c.lane;
-        if (c.row_pos[r] < 0) continue;
-        const int s = r / a.g.rps, j = r - s * a.g.rps;
-        float v;
-        if (a.kind == KIND_MB) {
-            v = d.hpend[((size_t)s * (d.block_b + 1) + j) * dm + col];
-            const int e = c.row_tok[r];
-            if (e > 0 && d.use_posemb) v += __bfloat162float(m.posemb[(size_t)(e - 1) * dm + col]);
-        } else if (a.kind == KIND_PREFILL_B) {
-            v = __ldcg(d.hidden + (size_t)r * dm + col);
-        } else {
-            v = __bfloat162float(m.embed[(size_t)c.row_tok[r] * dm + col]);
+    const int dm = m.cfg.d_model, ntiles = dm >> 4, rpad = nt_total * 8;
+    const int half = c.lane >> 4, col16 = c.lane & 15;
+    for (int tile = c.cta * MMA_WARPS + c.warp; tile < ntiles; tile += c.ncta * MMA_WARPS) {
+        const int col = tile * 16 + col16;
+        const float gain = __bfloat162float(m.norm1[col]);
+        for (int rr = 0; rr < rpad; rr += 2) {
+            const int r = rr + half;
+            float v = 0.f;
+            if (r < a.g.rtot && c.row_pos[r] >= 0) {
+                const int s = r / a.g.rps, j = r - s * a.g.rps;
+                if (a.kind == KIND_MB) {
+                    v = d.hpend[((size_t)s * (d.block_b + 1) + j) * dm + col];
+                    const int e = c.row_tok[r];
+                    if (e > 0 && d.use_posemb) v += __bfloat162float(m.posemb[(size_t)(e - 1) * dm + col]);
+                } else if (a.kind == KIND_PREFILL_B) {
+                    v = __ldcg(d.hidden + (size_t)r * dm + col);
+                } else {
+                    v = __bfloat162float(m.embed[(size_t)c.row_tok[r] * dm + col]);
+                }
+            }
+            d.xres[(size_t)r * dm + col] = v;          // idle rows hold zeros: they stay finite through the layers
+            a.fb.xg[xfrag_index(r, col, nt_total)] = __float2bfloat16(v * gain);
+            float ss = v * v;
+#pragma unroll
+            for (int o = 8; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+            if (col16 == 0) a.fb.ssq[tile * MAX_ROWS + r] = ss;
         }
-        d.xres[(size_t)r * dm + col] = v;
     }
 }
 
@@ -110,24 +123,43 @@ __device__ __forceinline__ void epi_qkv(Ctx &c, const Args &a, int tile, float (
     }
 }
 
-// Tile of the attention-output / down projection (one k slice of it): added to
-// the fp32 residual stream with atomic adds that return nothing, so the warp
-// never waits for them.
+// Tile of the attention-output / down projection.  The accumulators started from
+// the residual rows, so they hold the new x: store it, store x * gain of the
+// RMSNorm that follows as bf16 in fragment order (the next projection's input),
+// and the tile's share of sum(x^2) per row.
 template <int NT>
-__device__ __forceinline__ void epi_residual(Ctx &c, const Args &a, int tile, float (&acc)[NT][4]) {
+__device__ __forceinline__ void epi_residual(Ctx &c, const Args &a, const bf16 *gain_next, int tile, float (&acc)[NT][4]) {
     const int g = c.lane >> 2, t = c.lane & 3, dm = a.m.cfg.d_model;
     const int n0 = tile * 16 + g, n1 = n0 + 8;
+    const float g0 = n0 < dm ? __bfloat162float(gain_next[n0]) : 0.f, g1 = n1 < dm ? __bfloat162float(gain_next[n1]) : 0.f;
 #pragma unroll
-    for (int nt = 0; nt < NT; ++nt)
+    for (int nt = 0; nt < NT; ++nt) {
+        float ss[2] = {0.f, 0.f};
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
             const int r = nt * 8 + 2 * t + i;
-            if (r < a.g.rtot && c.row_pos[r] >= 0) {
-                float *x = a.d.xres + (size_t)r * dm;
-                if (n0 < dm) atomicAdd(x + n0, acc[nt][i]);
-                if (n1 < dm) atomicAdd(x + n1, acc[nt][2 + i]);
+            float *x = a.d.xres + (size_t)r * dm;
+            if (n0 < dm) {
+                const float v = acc[nt][i];
+                x[n0] = v; ss[i] += v * v;
+                a.fb.xg[xfrag_index(r, n0, NT)] = __float2bfloat16(v * g0);
+            }
+            if (n1 < dm) {
+                const float v = acc[nt][2 + i];
+                x[n1] = v; ss[i] += v * v;
+                a.fb.xg[xfrag_index(r, n1, NT)] = __float2bfloat16(v * g1);
             }
         }
+#pragma unroll
+        for (int o = 4; o < 32; o <<= 1) {
+            ss[0] += __shfl_xor_sync(0xffffffffu, ss[0], o);
+            ss[1] += __shfl_xor_sync(0xffffffffu, ss[1], o);
+        }
+        if (g == 0) {
+            a.fb.ssq[tile * MAX_ROWS + nt * 8 + 2 * t] = ss[0];
+            a.fb.ssq[tile * MAX_ROWS + nt * 8 + 2 * t + 1] = ss[1];
+        }
+    }
 }
 
 // Interleaved gate/up tile: rows 0..7 are gate rows f = 8*tile + g, rows 8..15 the

@@ -81,130 +81,70 @@ __device__ __forceinline__ void weight_producer(Ctx &c, const FwdBufs &fb, const
     }
 }
 
-// What the activation producers read.
-struct XSrc {
-    const float *xres;                       // fp32 residual stream [row][d]
-    const bf16 *norm1, *norm2, *normf;       // RMSNorm gains
-    int32_t dm, rtot;
-    float eps;
-    float *xss;                              // shared: [X_PRODUCERS][MAX_ROWS] partial sums of x^2
-};
-
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t *>(&v);
 }
 
-// One k step of RMSNorm's input side: x * gain as bf16 in fragment order
-// [chunk of 32 k][row tile][lane = (r % 8) * 4 + (k % 32) / 8] x 8 values, written
-// into an activation stage by one warp; ss[r] gathers this lane's share of sum(x_r^2).
-template <int NT>
-__device__ __forceinline__ void convert_chunk(Ctx &c, const XSrc &xs, const bf16 *gain, int k0, int nch, uint4 *stage,
-                                              float (&ss)[NT * 8], bool sum) {
-    for (int p = c.lane; p < nch * 4; p += 32) {            // 16-byte pieces (8 k) of the k step
-        const int k = k0 + p * 8;
-        const uint4 gw = *reinterpret_cast<const uint4 *>(gain + k);
-        const __nv_bfloat162 *g2 = reinterpret_cast<const __nv_bfloat162 *>(&gw);
-        const float2 ga = __bfloat1622float2(g2[0]), gb = __bfloat1622float2(g2[1]);
-        const float2 gc = __bfloat1622float2(g2[2]), gd = __bfloat1622float2(g2[3]);
-        constexpr int RB = 8;                // rows whose loads are issued together (one round trip per group)
-#pragma unroll
-        for (int r0 = 0; r0 < NT * 8; r0 += RB) {
-            float4 xa[RB], xb[RB];
-            bool act[RB];
-#pragma unroll
-            for (int j = 0; j < RB; ++j) {
-                const int r = r0 + j;
-                act[j] = r < xs.rtot && c.row_pos[r] >= 0;                             // the same in every lane
-                if (act[j]) {
-                    const float *src = xs.xres + (size_t)r * xs.dm + k;
-                    xa[j] = __ldcg(reinterpret_cast<const float4 *>(src));
-                    xb[j] = __ldcg(reinterpret_cast<const float4 *>(src + 4));
-                }
-            }
-#pragma unroll
-            for (int j = 0; j < RB; ++j) {
-                const int r = r0 + j;
-                uint4 out = make_uint4(0u, 0u, 0u, 0u);
-                if (act[j]) {
-                    const float4 x0 = xa[j], x1 = xb[j];
-                    out.x = pack_bf16x2(x0.x * ga.x, x0.y * ga.y);
-                    out.y = pack_bf16x2(x0.z * gb.x, x0.w * gb.y);
-                    out.z = pack_bf16x2(x1.x * gc.x, x1.y * gc.y);
-                    out.w = pack_bf16x2(x1.z * gd.x, x1.w * gd.y);
-                    if (sum)
-                        ss[r] += (x0.x * x0.x + x0.y * x0.y) + (x0.z * x0.z + x0.w * x0.w) + (x1.x * x1.x + x1.y * x1.y) +
-                                 (x1.z * x1.z + x1.w * x1.w);
-                }
-                stage[((p >> 2) * NT + (r >> 3)) * 32 + ((r & 7) << 2) + (p & 3)] = out;
-            }
-        }
+// inv_rms[r] = 1 / sqrt(mean(x_r^2) + eps) from the per-tile sums ssq[tile][row], in a fixed
+// order (one warp, lane = row; four running sums keep the loads independent).
+__device__ __forceinline__ void compute_inv(Ctx &c, const FwdBufs &fb, int dm, float eps) {
+    const int ntiles = dm >> 4;
+    const float *p = fb.ssq + c.lane;
+    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+    int t = 0;
+    for (; t + 4 <= ntiles; t += 4) {
+        s0 += __ldcg(p + (t + 0) * MAX_ROWS);
+        s1 += __ldcg(p + (t + 1) * MAX_ROWS);
+        s2 += __ldcg(p + (t + 2) * MAX_ROWS);
+        s3 += __ldcg(p + (t + 3) * MAX_ROWS);
     }
+    for (; t < ntiles; ++t) s0 += __ldcg(p + t * MAX_ROWS);
+    c.inv_rms[c.lane] = rsqrtf(((s0 + s1) + (s2 + s3)) / (float)dm + eps);
+    __syncwarp();
 }
 
 // Warps X_PRODUCER ..: the activation chunk of every k step, once the projection's
-// inputs are complete (the MMA warps raise ready_op[0] after the grid barrier).
-// Projections that follow an RMSNorm get x * gain converted on the fly, and the
-// producers leave 1/rms per row for the epilogues (ready_op[1]); the others get a
-// bulk copy of a bf16 buffer that already has fragment order.
+// inputs are complete (the MMA warps raise ready_op[0] after the grid barrier): a
+// bulk copy of a bf16 buffer that already has fragment order.  Stage s is fed by
+// producer s, so its generations stay in order.  The last producer warp computes
+// 1/rms per row for the projections that follow an RMSNorm (ready_op[1]).
 template <int NT>
-__device__ __forceinline__ void activation_producer(Ctx &c, const FwdBufs &fb, const Plan &P, const XSrc &xs, int me,
+__device__ __forceinline__ void activation_producer(Ctx &c, const FwdBufs &fb, const Plan &P, int dm, float eps, int me,
                                                     uint64_t keep_policy) {
     constexpr int XS = x_stages(NT), XSTAGE_BYTES = xstage_bytes(NT);
     int m = 0;
-    bool dead = false;                       // a wait gave up: keep walking (the barriers below must be met), do nothing
     for (int q = 0; q < n_ops(P); ++q) {
-        const int opi = op_index(P, q), layer = op_layer(P, q);
+        const int opi = op_index(P, q);
         const GemmOp &op = P.op[opi];
         const bool normed = opi == OP_QKV || opi == OP_GU || opi == OP_HEAD;
-        const bf16 *gain = opi == OP_QKV ? xs.norm1 + (size_t)layer * xs.dm : opi == OP_GU ? xs.norm2 + (size_t)layer * xs.dm : xs.normf;
         int t0, T, k_lo, k_hi;
         op_range(op, c.cta, c.ncta, t0, T, k_lo, k_hi);
         if (T == 0) continue;
         wait_count(fb, c.ready_op, q + 1, 6);
         __threadfence_block();
         asm volatile("fence.proxy.async;" ::: "memory");
-        float ss[NT * 8];
-#pragma unroll
-        for (int r = 0; r < NT * 8; ++r) ss[r] = 0.f;
+        if (me == X_PRODUCERS - 1) {
+            if (normed) {
+                compute_inv(c, fb, dm, eps);
+                __threadfence_block();
+                if (c.lane == 0) c.ready_op[1] = q + 1;
+                __syncwarp();
+            }
+            if (me >= XS) { for (int p0 = 0; p0 < T; p0 += MAX_TILES) for (int k = k_lo; k < k_hi; k += KC) ++m; continue; }
+        }
         for (int p0 = 0; p0 < T; p0 += MAX_TILES) {
             for (int k = k_lo; k < k_hi; k += KC, ++m) {
-                if (m % XS != me || dead) continue;      // one producer per stage: its generations stay in order
+                if (m % XS != me) continue;
                 const int slot = m % XS, nch = min(KC, k_hi - k) >> 5;
-                if (!wait_bar(fb, c.xempty + slot, (((uint32_t)(m / XS)) & 1u) ^ 1u, 7, m)) { dead = true; continue; }
-                if (normed) {
-                    convert_chunk<NT>(c, xs, gain, k, nch, reinterpret_cast<uint4 *>(c.scratch + slot * XSTAGE_BYTES), ss, p0 == 0);
-                    __syncwarp();
-                    if (c.lane == 0) mbar_arrive(c.xfull + slot);
-                } else if (c.lane == 0) {
+                if (!wait_bar(fb, c.xempty + slot, (((uint32_t)(m / XS)) & 1u) ^ 1u, 7, m)) return;
+                if (c.lane == 0) {
                     const uint32_t bytes = (uint32_t)nch * (uint32_t)NT * 512u;
                     mbar_expect_tx(c.xfull + slot, bytes);
                     bulk_g2s(c.scratch + slot * XSTAGE_BYTES, op.X + (size_t)(k >> 5) * NT * 256, bytes, c.xfull + slot,
                              keep_policy);
                 }
                 __syncwarp();
-            }
-            if (normed && p0 == 0) {         // 1/rms per row from the four producers' shares, in a fixed order
-#pragma unroll
-                for (int r = 0; r < NT * 8; ++r) {
-                    float v = ss[r];
-#pragma unroll
-                    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-                    if (c.lane == 0) xs.xss[me * MAX_ROWS + r] = v;
-                }
-                asm volatile("bar.sync 2, 128;" ::: "memory");
-                if (me == 0) {
-                    if (c.lane < NT * 8) {
-                        float v = 0.f;
-#pragma unroll
-                        for (int j = 0; j < X_PRODUCERS; ++j) v += xs.xss[j * MAX_ROWS + c.lane];
-                        c.inv_rms[c.lane] = rsqrtf(v / (float)xs.dm + xs.eps);
-                    }
-                    __syncwarp();
-                    __threadfence_block();
-                    if (c.lane == 0) c.ready_op[1] = q + 1;
-                }
-                asm volatile("bar.sync 2, 128;" ::: "memory");
             }
         }
     }
@@ -238,7 +178,8 @@ __device__ __forceinline__ void consume_unit(const unsigned char *stage, const u
 // full k extent; epi(tile, acc) gets the complete sums.
 // Accumulator element (nt, i): token row nt*8 + 2t + (i & 1), tile column g + 8*(i >> 1).
 template <int NT, class Epi>
-__device__ __forceinline__ void gemm_op(Ctx &c, const FwdBufs &fb, const Plan &P, int q, Epi epi) {
+__device__ __forceinline__ void gemm_op(Ctx &c, const FwdBufs &fb, const Plan &P, int q, const float *resid, int resid_ld,
+                                        Epi epi) {
     const GemmOp &op = P.op[op_index(P, q)];
     if (threadIdx.x == 0) {
         __threadfence_block();
@@ -252,11 +193,24 @@ __device__ __forceinline__ void gemm_op(Ctx &c, const FwdBufs &fb, const Plan &P
     for (int p0 = 0; p0 < T; p0 += MAX_TILES) {
         const int Tp = min(MAX_TILES, T - p0);
         const bool has0 = c.warp < Tp, has1 = c.warp + MMA_WARPS < Tp;
+        // Accumulators start from the residual rows when the projection adds into the residual stream: the
+        // loads are issued before the k loop, so the epilogue has no global round trip of its own.
         float acc0[NT][4], acc1[NT][4];
+        {
+            const int g = c.lane >> 2, t = c.lane & 3;
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt)
+            for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-            for (int i = 0; i < 4; ++i) acc0[nt][i] = acc1[nt][i] = 0.f;
+                for (int i = 0; i < 4; ++i) {
+                    acc0[nt][i] = acc1[nt][i] = 0.f;
+                    if (resid) {
+                        const int r = nt * 8 + 2 * t + (i & 1);
+                        const int n0 = (t0 + p0 + c.warp) * 16 + g + 8 * (i >> 1), n1 = n0 + MMA_WARPS * 16;
+                        if (has0 && n0 < op.N) acc0[nt][i] = __ldcg(resid + (size_t)r * resid_ld + n0);
+                        if (has1 && n1 < op.N) acc1[nt][i] = __ldcg(resid + (size_t)r * resid_ld + n1);
+                    }
+                }
+        }
         for (int k = k_lo; k < k_hi; k += KC) {
             const int nch = min(KC, k_hi - k) >> 5;
             const int xslot = c.xn % XS;

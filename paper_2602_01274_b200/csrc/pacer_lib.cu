@@ -242,7 +242,7 @@ extern "C" int pacer_create(const pacer_cfg *cfg, void *dev_workspace, size_t wo
     d.row_arg = (int32_t *)(w + L.row_arg); d.row_margin = (float *)(w + L.row_margin);
     d.xres = (float *)(w + L.xres); d.xn = nullptr; d.att = (bf16 *)(w + L.att); d.act = (bf16 *)(w + L.act);
     d.q = nullptr; d.hidden = (float *)(w + L.hidden); d.part = (float *)(w + L.part);
-    c->fb.qkv = (float *)(w + L.qkv);
+    c->fb.qkv = (float *)(w + L.qkv); c->fb.xg = (bf16 *)(w + L.xg); c->fb.ssq = (float *)(w + L.ssq);
     c->fb.tile_top = (float *)(w + L.tile_top); c->fb.attp = (float *)(w + L.attp);
     c->fb.att_cnt = (int32_t *)(w + L.att_cnt); c->fb.bar = (unsigned long long *)(w + L.bar);
     c->fb.abort_flag = (int32_t *)(w + L.abort_flag);
