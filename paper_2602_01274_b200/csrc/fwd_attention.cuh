@@ -4,9 +4,9 @@
 // Inside an item the eight MMA warps split the keys in steps of 16 (and the two
 // 16-row query tiles when there are more than 16 rows); every warp keeps a
 // running (max, sum, output) per row, FlashAttention style.  The warps' results
-// are merged through shared memory into the item's partial, and the item that
-// finishes last for a (sequence, head) merges the splits and writes the bf16
-// attention output in the fragment order the output projection reads.
+// are merged through shared memory into the item's partial; after a grid barrier
+// the splits of every (sequence, head, row) are merged by one warp each into the
+// bf16 attention output, in the fragment order the output projection reads.
 #pragma once
 #include "fwd_phases.cuh"
 
@@ -215,7 +215,8 @@ __device__ __forceinline__ void attention_item(Ctx &c, const Args &a, int layer,
         if (t == 0) { rw0[HD] = mx[0]; rw0[HD + 1] = lsum[0]; rw1[HD] = mx[1]; rw1[HD + 1] = lsum[1]; }
     }
     bsync();
-    // merge the warps of each query tile -> the item's partial in global memory
+    // merge the warps of each query tile -> the item's partial in global memory; with a single split the
+    // result is final and goes straight to the output projection's input buffer
     float *outp = a.fb.attp + (((size_t)(seq * H + h) * MAX_SPLIT + split) * a.g.rps) * PW;
     for (int i = threadIdx.x; i < n_r * HD; i += MMA_THREADS) {
         const int j = i / HD, ch = i - j * HD;
@@ -229,49 +230,59 @@ __device__ __forceinline__ void attention_item(Ctx &c, const Args &a, int layer,
             L += rw[HD + 1] * f;
             ov += rw[ch] * f;
         }
-        float *op = outp + (size_t)j * PW;
-        op[ch] = ov;
-        if (ch == 0) { op[HD] = M; op[HD + 1] = L; }
-    }
-
-    // the item that finishes last for (seq, h) merges the splits
-    __threadfence();
-    bsync();
-    if (threadIdx.x == 0) {
-        const int old = atomicAdd(a.fb.att_cnt + seq * H + h, 1);
-        c.flag[0] = old == nsplit - 1;
-        if (old == nsplit - 1) a.fb.att_cnt[seq * H + h] = 0;
-    }
-    bsync();
-    if (c.flag[0]) {
-        __threadfence();
-        const float *base = a.fb.attp + ((size_t)(seq * H + h) * MAX_SPLIT) * a.g.rps * PW;
-        for (int i = threadIdx.x; i < n_r * HD; i += MMA_THREADS) {
-            const int j = i / HD, ch = i - j * HD;
-            float M = -INFINITY;
-            for (int sp = 0; sp < nsplit; ++sp) M = fmaxf(M, __ldcg(base + ((size_t)sp * a.g.rps + j) * PW + HD));
-            float L = 0.f, ov = 0.f;
-            for (int sp = 0; sp < nsplit; ++sp) {
-                const float *pp = base + ((size_t)sp * a.g.rps + j) * PW;
-                const float ms = __ldcg(pp + HD);
-                const float f = ms == -INFINITY ? 0.f : __expf(ms - M);
-                L += __ldcg(pp + HD + 1) * f;
-                ov += __ldcg(pp + ch) * f;
-            }
+        if (nsplit == 1) {
             d.att[xfrag_index(r_base + j, h * HD + ch, nt_total)] = __float2bfloat16(ov / L);
+        } else {
+            float *op = outp + (size_t)j * PW;
+            op[ch] = ov;
+            if (ch == 0) { op[HD] = M; op[HD + 1] = L; }
         }
     }
     bsync();
 }
 
-// All blocks: the attention of one layer.
-__device__ __forceinline__ void phase_attention(Ctx &c, const Args &a, int layer, int nt_total) {
-    const int H = a.m.cfg.n_heads, batch = a.g.batch;
+// Key-range splits of a head in this forward (the same value in every block).
+__device__ __forceinline__ int attention_splits(const Ctx &c, const Args &a) {
     int lmax = 0;
-    for (int s = 0; s < batch; ++s)
+    for (int s = 0; s < a.g.batch; ++s)
         if (c.n_rows[s] > 0) lmax = max(lmax, c.row_pos[s * a.g.rps]);
-    int nsplit = c.ncta / (batch * H);
-    nsplit = max(1, min(nsplit, min(MAX_SPLIT, lmax / 64)));
+    const int nsplit = c.ncta / (a.g.batch * a.m.cfg.n_heads);
+    return max(1, min(nsplit, min(MAX_SPLIT, lmax / 64)));
+}
+
+// All blocks, after the grid barrier that follows the items: the splits of every
+// (sequence, head, row) merged by one warp each, into the bf16 attention output in
+// the fragment order the output projection reads.
+__device__ __forceinline__ void phase_attention_merge(Ctx &c, const Args &a, int nsplit, int nt_total) {
+    const int H = a.m.cfg.n_heads, hd = a.m.hd, PW = hd + 2, rps = a.g.rps;
+    const int tasks = a.g.batch * H * rps;
+    for (int task = c.cta * MMA_WARPS + c.warp; task < tasks; task += c.ncta * MMA_WARPS) {
+        const int j = task % rps, sh = task / rps, h = sh % H, seq = sh / H;
+        if (j >= c.n_rows[seq]) continue;
+        const float *base = a.fb.attp + ((size_t)(seq * H + h) * MAX_SPLIT * rps + j) * PW;
+        float M = -INFINITY;
+        for (int sp = 0; sp < nsplit; ++sp) M = fmaxf(M, __ldcg(base + (size_t)sp * rps * PW + hd));
+        float L = 0.f, ov[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int sp = 0; sp < nsplit; ++sp) {
+            const float *pp = base + (size_t)sp * rps * PW;
+            const float ms = __ldcg(pp + hd);
+            const float f = ms == -INFINITY ? 0.f : __expf(ms - M);
+            L += __ldcg(pp + hd + 1) * f;
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+                if (c.lane + 32 * e < hd) ov[e] += __ldcg(pp + c.lane + 32 * e) * f;
+        }
+        const float inv = 1.f / L;
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+            if (c.lane + 32 * e < hd)
+                a.d.att[xfrag_index(seq * rps + j, h * hd + c.lane + 32 * e, nt_total)] = __float2bfloat16(ov[e] * inv);
+    }
+}
+
+// All blocks: the attention items of one layer.
+__device__ __forceinline__ void phase_attention(Ctx &c, const Args &a, int layer, int nsplit, int nt_total) {
+    const int H = a.m.cfg.n_heads, batch = a.g.batch;
     const int items = batch * H * nsplit;
     for (int it = c.cta; it < items; it += c.ncta) {
         const int split = it % nsplit, sh = it / nsplit, h = sh % H, seq = sh / H;

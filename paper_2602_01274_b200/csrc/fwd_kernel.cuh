@@ -233,9 +233,14 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
         stamp();
         grid_barrier(c, a.fb);
         stamp();
-        phase_attention(c, a, l, NT);
+        const int nsplit = attention_splits(c, a);
+        phase_attention(c, a, l, nsplit, NT);
         stamp();
         grid_barrier(c, a.fb);
+        if (nsplit > 1) {                       // the same decision in every block
+            phase_attention_merge(c, a, nsplit, NT);
+            grid_barrier(c, a.fb);
+        }
         stamp();
         gemm_op<NT>(c, a.fb, a.P, 4 * l + OP_O, d.xres, dm,
                     [&](int tile, float (&acc)[NT][4]) { epi_residual<NT>(c, a, m.norm2 + (size_t)l * dm, tile, acc); });
