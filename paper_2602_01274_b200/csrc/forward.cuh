@@ -63,7 +63,8 @@ struct GemmOp {
     int32_t N;               // weight rows in all (gate/up: 2F)
     int32_t MT;              // 16-row tiles
     int32_t K;
-    int32_t S;               // k slices (1: every block covers the full k extent of its tiles)
+    int32_t S;               // k slices: 1, or (attention output / MLP down, which have few tiles) a divisor of the
+                             // grid size: the slices' partial tiles are summed by a small pass after a grid barrier
     int32_t rot;             // block that gets the first tile range (spreads the one-tile imbalance)
     int32_t interleave;      // 1: tile t = gate rows 8t..8t+7 then up rows 8t..8t+7
 };
@@ -78,6 +79,7 @@ struct FwdBufs {
     float *qkv;              // [MAX_ROWS][qrows] fp32
     bf16 *xg;                // x * gain of the next RMSNorm, bf16 in fragment order (its 1/rms comes later)
     float *ssq;              // [d/16][MAX_ROWS] sum of squares of x over the 16 columns of a tile
+    float *part;             // k-slice partial tiles [S][d/16][row tiles * 8][16] of the two residual projections
     float *tile_top;         // [MT(head)][MAX_ROWS][4]: max, argmax (int bits), runner-up, unused
     float *attp;             // attention partials [seq*H + h][split][row][hd + 2]
     int32_t *att_cnt;        // [batch * H]
@@ -177,6 +179,13 @@ __device__ __host__ __forceinline__ void op_range(const GemmOp &op, int cta, int
     k_hi = k_lo + (sb + (s < sr ? 1 : 0)) * KC;
     if (k_hi > op.K) k_hi = op.K;
     if (k_lo >= k_hi) T = 0;
+}
+
+// k slice of block `cta` in a sliced projection.
+__device__ __host__ __forceinline__ int op_slice(const GemmOp &op, int cta, int ncta) {
+    int ci = cta - op.rot;
+    if (ci < 0) ci += ncta;
+    return ci % op.S;
 }
 
 // Grid barrier (MMA warps only): every block arrives once; waits are bounded.  A wait that runs

@@ -242,21 +242,48 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
             grid_barrier(c, a.fb);
         }
         stamp();
-        gemm_op<NT>(c, a.fb, a.P, 4 * l + OP_O, d.xres, dm,
-                    [&](int tile, float (&acc)[NT][4]) { epi_residual<NT>(c, a, m.norm2 + (size_t)l * dm, tile, acc); });
-        stamp();
-        grid_barrier(c, a.fb);
-        stamp();
+        {
+            const GemmOp &op = a.P.op[OP_O];
+            const bf16 *gain_next = m.norm2 + (size_t)l * dm;
+            if (op.S == 1) {
+                gemm_op<NT>(c, a.fb, a.P, 4 * l + OP_O, d.xres, dm,
+                            [&](int tile, float (&acc)[NT][4]) { epi_residual<NT>(c, a, gain_next, tile, acc); });
+            } else {
+                const int slice = op_slice(op, c.cta, c.ncta);
+                gemm_op<NT>(c, a.fb, a.P, 4 * l + OP_O, nullptr, 0,
+                            [&](int tile, float (&acc)[NT][4]) { epi_partial<NT>(c, a, op, slice, tile, acc); });
+            }
+            stamp();
+            grid_barrier(c, a.fb);
+            if (op.S > 1) {
+                phase_residual<NT>(c, a, op, gain_next);
+                grid_barrier(c, a.fb);
+            }
+            stamp();
+        }
         gemm_op<NT>(c, a.fb, a.P, 4 * l + OP_GU, nullptr, 0, [&](int tile, float (&acc)[NT][4]) { epi_swiglu<NT>(c, a, tile, acc); });
         stamp();
         grid_barrier(c, a.fb);
         stamp();
-        const bf16 *gain_next = l + 1 < L ? m.norm1 + (size_t)(l + 1) * dm : m.normf;
-        gemm_op<NT>(c, a.fb, a.P, 4 * l + OP_DOWN, d.xres, dm,
-                    [&](int tile, float (&acc)[NT][4]) { epi_residual<NT>(c, a, gain_next, tile, acc); });
-        stamp();
-        grid_barrier(c, a.fb);
-        stamp();
+        {
+            const GemmOp &op = a.P.op[OP_DOWN];
+            const bf16 *gain_next = l + 1 < L ? m.norm1 + (size_t)(l + 1) * dm : m.normf;
+            if (op.S == 1) {
+                gemm_op<NT>(c, a.fb, a.P, 4 * l + OP_DOWN, d.xres, dm,
+                            [&](int tile, float (&acc)[NT][4]) { epi_residual<NT>(c, a, gain_next, tile, acc); });
+            } else {
+                const int slice = op_slice(op, c.cta, c.ncta);
+                gemm_op<NT>(c, a.fb, a.P, 4 * l + OP_DOWN, nullptr, 0,
+                            [&](int tile, float (&acc)[NT][4]) { epi_partial<NT>(c, a, op, slice, tile, acc); });
+            }
+            stamp();
+            grid_barrier(c, a.fb);
+            if (op.S > 1) {
+                phase_residual<NT>(c, a, op, gain_next);
+                grid_barrier(c, a.fb);
+            }
+            stamp();
+        }
     }
     if (a.P.has_head) {
         gemm_op<NT>(c, a.fb, a.P, 4 * L, nullptr, 0,
@@ -296,6 +323,11 @@ static inline Plan make_plan(const ModelDev &m, const DevPtrs &d, const FwdBufs 
         GemmOp &o = P.op[i];
         o.W1 = w1; o.W2 = w2 ? w2 : w1; o.X = x; o.lstride = lstride; o.N = N; o.K = K; o.MT = MT; o.interleave = inter;
         o.S = 1;
+        if (i == OP_O || i == OP_DOWN) {      // few tiles: also cut along k, so that a block needs less of the activations
+            const int nks = (K + KC - 1) / KC;
+            for (int sdiv = 2; sdiv <= 8; ++sdiv)
+                if (ncta % sdiv == 0 && sdiv <= nks && MT * (sdiv / 2) < 4 * ncta) o.S = sdiv;
+        }
         o.rot = rot;
         rot = (rot + (MT % (ncta / o.S)) * o.S) % ncta;       // the next projection's extra tiles go to other blocks
     };

@@ -162,6 +162,62 @@ __device__ __forceinline__ void epi_residual(Ctx &c, const Args &a, const bf16 *
     }
 }
 
+// One k slice of a residual-projection tile: stored as a partial, nothing waits for it.
+template <int NT>
+__device__ __forceinline__ void epi_partial(Ctx &c, const Args &a, const GemmOp &op, int slice, int tile, float (&acc)[NT][4]) {
+    const int g = c.lane >> 2, t = c.lane & 3;
+    float *mine = a.fb.part + ((size_t)slice * op.MT + tile) * (NT * 8 * 16);
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+        const int r0 = nt * 8 + 2 * t;
+        mine[r0 * 16 + g] = acc[nt][0];
+        mine[(r0 + 1) * 16 + g] = acc[nt][1];
+        mine[r0 * 16 + g + 8] = acc[nt][2];
+        mine[(r0 + 1) * 16 + g + 8] = acc[nt][3];
+    }
+}
+
+// After the grid barrier that completes the partials of a k-sliced residual
+// projection: x += the slices' sums (slice order, so the result does not depend
+// on timing); x * gain of the next RMSNorm as bf16 fragments; sum(x^2) per tile.
+// Spread over the MMA warps of the grid by 16-column tiles.
+template <int NT>
+__device__ __forceinline__ void phase_residual(Ctx &c, const Args &a, const GemmOp &op, const bf16 *gain_next) {
+    constexpr int RPAD = NT * 8, NIT = RPAD / 2;
+    const int dm = a.m.cfg.d_model, ntiles = dm >> 4;
+    const int half = c.lane >> 4, col16 = c.lane & 15;
+    for (int tile = c.cta * MMA_WARPS + c.warp; tile < ntiles; tile += c.ncta * MMA_WARPS) {
+        const int col = tile * 16 + col16;
+        const float gain = __bfloat162float(gain_next[col]);
+        float v[NIT];
+#pragma unroll
+        for (int it = 0; it < NIT; ++it) v[it] = __ldcg(a.d.xres + (size_t)(2 * it + half) * dm + col);
+        for (int s0 = 0; s0 < op.S; s0 += 4) {          // four slices' loads in flight together
+            float p[4][NIT];
+#pragma unroll
+            for (int ds = 0; ds < 4; ++ds)
+#pragma unroll
+                for (int it = 0; it < NIT; ++it)
+                    p[ds][it] = s0 + ds < op.S
+                        ? __ldcg(a.fb.part + (((size_t)(s0 + ds) * op.MT + tile) * RPAD + 2 * it + half) * 16 + col16) : 0.f;
+#pragma unroll
+            for (int ds = 0; ds < 4; ++ds)              // slice order: the sum does not depend on timing
+#pragma unroll
+                for (int it = 0; it < NIT; ++it) v[it] += p[ds][it];
+        }
+#pragma unroll
+        for (int it = 0; it < NIT; ++it) {
+            const int r = 2 * it + half;
+            a.d.xres[(size_t)r * dm + col] = v[it];
+            a.fb.xg[xfrag_index(r, col, NT)] = __float2bfloat16(v[it] * gain);
+            float ss = v[it] * v[it];
+#pragma unroll
+            for (int o = 8; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+            if (col16 == 0) a.fb.ssq[tile * MAX_ROWS + r] = ss;
+        }
+    }
+}
+
 // Interleaved gate/up tile: rows 0..7 are gate rows f = 8*tile + g, rows 8..15 the
 // up rows of the same f, so a lane holds both; 1/rms of the input RMSNorm, then
 // silu(gate) * up as bf16 in the fragment order the down projection reads.

@@ -180,7 +180,7 @@ static Layout make_layout(const pacer_cfg &c) {
     L.ssq = cv.take(sizeof(float) * fwd::MAX_ROWS * (d_max / 16 + 1));
     L.tile_top = cv.take(sizeof(float) * 4 * fwd::MAX_ROWS * ((size_t)V / 16 + 1));
     L.attp = cv.take(sizeof(float) * (size_t)B * h_max * fwd::MAX_SPLIT * rps_max * (hd_max + 2));
-    L.part_bytes = 256;
+    L.part_bytes = sizeof(float) * 8 * (size_t)d_max * fwd::MAX_ROWS;      // up to 8 k slices of [d/16][32][16]
     L.part = cv.take(L.part_bytes);
     for (int i = 0; i < 3; ++i) {
         const int hd = ms[i]->d_model / ms[i]->n_heads;
@@ -243,6 +243,7 @@ extern "C" int pacer_create(const pacer_cfg *cfg, void *dev_workspace, size_t wo
     d.xres = (float *)(w + L.xres); d.xn = nullptr; d.att = (bf16 *)(w + L.att); d.act = (bf16 *)(w + L.act);
     d.q = nullptr; d.hidden = (float *)(w + L.hidden); d.part = (float *)(w + L.part);
     c->fb.qkv = (float *)(w + L.qkv); c->fb.xg = (bf16 *)(w + L.xg); c->fb.ssq = (float *)(w + L.ssq);
+    c->fb.part = (float *)(w + L.part);
     c->fb.tile_top = (float *)(w + L.tile_top); c->fb.attp = (float *)(w + L.attp);
     c->fb.att_cnt = (int32_t *)(w + L.att_cnt); c->fb.bar = (unsigned long long *)(w + L.bar);
     c->fb.abort_flag = (int32_t *)(w + L.abort_flag);
