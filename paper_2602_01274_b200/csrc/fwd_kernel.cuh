@@ -5,6 +5,7 @@
 #include <vector>
 
 #include "fwd_attention.cuh"
+#include "sampling.cuh"
 
 namespace fwd {
 
@@ -35,6 +36,10 @@ __device__ __forceinline__ void tail_draft(Ctx &c, const Args &a, int s) {
     const int n_in = c.n_rows[s], dm = a.m.cfg.d_model;
     if (n_in == 0) return;
     const int gamma = st.gamma, n_pend = st.n_pend, r_last = s * a.g.rps + n_in - 1;
+    int y_new = 0;
+    if (st.mode == PACER_SAMPLE)                          // y_i ~ q_i by the Gumbel-max rule at the token's position
+        y_new = gumbel_argmax(d.draft_logits + ((size_t)s * d.gamma_cap + gamma) * a.m.cfg.vocab, a.m.cfg.vocab, st.seed,
+                              st.P + gamma, s, TAG_DRAFT, MMA_THREADS, reinterpret_cast<BestD *>(c.scratch), true);
     for (int jj = 0; jj < n_in; ++jj) {
         float *dst = d.hpend + ((size_t)s * (d.block_b + 1) + n_pend + jj) * dm;
         for (int i = threadIdx.x; i < dm; i += MMA_THREADS) dst[i] = hidden_at(a, c, s * a.g.rps + jj, i);
@@ -43,7 +48,7 @@ __device__ __forceinline__ void tail_draft(Ctx &c, const Args &a, int s) {
     if (threadIdx.x == 0) {
         for (int jj = 0; jj < n_in; ++jj)
             d.hpend_e[s * (d.block_b + 1) + n_pend + jj] = (jj == n_in - 1) ? gamma + 1 : 0;
-        d.y[(size_t)s * d.gamma_cap + gamma] = d.row_arg[r_last];
+        d.y[(size_t)s * d.gamma_cap + gamma] = st.mode == PACER_SAMPLE ? y_new : d.row_arg[r_last];
         st.n_pend = n_pend + n_in;
         st.gamma = gamma + 1;
         st.len_D += n_in;
@@ -111,10 +116,15 @@ __device__ __forceinline__ void tail_prefill(Ctx &c, const Args &a, int s, int w
 
 // End of one autoregressive target step (Eq. 1).
 __device__ __forceinline__ void tail_ar(Ctx &c, const Args &a, int s) {
-    if (c.n_rows[s] == 0 || threadIdx.x != 0) return;
+    if (c.n_rows[s] == 0) return;
     const DevPtrs &d = a.d;
     SeqState &st = d.st[s];
-    d.x[(size_t)s * d.max_ctx + st.P] = d.row_arg[s * a.g.rps];
+    int tok = d.row_arg[s * a.g.rps];
+    if (st.mode == PACER_SAMPLE)
+        tok = gumbel_argmax(d.verify_logits + (size_t)s * (d.gamma_cap + 1) * a.m.cfg.vocab, a.m.cfg.vocab, st.seed, st.P, s,
+                            TAG_NEXT, MMA_THREADS, reinterpret_cast<BestD *>(c.scratch), true);
+    if (threadIdx.x != 0) return;
+    d.x[(size_t)s * d.max_ctx + st.P] = tok;
     st.P += 1;
     st.len_T += 1;
     st.n_target_fwd += 1;

@@ -29,6 +29,7 @@ struct pacer_ctx {
     std::map<int, fwd::Plan> plans;   // key: which * 2 + has_head
     unsigned long long *prof_stamps;
     int batch;                 // sequences of the current run
+    int mode;                  // PACER_GREEDY / PACER_SAMPLE of the current run
     int prefilled;
     int64_t launches;
     cudaEvent_t ev[4];
@@ -409,12 +410,12 @@ static int start_run(pacer_ctx *c, const int32_t *prompt, int batch, int n_promp
     if (gm < k.block_b || gm > k.gamma_cap) return fail(c, PACER_EINVAL, "prefill: gamma_max outside [block_b, gamma_cap]");
     if ((int64_t)n_prompt + max_new + k.gamma_cap + 2 > k.max_ctx) return fail(c, PACER_EINVAL, "prefill: n_prompt + max_new + gamma_cap + 2 exceeds max_ctx");
     if (mode != PACER_GREEDY && mode != PACER_SAMPLE) return fail(c, PACER_EINVAL, "prefill: bad mode");
-    if (mode == PACER_SAMPLE) return fail(c, PACER_EUNSUPPORTED, "sampling mode is not built yet");
     for (int s = 0; s < batch; ++s)
         for (int i = 0; i < n_prompt; ++i)
             if (prompt[(size_t)s * n_prompt + i] < 0 || prompt[(size_t)s * n_prompt + i] >= k.target.vocab)
                 return fail(c, PACER_EINVAL, "prefill: token id out of range");
     set_geoms(c, batch);
+    c->mode = mode;
     std::vector<SeqState> hs(k.max_batch);
     memset(hs.data(), 0, sizeof(SeqState) * hs.size());
     for (int s = 0; s < batch; ++s) {
@@ -477,7 +478,8 @@ extern "C" int pacer_verify(pacer_ctx *c) {
 extern "C" int pacer_accept_rollback(pacer_ctx *c) {
     int rc = need_ready(c, true);
     if (rc) return rc;
-    k_accept_greedy<<<1, 64, 0, c->stream>>>(c->d, c->g_verify);
+    if (c->mode == PACER_SAMPLE) k_accept_sample<<<c->batch, ACCEPT_THREADS, 0, c->stream>>>(c->d, c->g_verify, c->cfg.target.vocab);
+    else k_accept_greedy<<<1, 64, 0, c->stream>>>(c->d, c->g_verify);
     LAUNCH_CHECK();
     return PACER_OK;
 }

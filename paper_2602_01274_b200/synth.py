@@ -242,16 +242,16 @@ def make_prompts(vocab: int, batch: int, n_prompt: int, seed: int = 0) -> torch.
 
 
 def make_pair(cfg: PairConfig, seed: int = 0, device="cpu",
-              which=("target", "draft", "preverify")) -> Dict[str, Optional[dict]]:
+              which=("target", "draft", "preverify"), std: float = 0.02) -> Dict[str, Optional[dict]]:
     """Weights of the requested models of a pair plus the successor tables."""
     out: Dict[str, Optional[dict]] = {}
     if "target" in which:
-        out["target"] = make_model(cfg.target, "target", seed, device)
+        out["target"] = make_model(cfg.target, "target", seed, device, std=std)
     if "draft" in which:
-        out["draft"] = make_model(cfg.draft, "draft", seed, device)
+        out["draft"] = make_model(cfg.draft, "draft", seed, device, std=std)
     if "preverify" in which:
         out["preverify"] = make_model(preverify_shape(cfg.draft), "preverify", seed, device,
-                                      gamma_cap=cfg.gamma_cap)
+                                      gamma_cap=cfg.gamma_cap, std=std)
     st, sd = make_succ_tables(cfg.target.vocab, cfg.agree, seed, device)
     out["succ_T"], out["succ_D"] = st, sd
     return out
