@@ -172,6 +172,7 @@ def main():
     ap.add_argument("--impl", default="pacer", choices=["pacer", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-sample-new", type=int, default=4)
+    ap.add_argument("--sample", action="store_true", help="temperature-1 rejection sampling (Philox seed 1) instead of greedy")
     ap.add_argument("--only", default="all", choices=["all", "verify"],
                     help="verify: short prefill, one full draft window, then timed verify forwards only "
                          "(the small, few-launch command the ncu captures use)")
@@ -190,9 +191,10 @@ def main():
     t0 = PACER_T0
     workload = {"workload": f"{cfg.name}: target {cfg.target.n_layers}L d={cfg.target.d_model}, draft "
                             f"{cfg.draft.n_layers}L d={cfg.draft.d_model}, prompt {cfg.n_prompt}, new {cfg.max_new}, "
-                            f"gamma_max {cfg.gamma_max}, b {cfg.block_b}, rho {cfg.rho}, t0 {t0}, greedy, batch 1",
+                            f"gamma_max {cfg.gamma_max}, b {cfg.block_b}, rho {cfg.rho}, t0 {t0}, "
+                            f"{'sampling T=1 seed 1' if args.sample else 'greedy'}, batch 1",
                 "weights": "N(0,0.02) seed 0, planted successor bias +8, agreement %.2f" % cfg.agree,
-                "l2": "inputs (13.2 GB of weights per forward) exceed L2; no flush needed"}
+                "l2": "inputs (%.1f GB of weights per forward) exceed L2; no flush needed" % (cfg.target.streamed_weight_bytes() / 1e9)}
 
     if args.impl == "reference":
         if rank != 0:
@@ -243,8 +245,9 @@ def main():
                                                                                              args.warmup)}))
         return
 
+    mode, seed = (b.PACER_SAMPLE, 1) if args.sample else (b.PACER_GREEDY, 0)
     for _ in range(args.warmup):
-        ctx.pacer_generate(prompt, cfg.max_new, cfg.gamma_max, t0)
+        ctx.pacer_generate(prompt, cfg.max_new, cfg.gamma_max, t0, mode, seed)
     sampler = ClockSampler(local_rank)
     barrier()
     sampler.start()
@@ -253,7 +256,7 @@ def main():
     wall0 = time.perf_counter()
     for _ in range(args.steps):
         ts = time.perf_counter()
-        toks, ns, dl, al, st = ctx.pacer_generate(prompt, cfg.max_new, cfg.gamma_max, t0)
+        toks, ns, dl, al, st = ctx.pacer_generate(prompt, cfg.max_new, cfg.gamma_max, t0, mode, seed)
         torch.cuda.synchronize()
         e2e_s += time.perf_counter() - ts
         dec_ms += st["ms_decode"]; tok += cfg.max_new; launches += st["n_kernel_launches"]
@@ -263,12 +266,21 @@ def main():
     clocks = sampler.stop()
 
     # baselines on the same kernels (outside the timed region): autoregressive and fixed windows
-    ar_tok, ar_st = ctx.pacer_generate_ar(prompt, cfg.max_new)
+    ar_tok, ar_st = ctx.pacer_generate_ar(prompt, cfg.max_new, mode, seed)
     ar_tps = cfg.max_new / (ar_st["ms_decode"] * 1e-3)
-    lossless = bool((ar_tok[0] == toks[0]).all())
+    lossless = None if args.sample else bool((ar_tok[0] == toks[0]).all())
+    mismatch = None
+    if lossless is False:
+        # greedy outputs may part ways only where the target's two best logits tie within the tolerance: show the tie
+        i = int(np.nonzero(ar_tok[0] != toks[0])[0][0])
+        ctx.pacer_generate_ar(prompt, i + 1)
+        lg = ctx.pacer_read_buffer(b.BUF_VERIFY_LOGITS, np.float32, cfg.target.vocab)
+        top = np.argsort(lg)[-2:][::-1]
+        mismatch = {"new_token_index": i, "ar_top2_logits": [float(lg[top[0]]), float(lg[top[1]])],
+                    "ar_top2_margin": float(lg[top[0]] - lg[top[1]]), "tolerance": 2e-2}
     fixed = {}
     for g in range(cfg.block_b, cfg.gamma_cap + 1, cfg.block_b):
-        _, _, _, _, s2 = ctx.pacer_generate(prompt, cfg.max_new, g, -1.0)
+        _, _, _, _, s2 = ctx.pacer_generate(prompt, cfg.max_new, g, -1.0, mode, seed)
         fixed[g] = cfg.max_new / (s2["ms_decode"] * 1e-3)
     best_g = max(fixed, key=fixed.get)
 
@@ -303,7 +315,8 @@ def main():
                     "speedup_vs_best_fixed": value / fixed[best_g], "tau": float(al.mean()),
                     "mean_gamma": float(dl.mean()), "steps": int(ns), "n_draft_fwd": st["n_draft_fwd"],
                     "n_mb_calls": st["n_mb_calls"], "n_target_fwd": st["n_target_fwd"],
-                    "ms_prefill": st["ms_prefill"], "lossless_vs_gpu_ar": lossless},
+                    "ms_prefill": st["ms_prefill"], "lossless_vs_gpu_ar": lossless,
+                    "first_mismatch_vs_gpu_ar": mismatch},
            "wall_s_timed_region": wall}
     if not args.no_cpu_baseline:
         try:
