@@ -333,7 +333,9 @@ static inline Plan make_plan(const ModelDev &m, const DevPtrs &d, const FwdBufs 
         GemmOp &o = P.op[i];
         o.W1 = w1; o.W2 = w2 ? w2 : w1; o.X = x; o.lstride = lstride; o.N = N; o.K = K; o.MT = MT; o.interleave = inter;
         o.S = 1;
-        if (i == OP_O || i == OP_DOWN) {      // few tiles: also cut along k, so that a block needs less of the activations
+        // few tiles and enough bytes to be bandwidth bound: also cut along k, so that a block needs less of the
+        // activations (a small projection is latency bound and better off without the extra pass and barrier)
+        if ((i == OP_O || i == OP_DOWN) && (long long)N * K * 2 >= (16ll << 20)) {
             const int nks = (K + KC - 1) / KC;
             for (int sdiv = 2; sdiv <= 8; ++sdiv)
                 if (ncta % sdiv == 0 && sdiv <= nks && MT * (sdiv / 2) < 4 * ncta) o.S = sdiv;
