@@ -116,7 +116,7 @@ enum {
     PACER_BUF_VCACHE_T = 9,      /* bf16  same shape                        (also _D = 11, _B = 13) */
     PACER_BUF_KCACHE_D = 10, PACER_BUF_VCACHE_D = 11, PACER_BUF_KCACHE_B = 12, PACER_BUF_VCACHE_B = 13,
     PACER_BUF_PHASE_NS = 14      /* u64 [256 blocks][512] device clock (ns) at the phase boundaries of the last
-                                    profiled target forward, per block: start, input rows, barrier, then per
+                                    forward run while profiling (any model), per block: start, input rows, barrier, then per
                                     layer QKV, barrier, attention, barrier, O, barrier, gate/up, barrier, down,
                                     barrier; LM head, barrier; end (at most 512 stamps are kept) */
 };
@@ -206,8 +206,8 @@ int pacer_generate_ar(pacer_ctx *ctx, const int32_t *prompt, int batch, int n_pr
  * pacer_profile_end every forward of the TARGET model (one launch of the
  * persistent forward kernel) is bracketed by a pair of CUDA events on the
  * context's stream (at most 4096 launches are recorded; later ones run untimed)
- * and every block of the kernel stamps the device clock at its phase boundaries
- * (PACER_BUF_PHASE_NS).  pacer_profile_end [sync] returns the summed device time
+ * and every block of every forward (any model) stamps the device clock at its phase
+ * boundaries (PACER_BUF_PHASE_NS keeps the last forward's).  pacer_profile_end [sync] returns the summed device time
  * of those launches (ms), the bf16 weight bytes they streamed and their count.
  * Whole-loop timings are taken without it. */
 int pacer_profile_begin(pacer_ctx *ctx);

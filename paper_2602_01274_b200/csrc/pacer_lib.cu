@@ -378,7 +378,7 @@ static int run_forward(pacer_ctx *c, int which, const Geom &g, int kind, int aux
     if (it == c->plans.end()) it = c->plans.emplace(key, fwd::make_plan(m, c->d, c->fb, c->ncta, head)).first;
     fwd::Args a;
     a.d = c->d; a.m = m; a.g = g; a.P = it->second; a.fb = c->fb; a.kind = kind; a.aux = aux;
-    a.fb.prof = (c->prof_on && which == PACER_TARGET && c->ncta <= fwd::PROF_BLOCKS) ? c->prof_stamps : nullptr;
+    a.fb.prof = (c->prof_on && c->ncta <= fwd::PROF_BLOCKS) ? c->prof_stamps : nullptr;
     const bool prof = c->prof_on && which == PACER_TARGET && c->prof_used + 2 <= c->prof_ev.size();
     if (prof) CK(cudaEventRecord(c->prof_ev[c->prof_used], c->stream));
     CK(fwd::launch(a, which, c->ncta, c->stream));
