@@ -159,6 +159,19 @@ def verify_forward_numbers(ctx, cfg, prompt, n_ver, n_warm):
     return {"roofline": roofline, "verify_forward": verify}
 
 
+def aggregate_replicas(dec_ms: float, e2e_s: float, tokens: float, steps: int, world: int, device="cpu"):
+    """Whole-job numbers of `world` independent replicas (the path does not shard: no data-path collective):
+    tokens summed over ranks, divided by the slowest rank's time.  Returns (tokens/s device-timed, tokens/s end to
+    end, ms per step).  Only this reporting step talks between ranks (one MAX and one SUM all-reduce)."""
+    if world <= 1:
+        return tokens / (dec_ms * 1e-3), tokens / e2e_s, dec_ms / steps
+    import torch.distributed as dist
+    t = torch.tensor([dec_ms, e2e_s, float(tokens)], device=device, dtype=torch.float64)
+    mx = t.clone(); dist.all_reduce(mx, op=dist.ReduceOp.MAX)
+    sm = t.clone(); dist.all_reduce(sm, op=dist.ReduceOp.SUM)
+    return sm[2].item() / (mx[0].item() * 1e-3), sm[2].item() / mx[1].item(), mx[0].item() / steps
+
+
 def pair_to_cpu(pair):
     return {k: ({n: t.cpu() for n, t in v.items()} if isinstance(v, dict) else v.cpu()) for k, v in pair.items()}
 
@@ -287,17 +300,7 @@ def main():
     vf = verify_forward_numbers(ctx, cfg, prompt, 10, 3)
     roofline, verify = vf["roofline"], vf["verify_forward"]
 
-    val_local = tok / (dec_ms * 1e-3)
-    e2e_local = tok / e2e_s
-    if world > 1:
-        t = torch.tensor([dec_ms, e2e_s, float(tok)], device=dev, dtype=torch.float64)
-        mx = t.clone(); dist.all_reduce(mx, op=dist.ReduceOp.MAX)
-        sm = t.clone(); dist.all_reduce(sm, op=dist.ReduceOp.SUM)
-        value = sm[2].item() / (mx[0].item() * 1e-3)
-        e2e_val = sm[2].item() / mx[1].item()
-        ms_step = mx[0].item() / args.steps
-    else:
-        value, e2e_val, ms_step = val_local, e2e_local, dec_ms / args.steps
+    value, e2e_val, ms_step = aggregate_replicas(dec_ms, e2e_s, tok, args.steps, world, dev)
     if rank != 0:
         return
 
