@@ -29,7 +29,8 @@ namespace fwd {
 constexpr int MMA_WARPS = 8, MMA_THREADS = 256;  // warps 0..7: MMAs, epilogues and all block-wide phases
 constexpr int W_PRODUCERS = 4;                   // warps 8..11 stream weights: unit n by producer n % 4 (one warp alone
                                                  // cannot issue the bulk copies fast enough)
-constexpr int X_PRODUCERS = 4;                   // warps 12..15 provide the activation chunks: stage s by producer s
+constexpr int X_PRODUCERS = 4;                   // warps 12..14 provide the activation chunks (stage s by producer s); warp 15
+                                                 // computes the RMS statistics
 constexpr int W_PRODUCER = MMA_WARPS, X_PRODUCER = W_PRODUCER + W_PRODUCERS;
 constexpr int THREADS = 32 * (X_PRODUCER + X_PRODUCERS);
 constexpr int KC = 512;                         // k columns of one weight unit: 1 KB per row and copy (DRAM likes long runs)
@@ -37,14 +38,14 @@ constexpr int PITCH = KC * 2 + 64;              // bytes between the rows of a s
 constexpr int STAGE_BYTES = 16 * PITCH;         // 17408
 constexpr int NS = 8;                           // weight stages in the ring: one wave of the eight MMA warps
 constexpr int RING_BYTES = NS * STAGE_BYTES;    // 139264
-constexpr int XS_MAX = 4;                       // activation stages: as many as fit the scratch, at most 4
+constexpr int XS_MAX = 3;                       // activation stages: as many as fit the scratch, at most 3 (one producer warp each)
 __host__ __device__ constexpr int xstage_bytes(int NT) { return NT * (KC / 32) * 512; }   // row tiles x chunks x 512 B
 __host__ __device__ constexpr int x_stages(int NT) { return (80 * 1024) / xstage_bytes(NT) < XS_MAX ? (80 * 1024) / xstage_bytes(NT) : XS_MAX; }
 constexpr int SCRATCH_BYTES = 80 * 1024;        // the activation ring lives in its first 48 KB; the attention
                                                 // phase and the tails use all of it (no activations in flight then)
 constexpr int MISC_BYTES = 2048;
 constexpr int SMEM_BYTES = SCRATCH_BYTES + RING_BYTES + MISC_BYTES;
-constexpr int MAX_TILES = 16;                   // tiles of one pass of a block (two per MMA warp)
+constexpr int MAX_TILES = 8;                    // tiles of one pass of a block: one per MMA warp, one ring generation per k step
 constexpr int MAX_ROWS = 32;                    // rows of one forward (all sequences together)
 constexpr int MAX_SPLIT = 16;                   // key-range splits of one attention head
 constexpr unsigned SPIN_LIMIT = 1u << 22;        // polls of a global word or a shared counter
@@ -55,7 +56,7 @@ constexpr int PROF_BLOCKS = 256;              // blocks the stamp buffer has roo
 enum OpKind { OP_QKV = 0, OP_O = 1, OP_GU = 2, OP_DOWN = 3, OP_HEAD = 4, N_OPS = 5 };
 
 // One weight-streaming projection.  Block c owns the contiguous tiles
-// [t0, t0 + T) given by tile_range(); it runs them in passes of MAX_TILES.
+// [t0, t0 + T) given by op_range(); it runs them in passes of at most MAX_TILES, evenly sized.
 struct GemmOp {
     const bf16 *W1, *W2;     // layer-0 base; W2 only for the interleaved gate/up projection
     const bf16 *X;           // activations, bf16 in fragment order [K/32][row tiles][32 lanes][8]
@@ -179,6 +180,15 @@ __device__ __host__ __forceinline__ void op_range(const GemmOp &op, int cta, int
     k_hi = k_lo + (sb + (s < sr ? 1 : 0)) * KC;
     if (k_hi > op.K) k_hi = op.K;
     if (k_lo >= k_hi) T = 0;
+}
+
+// Passes of a block over its T tiles: as few as possible, evenly sized (the activations are streamed
+// once per pass, and an even split keeps every pass bandwidth bound rather than latency bound).
+__device__ __host__ __forceinline__ int n_passes(int T) { return (T + MAX_TILES - 1) / MAX_TILES; }
+__device__ __host__ __forceinline__ void pass_range(int T, int p, int &p0, int &Tp) {
+    const int np = n_passes(T), base = T / np, rem = T % np;
+    Tp = base + (p < rem ? 1 : 0);
+    p0 = p * base + (p < rem ? p : rem);
 }
 
 // k slice of block `cta` in a sliced projection.

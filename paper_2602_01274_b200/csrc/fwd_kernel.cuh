@@ -218,10 +218,11 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
 
     // the two producer warps live in their streams until the forward's last unit
     if (c.warp >= W_PRODUCER && c.warp < X_PRODUCER) { weight_producer(c, a.fb, a.P, c.warp - W_PRODUCER); return; }
+    if (c.warp == X_PRODUCER + X_PRODUCERS - 1) { helper_warp(c, a.fb, a.P, m.cfg.d_model, m.cfg.rms_eps); return; }
     if (c.warp >= X_PRODUCER) {
         uint64_t keep;
         asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(keep));
-        activation_producer<NT>(c, a.fb, a.P, m.cfg.d_model, m.cfg.rms_eps, c.warp - X_PRODUCER, keep);
+        activation_producer<NT>(c, a.fb, a.P, c.warp - X_PRODUCER, keep);
         return;
     }
 

@@ -3,7 +3,7 @@
 //
 // Order of everything, identical on both sides: projections q = 0, 1, ... of the
 // forward (four per layer, then the LM head); inside a projection the passes of
-// this block (at most MAX_TILES tiles each); inside a pass the k steps of KC
+// this block (at most MAX_TILES tiles each, evenly sized); inside a pass the k steps of KC
 // columns; inside a k step the tiles of the pass.  Weight unit number n of the
 // block lives in ring stage n % NS, activation chunk number m in stage m % XS.
 #pragma once
@@ -54,8 +54,9 @@ __device__ __forceinline__ void weight_producer(Ctx &c, const FwdBufs &fb, const
         const size_t lbase = (size_t)op_layer(P, q) * op.lstride;
         int t0, T, k_lo, k_hi;
         op_range(op, c.cta, c.ncta, t0, T, k_lo, k_hi);
-        for (int p0 = 0; p0 < T; p0 += MAX_TILES) {
-            const int Tp = min(MAX_TILES, T - p0);
+        for (int p = 0; p < n_passes(T); ++p) {
+            int p0, Tp;
+            pass_range(T, p, p0, Tp);
             for (int k = k_lo; k < k_hi; k += KC) {
                 const uint32_t bytes = (uint32_t)min(KC, k_hi - k) * 2u;
                 for (int i = 0; i < Tp; ++i, ++n) {
@@ -104,36 +105,24 @@ __device__ __forceinline__ void compute_inv(Ctx &c, const FwdBufs &fb, int dm, f
     __syncwarp();
 }
 
-// Warps X_PRODUCER ..: the activation chunk of every k step, once the projection's
-// inputs are complete (the MMA warps raise ready_op[0] after the grid barrier): a
-// bulk copy of a bf16 buffer that already has fragment order.  Stage s is fed by
-// producer s, so its generations stay in order.  The last producer warp computes
-// 1/rms per row for the projections that follow an RMSNorm (ready_op[1]).
+// Warps X_PRODUCER .. X_PRODUCER + XS - 1: the activation chunk of every k step,
+// once the projection's inputs are complete (the MMA warps raise ready_op[0] after
+// the grid barrier): a bulk copy of a bf16 buffer that already has fragment order.
+// Stage s is fed by producer s, so its generations stay in order.
 template <int NT>
-__device__ __forceinline__ void activation_producer(Ctx &c, const FwdBufs &fb, const Plan &P, int dm, float eps, int me,
-                                                    uint64_t keep_policy) {
+__device__ __forceinline__ void activation_producer(Ctx &c, const FwdBufs &fb, const Plan &P, int me, uint64_t keep_policy) {
     constexpr int XS = x_stages(NT), XSTAGE_BYTES = xstage_bytes(NT);
+    if (me >= XS) return;
     int m = 0;
     for (int q = 0; q < n_ops(P); ++q) {
-        const int opi = op_index(P, q);
-        const GemmOp &op = P.op[opi];
-        const bool normed = opi == OP_QKV || opi == OP_GU || opi == OP_HEAD;
+        const GemmOp &op = P.op[op_index(P, q)];
         int t0, T, k_lo, k_hi;
         op_range(op, c.cta, c.ncta, t0, T, k_lo, k_hi);
         if (T == 0) continue;
         wait_count(fb, c.ready_op, q + 1, 6);
         __threadfence_block();
         asm volatile("fence.proxy.async;" ::: "memory");
-        if (me == X_PRODUCERS - 1) {
-            if (normed) {
-                compute_inv(c, fb, dm, eps);
-                __threadfence_block();
-                if (c.lane == 0) c.ready_op[1] = q + 1;
-                __syncwarp();
-            }
-            if (me >= XS) { for (int p0 = 0; p0 < T; p0 += MAX_TILES) for (int k = k_lo; k < k_hi; k += KC) ++m; continue; }
-        }
-        for (int p0 = 0; p0 < T; p0 += MAX_TILES) {
+        for (int p = 0; p < n_passes(T); ++p) {
             for (int k = k_lo; k < k_hi; k += KC, ++m) {
                 if (m % XS != me) continue;
                 const int slot = m % XS, nch = min(KC, k_hi - k) >> 5;
@@ -147,6 +136,24 @@ __device__ __forceinline__ void activation_producer(Ctx &c, const FwdBufs &fb, c
                 __syncwarp();
             }
         }
+    }
+}
+
+// Last warp of the block: 1/rms per row for the projections that follow an RMSNorm,
+// as soon as the projection's inputs are complete (ready_op[1] tells the epilogues).
+__device__ __forceinline__ void helper_warp(Ctx &c, const FwdBufs &fb, const Plan &P, int dm, float eps) {
+    for (int q = 0; q < n_ops(P); ++q) {
+        const int opi = op_index(P, q);
+        if (opi != OP_QKV && opi != OP_GU && opi != OP_HEAD) continue;
+        int t0, T, k_lo, k_hi;
+        op_range(P.op[opi], c.cta, c.ncta, t0, T, k_lo, k_hi);
+        if (T == 0) continue;
+        wait_count(fb, c.ready_op, q + 1, 6);
+        __threadfence_block();
+        compute_inv(c, fb, dm, eps);
+        __threadfence_block();
+        if (c.lane == 0) c.ready_op[1] = q + 1;
+        __syncwarp();
     }
 }
 
@@ -174,8 +181,8 @@ __device__ __forceinline__ void consume_unit(const unsigned char *stage, const u
 }
 
 // One projection, run by the eight MMA warps after the grid barrier that
-// completed its inputs.  Warp w owns tiles w and w + 8 of every pass, over the
-// full k extent; epi(tile, acc) gets the complete sums.
+// completed its inputs.  Warp w owns tile w of every pass, over the block's k
+// range; epi(tile, acc) gets the sums.
 // Accumulator element (nt, i): token row nt*8 + 2t + (i & 1), tile column g + 8*(i >> 1).
 template <int NT, class Epi>
 __device__ __forceinline__ void gemm_op(Ctx &c, const FwdBufs &fb, const Plan &P, int q, const float *resid, int resid_ld,
@@ -190,24 +197,23 @@ __device__ __forceinline__ void gemm_op(Ctx &c, const FwdBufs &fb, const Plan &P
     int t0, T, k_lo, k_hi;
     op_range(op, c.cta, c.ncta, t0, T, k_lo, k_hi);
     constexpr int XS = x_stages(NT), XSTAGE_BYTES = xstage_bytes(NT);
-    for (int p0 = 0; p0 < T; p0 += MAX_TILES) {
-        const int Tp = min(MAX_TILES, T - p0);
-        const bool has0 = c.warp < Tp, has1 = c.warp + MMA_WARPS < Tp;
+    for (int p = 0; p < n_passes(T); ++p) {
+        int p0, Tp;
+        pass_range(T, p, p0, Tp);
+        const bool has = c.warp < Tp;
         // Accumulators start from the residual rows when the projection adds into the residual stream: the
         // loads are issued before the k loop, so the epilogue has no global round trip of its own.
-        float acc0[NT][4], acc1[NT][4];
+        float acc[NT][4];
         {
             const int g = c.lane >> 2, t = c.lane & 3;
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
-                    acc0[nt][i] = acc1[nt][i] = 0.f;
-                    if (resid) {
-                        const int r = nt * 8 + 2 * t + (i & 1);
-                        const int n0 = (t0 + p0 + c.warp) * 16 + g + 8 * (i >> 1), n1 = n0 + MMA_WARPS * 16;
-                        if (has0 && n0 < op.N) acc0[nt][i] = __ldcg(resid + (size_t)r * resid_ld + n0);
-                        if (has1 && n1 < op.N) acc1[nt][i] = __ldcg(resid + (size_t)r * resid_ld + n1);
+                    acc[nt][i] = 0.f;
+                    if (resid && has) {
+                        const int r = nt * 8 + 2 * t + (i & 1), n0 = (t0 + p0 + c.warp) * 16 + g + 8 * (i >> 1);
+                        if (n0 < op.N) acc[nt][i] = __ldcg(resid + (size_t)r * resid_ld + n0);
                     }
                 }
         }
@@ -216,38 +222,26 @@ __device__ __forceinline__ void gemm_op(Ctx &c, const FwdBufs &fb, const Plan &P
             const int xslot = c.xn % XS;
             wait_bar(fb, c.xfull + xslot, ((uint32_t)(c.xn / XS)) & 1u, 8, c.xn);
             const uint4 *xs = reinterpret_cast<const uint4 *>(c.scratch + xslot * XSTAGE_BYTES);
-            // The units of a k step are consumed in waves of eight (one per MMA warp) with a barrier after each
-            // wave.  A ring stage is shared by different warps over time, and a parity wait is exact only while
-            // the waiter is less than one stage generation ahead: with NS >= 8, unit n - NS lies in an earlier
-            // wave, which the barrier has seen consumed.
-            if (has0) {
+            if (has) {
                 const int n = c.wn + c.warp, slot = n % NS;
                 wait_bar(fb, c.wfull + slot, ((uint32_t)(n / NS)) & 1u, 9, n);
-                consume_unit<NT>(c.ring + slot * STAGE_BYTES, xs, nch, acc0, c.lane);
+                consume_unit<NT>(c.ring + slot * STAGE_BYTES, xs, nch, acc, c.lane);
                 __syncwarp();
                 if (c.lane == 0) mbar_arrive(c.wempty + slot);
             }
+            // Lockstep over k.  A ring stage is shared by different warps over time, and a parity wait is exact
+            // only while the waiter is less than one stage generation ahead: a k step has at most NS units, so
+            // after this barrier unit n - NS of any unit n of the next step has been consumed.
             bsync();
-            if (Tp > MMA_WARPS) {
-                if (has1) {
-                    const int n = c.wn + c.warp + MMA_WARPS, slot = n % NS;
-                    wait_bar(fb, c.wfull + slot, ((uint32_t)(n / NS)) & 1u, 9, n);
-                    consume_unit<NT>(c.ring + slot * STAGE_BYTES, xs, nch, acc1, c.lane);
-                    __syncwarp();
-                    if (c.lane == 0) mbar_arrive(c.wempty + slot);
-                }
-                bsync();
-            }
             if (c.lane == 0) mbar_arrive(c.xempty + xslot);
             c.wn += Tp;
             ++c.xn;
         }
-        if (normed && (has0 || has1)) {
+        if (normed && has) {
             wait_count(fb, c.ready_op + 1, q + 1, 10);                 // 1/rms of this projection's input rows
             __threadfence_block();
         }
-        if (has0) epi(t0 + p0 + c.warp, acc0);
-        if (has1) epi(t0 + p0 + c.warp + MMA_WARPS, acc1);
+        if (has) epi(t0 + p0 + c.warp, acc);
     }
 }
 
