@@ -112,7 +112,8 @@ enum {
     PACER_BUF_HPEND = 5,         /* f32   [max_batch][block_b+1][d_draft] hidden rows waiting for M_B */
     PACER_BUF_DRAFT_LEN = 6,     /* int32 [max_batch][max_steps] gamma of every step */
     PACER_BUF_ACCEPT_LEN = 7,    /* int32 [max_batch][max_steps] n of every step */
-    PACER_BUF_KCACHE_T = 8,      /* bf16  [L][max_batch][Hkv][max_ctx][hd] (also _D = 10, _B = 12) */
+    PACER_BUF_KCACHE_T = 8,      /* bf16  [2][L][max_batch][Hkv][max_ctx][hd]: the values rounded to bf16, then their rounding
+                                    remainders (value - bf16(value), also bf16)  (also _D = 10, _B = 12) */
     PACER_BUF_VCACHE_T = 9,      /* bf16  same shape                        (also _D = 11, _B = 13) */
     PACER_BUF_KCACHE_D = 10, PACER_BUF_VCACHE_D = 11, PACER_BUF_KCACHE_B = 12, PACER_BUF_VCACHE_B = 13,
     PACER_BUF_PHASE_NS = 14      /* u64 [256 blocks][512] device clock (ns) at the phase boundaries of the last

@@ -81,7 +81,8 @@ struct ModelDev {
     int32_t hd, qrows;
     const bf16 *embed, *wqkv, *wo, *wgate, *wup, *wdown, *norm1, *norm2, *normf, *head, *head_b, *posemb;
     const int32_t *succ;
-    bf16 *kcache, *vcache;     // [L][max_batch][Hkv][max_ctx][hd]
+    bf16 *kcache, *vcache;     // [2][L][max_batch][Hkv][max_ctx][hd]: the bf16 values, then their rounding remainders
+    size_t kv_lo;              // elements between the two parts
     const float2 *rope;        // [max_ctx][hd/2] (cos, sin)
     int32_t loaded;
 };

@@ -39,9 +39,12 @@ constexpr int STAGE_BYTES = 16 * PITCH;         // 17408
 constexpr int NS = 8;                           // weight stages in the ring: one wave of the eight MMA warps
 constexpr int RING_BYTES = NS * STAGE_BYTES;    // 139264
 constexpr int XS_MAX = 3;                       // activation stages: as many as fit the scratch, at most 3 (one producer warp each)
-__host__ __device__ constexpr int xstage_bytes(int NT) { return NT * (KC / 32) * 512; }   // row tiles x chunks x 512 B
+constexpr int XK = 256;                         // k columns of one activation chunk (half a weight unit)
+constexpr int XCH = XK / 32;                    // its 32-wide chunks
+// An activation stage holds one chunk twice: the bf16 value ("hi") and the bf16 rounding remainder ("lo").
+__host__ __device__ constexpr int xstage_bytes(int NT) { return 2 * NT * XCH * 512; }   // hi + lo, row tiles x chunks x 512 B
 __host__ __device__ constexpr int x_stages(int NT) { return (80 * 1024) / xstage_bytes(NT) < XS_MAX ? (80 * 1024) / xstage_bytes(NT) : XS_MAX; }
-constexpr int SCRATCH_BYTES = 80 * 1024;        // the activation ring lives in its first 48 KB; the attention
+constexpr int SCRATCH_BYTES = 88 * 1024;        // the activation ring lives in its first 48 KB; the attention
                                                 // phase and the tails use all of it (no activations in flight then)
 constexpr int MISC_BYTES = 2048;
 constexpr int SMEM_BYTES = SCRATCH_BYTES + RING_BYTES + MISC_BYTES;
@@ -59,7 +62,8 @@ enum OpKind { OP_QKV = 0, OP_O = 1, OP_GU = 2, OP_DOWN = 3, OP_HEAD = 4, N_OPS =
 // [t0, t0 + T) given by op_range(); it runs them in passes of at most MAX_TILES, evenly sized.
 struct GemmOp {
     const bf16 *W1, *W2;     // layer-0 base; W2 only for the interleaved gate/up projection
-    const bf16 *X;           // activations, bf16 in fragment order [K/32][row tiles][32 lanes][8]
+    const bf16 *X;           // activations, bf16 in fragment order [K/32][row tiles][32 lanes][8]: the values rounded to bf16
+    long long x_lo;          // element offset from X to the same layout holding the rounding remainders (also bf16)
     long long lstride;       // elements between layers
     int32_t N;               // weight rows in all (gate/up: 2F)
     int32_t MT;              // 16-row tiles
@@ -78,7 +82,8 @@ struct Plan {
 // Device buffers of the forward kernel beyond DevPtrs (all in the workspace).
 struct FwdBufs {
     float *qkv;              // [MAX_ROWS][qrows] fp32
-    bf16 *xg;                // x * gain of the next RMSNorm, bf16 in fragment order (its 1/rms comes later)
+    bf16 *xg;                // x * gain of the next RMSNorm, split bf16 in fragment order (its 1/rms comes later)
+    long long xg_lo, att_lo, act_lo;   // element offsets of the remainder halves of xg, DevPtrs::att, DevPtrs::act
     float *ssq;              // [d/16][MAX_ROWS] sum of squares of x over the 16 columns of a tile
     float *part;             // k-slice partial tiles [S][d/16][row tiles * 8][16] of the two residual projections
     float *tile_top;         // [MT(head)][MAX_ROWS][4]: max, argmax (int bits), runner-up, unused
@@ -161,6 +166,15 @@ struct Ctx {
     uint64_t policy;
     int wn, xn;                    // weight units / activation chunks of this block consumed (or produced) so far
 };
+
+// Activations enter the tensor cores as TWO bf16 numbers, hi = bf16(v) and lo = bf16(v - hi): together they carry
+// 16 mantissa bits, so rounding the inputs of a projection no longer shows in the logits (with single bf16 inputs
+// the error against an fp64 evaluation grows to 0.18 over 32 layers of width 4096).  The weights stay bf16 as given.
+__device__ __forceinline__ void store_split(bf16 *hi_base, long long lo_off, size_t idx, float v) {
+    const bf16 h = __float2bfloat16(v);
+    hi_base[idx] = h;
+    hi_base[idx + lo_off] = __float2bfloat16(v - __bfloat162float(h));
+}
 
 // Barrier of the eight MMA warps (the producer warps never join it).
 __device__ __forceinline__ void bsync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }

@@ -1,12 +1,15 @@
 // Attention phase of the forward kernel: rotary embedding of the new q/k rows,
-// append of k/v to the bf16 cache, and causal attention of the new rows over the
-// cache, on tensor cores.  Work items are (sequence, head, key-range split).
-// Inside an item the eight MMA warps split the keys in steps of 16 (and the two
-// 16-row query tiles when there are more than 16 rows); every warp keeps a
-// running (max, sum, output) per row, FlashAttention style.  The warps' results
-// are merged through shared memory into the item's partial; after a grid barrier
-// the splits of every (sequence, head, row) are merged by one warp each into the
-// bf16 attention output, in the fragment order the output projection reads.
+// append of k/v to the cache, and causal attention of the new rows over the
+// cache, on tensor cores.  q, k, v and the probabilities enter the MMAs as split
+// bf16 (value + rounding remainder, see store_split), and the cache keeps both
+// parts of k and v: single bf16 operands here alone put 0.14 of error on the
+// logits of a 32-layer model of width 4096.  Work items are (sequence, head,
+// key-range split).  Inside an item the eight MMA warps split the keys in steps
+// of 8 (and the two 16-row query tiles when there are more than 16 rows); every
+// warp keeps a running (max, sum, output) per row, FlashAttention style.  The
+// warps' results are merged through shared memory into the item's partial; after
+// a grid barrier the splits of every (sequence, head, row) are merged by one warp
+// each into the attention output, in the fragment order the output projection reads.
 #pragma once
 #include "fwd_phases.cuh"
 
@@ -21,24 +24,29 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], const void *
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(smem_u32(smem_row)));
 }
 
-// Geometry of the shared-memory scratch during an attention item.
+// Geometry of the shared-memory scratch during an attention item.  "Planes": [0] the bf16 values, [1] the remainders.
 template <int HD>
 struct AttSmem {
     static constexpr int QP = HD * 2 + 64;   // bytes between query rows (conflict-free 16-byte reads of rows g, g+8)
     static constexpr int VP = HD * 2 + 16;   // bytes between the rows of a V step (conflict-free ldmatrix)
     static constexpr int PW = HD + 2;        // floats of a partial row: values, running max, running sum
-    static constexpr int Q_OFF = 0;                       // [32][QP] bf16 q, scaled and rotated
-    static constexpr int KN_OFF = 32 * QP;                // [32][HD] bf16 new keys as cached
-    static constexpr int VN_OFF = KN_OFF + 32 * HD * 2;   // [32][HD] bf16 new values as cached
-    static constexpr int VS_OFF = VN_OFF + 32 * HD * 2;   // [8 warps][16][VP] V rows of the current step
+    static constexpr int Q_OFF = 0;                           // [2 planes][32][QP] q, scaled and rotated
+    static constexpr int KN_OFF = 2 * 32 * QP;                // [2 planes][32][HD] new keys as cached
+    static constexpr int VN_OFF = KN_OFF + 2 * 32 * HD * 2;   // [2 planes][32][HD] new values as cached
+    static constexpr int VS_OFF = VN_OFF + 2 * 32 * HD * 2;   // [8 warps][16][VP] V of the current step: 8 keys x 2 planes
     static constexpr int END = VS_OFF + MMA_WARPS * 16 * VP;
     static_assert(END <= SCRATCH_BYTES, "attention staging does not fit the scratch");
     static_assert(MMA_WARPS * 16 * PW * 4 <= SCRATCH_BYTES, "attention merge buffer does not fit the scratch");
 };
 
-// Rotary embedding of the new rows of (seq, head h): q (scaled) to shared memory
-// as bf16; k, v of the kv head rounded to bf16 as the cache holds them, to shared
-// memory and, by one item per kv head, to the cache.
+__device__ __forceinline__ void split_bf16(float v, bf16 &hi, bf16 &lo) {
+    hi = __float2bfloat16(v);
+    lo = __float2bfloat16(v - __bfloat162float(hi));
+}
+
+// Rotary embedding of the new rows of (seq, head h): q (scaled) to shared memory;
+// k, v of the kv head as the cache holds them, to shared memory and, by one item
+// per kv head, to the cache.  All as split bf16.
 template <int HD>
 __device__ __forceinline__ void attention_rows(Ctx &c, const Args &a, int layer, int seq, int h, bool writer) {
     using SM = AttSmem<HD>;
@@ -53,38 +61,46 @@ __device__ __forceinline__ void attention_rows(Ctx &c, const Args &a, int layer,
     for (int i = threadIdx.x; i < 32 * half; i += MMA_THREADS) {
         const int j = i / half, ii = i - j * half;
         bf16 *qrow = reinterpret_cast<bf16 *>(c.scratch + SM::Q_OFF + j * SM::QP);
+        bf16 *qrow_lo = reinterpret_cast<bf16 *>(c.scratch + SM::Q_OFF + (32 + j) * SM::QP);
         if (j < n_r) {
             const int pos = pos0 + j;
             const float *row = a.fb.qkv + (size_t)(r_base + j) * qrows;
             const float2 cs = m.rope[(size_t)pos * half + ii];
             const float qa = __ldcg(row + h * HD + ii), qb = __ldcg(row + h * HD + ii + half);
-            qrow[ii] = __float2bfloat16((qa * cs.x - qb * cs.y) * scale);
-            qrow[ii + half] = __float2bfloat16((qb * cs.x + qa * cs.y) * scale);
+            split_bf16((qa * cs.x - qb * cs.y) * scale, qrow[ii], qrow_lo[ii]);
+            split_bf16((qb * cs.x + qa * cs.y) * scale, qrow[ii + half], qrow_lo[ii + half]);
             const float ka = __ldcg(row + (H + kh) * HD + ii), kb = __ldcg(row + (H + kh) * HD + ii + half);
-            const bf16 k0 = __float2bfloat16(ka * cs.x - kb * cs.y), k1 = __float2bfloat16(kb * cs.x + ka * cs.y);
-            const bf16 v0 = __float2bfloat16(__ldcg(row + (H + Hkv + kh) * HD + ii));
-            const bf16 v1 = __float2bfloat16(__ldcg(row + (H + Hkv + kh) * HD + ii + half));
+            bf16 k0, k0l, k1, k1l, v0, v0l, v1, v1l;
+            split_bf16(ka * cs.x - kb * cs.y, k0, k0l);
+            split_bf16(kb * cs.x + ka * cs.y, k1, k1l);
+            split_bf16(__ldcg(row + (H + Hkv + kh) * HD + ii), v0, v0l);
+            split_bf16(__ldcg(row + (H + Hkv + kh) * HD + ii + half), v1, v1l);
             kn[j * HD + ii] = k0; kn[j * HD + ii + half] = k1;
+            kn[(32 + j) * HD + ii] = k0l; kn[(32 + j) * HD + ii + half] = k1l;
             vn[j * HD + ii] = v0; vn[j * HD + ii + half] = v1;
+            vn[(32 + j) * HD + ii] = v0l; vn[(32 + j) * HD + ii + half] = v1l;
             if (writer) {
                 bf16 *kc = m.kcache + cbase + (size_t)pos * HD, *vc = m.vcache + cbase + (size_t)pos * HD;
                 kc[ii] = k0; kc[ii + half] = k1;
+                kc[m.kv_lo + ii] = k0l; kc[m.kv_lo + ii + half] = k1l;
                 vc[ii] = v0; vc[ii + half] = v1;
+                vc[m.kv_lo + ii] = v0l; vc[m.kv_lo + ii + half] = v1l;
             }
         } else {
-            qrow[ii] = __float2bfloat16(0.f);
-            qrow[ii + half] = __float2bfloat16(0.f);
+            qrow[ii] = qrow_lo[ii] = __float2bfloat16(0.f);
+            qrow[ii + half] = qrow_lo[ii + half] = __float2bfloat16(0.f);
         }
     }
 }
 
-// The key loop of one warp: keys in steps of 16 (step st, st + KW, ...), first the
+// The key loop of one warp: keys in steps of 8 (step st, st + KW, ...), first the
 // cached keys [lo, hi), then (last split only) the n_r keys of this forward, which
 // row j sees up to key j.  mt: the warp's 16-row query tile.  Leaves running max,
 // sum (this lane's share) and un-normalised output of rows g and g+8 of the tile.
+// Products of two remainders (2^-18 relative) are left out.
 template <int HD>
-__device__ __forceinline__ void attention_keys(Ctx &c, const bf16 *kcache, const bf16 *vcache, int lo, int hi, int n_new,
-                                               int n_r, int mt, int kw, int KW, float (&mx)[2], float (&lsum)[2],
+__device__ __forceinline__ void attention_keys(Ctx &c, const bf16 *kcache, const bf16 *vcache, size_t kv_lo, int lo, int hi,
+                                               int n_new, int n_r, int mt, int kw, int KW, float (&mx)[2], float (&lsum)[2],
                                                float (&o)[HD / 8][4]) {
     using SM = AttSmem<HD>;
     constexpr int NCH = HD / 32, NOT = HD / 8, QP = SM::QP, VP = SM::VP;
@@ -92,47 +108,54 @@ __device__ __forceinline__ void attention_keys(Ctx &c, const bf16 *kcache, const
     const bf16 *kn = reinterpret_cast<const bf16 *>(c.scratch + SM::KN_OFF), *vn = reinterpret_cast<const bf16 *>(c.scratch + SM::VN_OFF);
     unsigned char *vslot = c.scratch + SM::VS_OFF + c.warp * (16 * VP);
     const unsigned char *q0 = c.scratch + SM::Q_OFF + (mt * 16 + g) * QP + t * 16, *q1 = q0 + 8 * QP;
-    const int steps_c = (hi - lo + 15) >> 4, steps_n = (n_new + 15) >> 4;
+    const int steps_c = (hi - lo + 7) >> 3, steps_n = (n_new + 7) >> 3;
     for (int st = kw; st < steps_c + steps_n; st += KW) {
         const bool fresh = st >= steps_c;                // keys of this forward (from shared memory), else cached keys
-        const int key0 = fresh ? (st - steps_c) * 16 : lo + st * 16;
+        const int key0 = fresh ? (st - steps_c) * 8 : lo + st * 8;
         const int kend = fresh ? n_r : hi;               // first invalid key index
         const bf16 *kb = fresh ? kn : kcache, *vb = fresh ? vn : vcache;
-        // V rows of the step into this warp's slot (rows past the end repeat the last valid row: finite, and masked)
+        const size_t plane = fresh ? (size_t)32 * HD : kv_lo;
+        // V of the step into this warp's slot: rows 0..7 the values of the 8 keys, rows 8..15 their remainders
+        // (keys past the end repeat the last valid key: finite, and masked)
         for (int i = c.lane; i < 16 * (HD / 8); i += 32) {
             const int kr = i / (HD / 8), piece = i - kr * (HD / 8);
-            const bf16 *src = vb + (size_t)min(key0 + kr, kend - 1) * HD + piece * 8;
+            const bf16 *src = vb + (kr >> 3) * plane + (size_t)min(key0 + (kr & 7), kend - 1) * HD + piece * 8;
             if (fresh) *reinterpret_cast<uint4 *>(vslot + kr * VP + piece * 16) = *reinterpret_cast<const uint4 *>(src);
             else cp_async16(vslot + kr * VP + piece * 16, src);
         }
-        // scores S = Q K^T for 16 keys: lane (g, t) reads 8 consecutive channels of key g of each 8-key tile and
-        // uses them as the k slots {2t, 2t+1, 2t+8, 2t+9} of two MMAs; q is read with the same rule
-        float s[2][4];
+        // scores S = Q K^T for 8 keys: lane (g, t) reads 8 consecutive channels of key g and uses them as the
+        // k slots {2t, 2t+1, 2t+8, 2t+9} of two MMAs; q is read with the same rule
+        float s[4] = {0.f, 0.f, 0.f, 0.f};
+        {
+            const bf16 *krow = kb + (size_t)min(key0 + g, kend - 1) * HD + t * 8;
+            uint4 kf[NCH], kl[NCH];
 #pragma unroll
-        for (int nb = 0; nb < 2; ++nb) {
-            s[nb][0] = s[nb][1] = s[nb][2] = s[nb][3] = 0.f;
-            const bf16 *krow = kb + (size_t)min(key0 + nb * 8 + g, kend - 1) * HD + t * 8;
-            uint4 kf[NCH];
-#pragma unroll
-            for (int cc = 0; cc < NCH; ++cc) kf[cc] = *reinterpret_cast<const uint4 *>(krow + cc * 32);
+            for (int cc = 0; cc < NCH; ++cc) {
+                kf[cc] = *reinterpret_cast<const uint4 *>(krow + cc * 32);
+                kl[cc] = *reinterpret_cast<const uint4 *>(krow + plane + cc * 32);
+            }
 #pragma unroll
             for (int cc = 0; cc < NCH; ++cc) {
                 const uint4 qa = *reinterpret_cast<const uint4 *>(q0 + cc * 64), qb = *reinterpret_cast<const uint4 *>(q1 + cc * 64);
-                mma16816(s[nb], qa.x, qb.x, qa.y, qb.y, kf[cc].x, kf[cc].y);
-                mma16816(s[nb], qa.z, qb.z, qa.w, qb.w, kf[cc].z, kf[cc].w);
+                mma16816(s, qa.x, qb.x, qa.y, qb.y, kf[cc].x, kf[cc].y);
+                mma16816(s, qa.z, qb.z, qa.w, qb.w, kf[cc].z, kf[cc].w);
+                mma16816(s, qa.x, qb.x, qa.y, qb.y, kl[cc].x, kl[cc].y);
+                mma16816(s, qa.z, qb.z, qa.w, qb.w, kl[cc].z, kl[cc].w);
+                const uint4 la = *reinterpret_cast<const uint4 *>(q0 + 32 * QP + cc * 64);
+                const uint4 lb = *reinterpret_cast<const uint4 *>(q1 + 32 * QP + cc * 64);
+                mma16816(s, la.x, lb.x, la.y, lb.y, kf[cc].x, kf[cc].y);
+                mma16816(s, la.z, lb.z, la.w, lb.w, kf[cc].z, kf[cc].w);
             }
         }
         // mask: keys past the end; among the keys of this forward, row j sees keys 0..j
         float rmax[2] = {-INFINITY, -INFINITY};
 #pragma unroll
-        for (int nb = 0; nb < 2; ++nb)
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int key = key0 + nb * 8 + 2 * t + (i & 1), row = mt * 16 + g + 8 * (i >> 1);
-                const bool ok = key < kend && (!fresh || key <= row);
-                if (!ok) s[nb][i] = -INFINITY;
-                rmax[i >> 1] = fmaxf(rmax[i >> 1], s[nb][i]);
-            }
+        for (int i = 0; i < 4; ++i) {
+            const int key = key0 + 2 * t + (i & 1), row = mt * 16 + g + 8 * (i >> 1);
+            const bool ok = key < kend && (!fresh || key <= row);
+            if (!ok) s[i] = -INFINITY;
+            rmax[i >> 1] = fmaxf(rmax[i >> 1], s[i]);
+        }
         float corr[2];
 #pragma unroll
         for (int hr = 0; hr < 2; ++hr) {
@@ -143,24 +166,25 @@ __device__ __forceinline__ void attention_keys(Ctx &c, const bf16 *kcache, const
             mx[hr] = mnew;
             lsum[hr] *= corr[hr];
         }
-        uint32_t pa[4];
+        uint32_t ph[2], pl[2];                           // probabilities of rows g / g+8, keys 2t, 2t+1: values, remainders
         {
-            float p[2][4];
+            float p[4], r[4];
 #pragma unroll
-            for (int nb = 0; nb < 2; ++nb)
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const float mm = mx[i >> 1];
-                    p[nb][i] = mm == -INFINITY ? 0.f : __expf(s[nb][i] - mm);
-                    lsum[i >> 1] += p[nb][i];
-                }
-            pa[0] = pack_bf16x2(p[0][0], p[0][1]); pa[1] = pack_bf16x2(p[0][2], p[0][3]);
-            pa[2] = pack_bf16x2(p[1][0], p[1][1]); pa[3] = pack_bf16x2(p[1][2], p[1][3]);
+            for (int i = 0; i < 4; ++i) {
+                const float mm = mx[i >> 1];
+                p[i] = mm == -INFINITY ? 0.f : __expf(s[i] - mm);
+                lsum[i >> 1] += p[i];
+                r[i] = p[i] - __bfloat162float(__float2bfloat16(p[i]));
+            }
+            ph[0] = pack_bf16x2(p[0], p[1]); ph[1] = pack_bf16x2(p[2], p[3]);
+            pl[0] = pack_bf16x2(r[0], r[1]); pl[1] = pack_bf16x2(r[2], r[3]);
         }
 #pragma unroll
         for (int i = 0; i < NOT; ++i) { o[i][0] *= corr[0]; o[i][1] *= corr[0]; o[i][2] *= corr[1]; o[i][3] *= corr[1]; }
         // O += P V: V^T fragments through ldmatrix.trans from the slot.  Lane l gives the row address of
-        // matrix l / 8: keys 0..7 or 8..15 (bit 3 of l), channel tile 0 or 1 of the pair (bit 4 of l).
+        // matrix l / 8: slot rows 0..7 or 8..15 (bit 3 of l), channel tile 0 or 1 of the pair (bit 4 of l).
+        // The 16 k slots of an MMA are the 8 keys' values and then their remainders, so the probabilities
+        // appear twice in the first product; the second adds (remainder of P) x (values of V).
         cp_async_wait_all();
         __syncwarp();
         const unsigned char *vrow = vslot + ((c.lane & 7) + ((c.lane >> 3) & 1) * 8) * VP + (c.lane >> 4) * 16;
@@ -168,8 +192,10 @@ __device__ __forceinline__ void attention_keys(Ctx &c, const bf16 *kcache, const
         for (int np = 0; np < NOT / 2; ++np) {
             uint32_t vf[4];
             ldmatrix_x4_trans(vf, vrow + np * 32);
-            mma16816(o[2 * np], pa[0], pa[1], pa[2], pa[3], vf[0], vf[1]);
-            mma16816(o[2 * np + 1], pa[0], pa[1], pa[2], pa[3], vf[2], vf[3]);
+            mma16816(o[2 * np], ph[0], ph[1], ph[0], ph[1], vf[0], vf[1]);
+            mma16816(o[2 * np], pl[0], pl[1], 0u, 0u, vf[0], vf[1]);
+            mma16816(o[2 * np + 1], ph[0], ph[1], ph[0], ph[1], vf[2], vf[3]);
+            mma16816(o[2 * np + 1], pl[0], pl[1], 0u, 0u, vf[2], vf[3]);
         }
         __syncwarp();                                    // the slot is read; the next step may overwrite it
     }
@@ -201,7 +227,7 @@ __device__ __forceinline__ void attention_item(Ctx &c, const Args &a, int layer,
     float o[NOT][4];
 #pragma unroll
     for (int i = 0; i < NOT; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
-    attention_keys<HD>(c, m.kcache + cbase, m.vcache + cbase, lo, hi, split == nsplit - 1 ? n_r : 0, n_r, mt, kw, KW, mx, lsum, o);
+    attention_keys<HD>(c, m.kcache + cbase, m.vcache + cbase, m.kv_lo, lo, hi, split == nsplit - 1 ? n_r : 0, n_r, mt, kw, KW, mx, lsum, o);
 
     bsync();                                             // every warp is done with q, the new rows and the slots
     float *red = reinterpret_cast<float *>(c.scratch);   // [8 warps][16 rows][PW]
@@ -231,7 +257,7 @@ __device__ __forceinline__ void attention_item(Ctx &c, const Args &a, int layer,
             ov += rw[ch] * f;
         }
         if (nsplit == 1) {
-            d.att[xfrag_index(r_base + j, h * HD + ch, nt_total)] = __float2bfloat16(ov / L);
+            store_split(d.att, a.fb.att_lo, xfrag_index(r_base + j, h * HD + ch, nt_total), ov / L);
         } else {
             float *op = outp + (size_t)j * PW;
             op[ch] = ov;
@@ -276,7 +302,7 @@ __device__ __forceinline__ void phase_attention_merge(Ctx &c, const Args &a, int
 #pragma unroll
         for (int e = 0; e < 4; ++e)
             if (c.lane + 32 * e < hd)
-                a.d.att[xfrag_index(seq * rps + j, h * hd + c.lane + 32 * e, nt_total)] = __float2bfloat16(ov[e] * inv);
+                store_split(a.d.att, a.fb.att_lo, xfrag_index(seq * rps + j, h * hd + c.lane + 32 * e, nt_total), ov[e] * inv);
     }
 }
 

@@ -330,9 +330,10 @@ static inline Plan make_plan(const ModelDev &m, const DevPtrs &d, const FwdBufs 
     const pacer_model_cfg &k = m.cfg;
     const long long dm = k.d_model, F = k.d_ffn, hh = (long long)k.n_heads * m.hd;
     int rot = 0;
-    auto set = [&](int i, const bf16 *w1, const bf16 *w2, const bf16 *x, long long lstride, int N, int K, int MT, int inter) {
+    auto set = [&](int i, const bf16 *w1, const bf16 *w2, const bf16 *x, long long x_lo, long long lstride, int N, int K, int MT,
+                   int inter) {
         GemmOp &o = P.op[i];
-        o.W1 = w1; o.W2 = w2 ? w2 : w1; o.X = x; o.lstride = lstride; o.N = N; o.K = K; o.MT = MT; o.interleave = inter;
+        o.W1 = w1; o.W2 = w2 ? w2 : w1; o.X = x; o.x_lo = x_lo; o.lstride = lstride; o.N = N; o.K = K; o.MT = MT; o.interleave = inter;
         o.S = 1;
         // few tiles and enough bytes to be bandwidth bound: also cut along k, so that a block needs less of the
         // activations (a small projection is latency bound and better off without the extra pass and barrier)
@@ -344,11 +345,11 @@ static inline Plan make_plan(const ModelDev &m, const DevPtrs &d, const FwdBufs 
         o.rot = rot;
         rot = (rot + (MT % (ncta / o.S)) * o.S) % ncta;       // the next projection's extra tiles go to other blocks
     };
-    set(OP_QKV, m.wqkv, nullptr, fb.xg, (long long)m.qrows * dm, m.qrows, (int)dm, (m.qrows + 15) / 16, 0);
-    set(OP_O, m.wo, nullptr, d.att, dm * hh, (int)dm, (int)hh, ((int)dm + 15) / 16, 0);
-    set(OP_GU, m.wgate, m.wup, fb.xg, F * dm, (int)(2 * F), (int)dm, ((int)F + 7) / 8, 1);
-    set(OP_DOWN, m.wdown, nullptr, d.act, dm * F, (int)dm, (int)F, ((int)dm + 15) / 16, 0);
-    set(OP_HEAD, m.head, nullptr, fb.xg, 0, k.vocab, (int)dm, (k.vocab + 15) / 16, 0);
+    set(OP_QKV, m.wqkv, nullptr, fb.xg, fb.xg_lo, (long long)m.qrows * dm, m.qrows, (int)dm, (m.qrows + 15) / 16, 0);
+    set(OP_O, m.wo, nullptr, d.att, fb.att_lo, dm * hh, (int)dm, (int)hh, ((int)dm + 15) / 16, 0);
+    set(OP_GU, m.wgate, m.wup, fb.xg, fb.xg_lo, F * dm, (int)(2 * F), (int)dm, ((int)F + 7) / 8, 1);
+    set(OP_DOWN, m.wdown, nullptr, d.act, fb.act_lo, dm * F, (int)dm, (int)F, ((int)dm + 15) / 16, 0);
+    set(OP_HEAD, m.head, nullptr, fb.xg, fb.xg_lo, 0, k.vocab, (int)dm, (k.vocab + 15) / 16, 0);
     P.n_layers = k.n_layers;
     P.has_head = has_head ? 1 : 0;
     return P;

@@ -98,7 +98,7 @@ __device__ __forceinline__ void phase_begin(Ctx &c, const Args &a, int nt_total)
                 }
             }
             d.xres[(size_t)r * dm + col] = v;          // idle rows hold zeros: they stay finite through the layers
-            a.fb.xg[xfrag_index(r, col, nt_total)] = __float2bfloat16(v * gain);
+            store_split(a.fb.xg, a.fb.xg_lo, xfrag_index(r, col, nt_total), v * gain);
             float ss = v * v;
 #pragma unroll
             for (int o = 8; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
@@ -144,12 +144,12 @@ __device__ __forceinline__ void epi_residual(Ctx &c, const Args &a, const bf16 *
             if (n0 < dm) {
                 const float v = acc[nt][i];
                 x[n0] = v; ss[i] += v * v;
-                a.fb.xg[xfrag_index(r, n0, NT)] = __float2bfloat16(v * g0);
+                store_split(a.fb.xg, a.fb.xg_lo, xfrag_index(r, n0, NT), v * g0);
             }
             if (n1 < dm) {
                 const float v = acc[nt][2 + i];
                 x[n1] = v; ss[i] += v * v;
-                a.fb.xg[xfrag_index(r, n1, NT)] = __float2bfloat16(v * g1);
+                store_split(a.fb.xg, a.fb.xg_lo, xfrag_index(r, n1, NT), v * g1);
             }
         }
 #pragma unroll
@@ -211,7 +211,7 @@ __device__ __forceinline__ void phase_residual(Ctx &c, const Args &a, const Gemm
         for (int it = 0; it < NIT; ++it) {
             const int r = 2 * it + half;
             a.d.xres[(size_t)r * dm + col] = v[it];
-            a.fb.xg[xfrag_index(r, col, NT)] = __float2bfloat16(v[it] * gain);
+            store_split(a.fb.xg, a.fb.xg_lo, xfrag_index(r, col, NT), v[it] * gain);
             float ss = v[it] * v[it];
 #pragma unroll
             for (int o = 8; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
@@ -236,7 +236,7 @@ __device__ __forceinline__ void epi_swiglu(Ctx &c, const Args &a, int tile, floa
             const float inv = c.inv_rms[r];
             const float gt = acc[nt][i] * inv, up = acc[nt][2 + i] * inv;
             const float v = (r < a.g.rtot && c.row_pos[r] >= 0) ? gt / (1.f + expf(-gt)) * up : 0.f;
-            a.d.act[xfrag_index(r, f, NT)] = __float2bfloat16(v);
+            store_split(a.d.act, a.fb.act_lo, xfrag_index(r, f, NT), v);
         }
     }
 }

@@ -123,15 +123,17 @@ __device__ __forceinline__ void activation_producer(Ctx &c, const FwdBufs &fb, c
         __threadfence_block();
         asm volatile("fence.proxy.async;" ::: "memory");
         for (int p = 0; p < n_passes(T); ++p) {
-            for (int k = k_lo; k < k_hi; k += KC, ++m) {
+            for (int k = k_lo; k < k_hi; k += XK, ++m) {
                 if (m % XS != me) continue;
-                const int slot = m % XS, nch = min(KC, k_hi - k) >> 5;
+                const int slot = m % XS, nch = min(XK, k_hi - k) >> 5;
                 if (!wait_bar(fb, c.xempty + slot, (((uint32_t)(m / XS)) & 1u) ^ 1u, 7, m)) return;
-                if (c.lane == 0) {
+                if (c.lane == 0) {                       // the chunk's bf16 values, then its rounding remainders
                     const uint32_t bytes = (uint32_t)nch * (uint32_t)NT * 512u;
-                    mbar_expect_tx(c.xfull + slot, bytes);
-                    bulk_g2s(c.scratch + slot * XSTAGE_BYTES, op.X + (size_t)(k >> 5) * NT * 256, bytes, c.xfull + slot,
-                             keep_policy);
+                    const bf16 *src = op.X + (size_t)(k >> 5) * NT * 256;
+                    unsigned char *dst = c.scratch + slot * XSTAGE_BYTES;
+                    mbar_expect_tx(c.xfull + slot, 2u * bytes);
+                    bulk_g2s(dst, src, bytes, c.xfull + slot, keep_policy);
+                    bulk_g2s(dst + XSTAGE_BYTES / 2, src + op.x_lo, bytes, c.xfull + slot, keep_policy);
                 }
                 __syncwarp();
             }
@@ -157,25 +159,25 @@ __device__ __forceinline__ void helper_warp(Ctx &c, const FwdBufs &fb, const Pla
     }
 }
 
-// acc[nt] += W(16 rows x 32*nchunks k) * X over one stage.  Lane (g, t) reads the
-// 8 consecutive weights of rows g and g+8 at k = 32c + 8t and uses them as the k
-// slots {2t, 2t+1, 2t+8, 2t+9} of two MMAs; the activation fragments are stored
-// with the same rule, so the products pair up.
+// acc[nt] += W(16 rows x 32*nchunks k, from chunk `chunk0` of the stage) * (X_hi + X_lo).  Lane (g, t) reads the
+// 8 consecutive weights of rows g and g+8 at k = 32c + 8t and uses them as the k slots {2t, 2t+1, 2t+8, 2t+9}
+// of two MMAs; the activation fragments are stored with the same rule, so the products pair up.
 template <int NT>
-__device__ __forceinline__ void consume_unit(const unsigned char *stage, const uint4 *xs, int nchunks, float (&acc)[NT][4],
-                                             int lane) {
+__device__ __forceinline__ void consume_unit(const unsigned char *stage, int chunk0, const uint4 *xhi, const uint4 *xlo, int nchunks,
+                                             float (&acc)[NT][4], int lane) {
     const int g = lane >> 2, t = lane & 3;
-    const unsigned char *p0 = stage + g * PITCH + t * 16, *p1 = p0 + 8 * PITCH;
+    const unsigned char *p0 = stage + g * PITCH + t * 16 + chunk0 * 64, *p1 = p0 + 8 * PITCH;
 #pragma unroll 2
     for (int cix = 0; cix < nchunks; ++cix) {
         const uint4 a0 = *reinterpret_cast<const uint4 *>(p0 + cix * 64);
         const uint4 a1 = *reinterpret_cast<const uint4 *>(p1 + cix * 64);
-        const uint4 *xb = xs + cix * (NT * 32) + lane;
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
-            const uint4 b = xb[nt * 32];
-            mma16816(acc[nt], a0.x, a1.x, a0.y, a1.y, b.x, b.y);
-            mma16816(acc[nt], a0.z, a1.z, a0.w, a1.w, b.z, b.w);
+            const uint4 bh = xhi[(cix * NT + nt) * 32 + lane], bl = xlo[(cix * NT + nt) * 32 + lane];
+            mma16816(acc[nt], a0.x, a1.x, a0.y, a1.y, bh.x, bh.y);
+            mma16816(acc[nt], a0.z, a1.z, a0.w, a1.w, bh.z, bh.w);
+            mma16816(acc[nt], a0.x, a1.x, a0.y, a1.y, bl.x, bl.y);
+            mma16816(acc[nt], a0.z, a1.z, a0.w, a1.w, bl.z, bl.w);
         }
     }
 }
@@ -219,23 +221,29 @@ __device__ __forceinline__ void gemm_op(Ctx &c, const FwdBufs &fb, const Plan &P
         }
         for (int k = k_lo; k < k_hi; k += KC) {
             const int nch = min(KC, k_hi - k) >> 5;
-            const int xslot = c.xn % XS;
-            wait_bar(fb, c.xfull + xslot, ((uint32_t)(c.xn / XS)) & 1u, 8, c.xn);
-            const uint4 *xs = reinterpret_cast<const uint4 *>(c.scratch + xslot * XSTAGE_BYTES);
+            int slot = 0;
             if (has) {
-                const int n = c.wn + c.warp, slot = n % NS;
+                const int n = c.wn + c.warp;
+                slot = n % NS;
                 wait_bar(fb, c.wfull + slot, ((uint32_t)(n / NS)) & 1u, 9, n);
-                consume_unit<NT>(c.ring + slot * STAGE_BYTES, xs, nch, acc, c.lane);
-                __syncwarp();
-                if (c.lane == 0) mbar_arrive(c.wempty + slot);
             }
+            for (int c0 = 0; c0 < nch; c0 += XCH) {           // the activations come in chunks of XK columns
+                const int xslot = c.xn % XS;
+                wait_bar(fb, c.xfull + xslot, ((uint32_t)(c.xn / XS)) & 1u, 8, c.xn);
+                if (has) {
+                    const uint4 *xhi = reinterpret_cast<const uint4 *>(c.scratch + xslot * XSTAGE_BYTES);
+                    consume_unit<NT>(c.ring + slot * STAGE_BYTES, c0, xhi, xhi + XSTAGE_BYTES / 32, min(XCH, nch - c0), acc, c.lane);
+                }
+                __syncwarp();
+                if (c.lane == 0) mbar_arrive(c.xempty + xslot);
+                ++c.xn;
+            }
+            if (has && c.lane == 0) mbar_arrive(c.wempty + slot);
             // Lockstep over k.  A ring stage is shared by different warps over time, and a parity wait is exact
-            // only while the waiter is less than one stage generation ahead: a k step has at most NS units, so
-            // after this barrier unit n - NS of any unit n of the next step has been consumed.
+            // only while the waiter is less than one stage generation ahead: a k step has at most NS units (and
+            // at most two activation chunks), so after this barrier the stage's previous user is done.
             bsync();
-            if (c.lane == 0) mbar_arrive(c.xempty + xslot);
             c.wn += Tp;
-            ++c.xn;
         }
         if (normed && has) {
             wait_count(fb, c.ready_op + 1, q + 1, 10);                 // 1/rms of this projection's input rows

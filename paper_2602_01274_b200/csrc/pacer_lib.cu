@@ -120,7 +120,7 @@ struct Layout {
     size_t kc[3], vc[3], rope[3];
     size_t kv_bytes[3], rope_bytes[3];
     size_t total;
-    int rtot_max, nt_max, max_steps;
+    int rtot_max, nt_max, max_steps, d_max, f_max;
     size_t part_bytes, state_bytes;
 };
 
@@ -172,12 +172,13 @@ static Layout make_layout(const pacer_cfg &c) {
     L.hpend = cv.take(sizeof(float) * B * (c.block_b + 1) * c.draft.d_model);
     L.verify_logits = cv.take(sizeof(float) * B * (gc + 1) * V);
     L.draft_logits = cv.take(sizeof(float) * B * gc * V);
+    L.d_max = d_max; L.f_max = f_max;
     L.xres = cv.take(sizeof(float) * fwd::MAX_ROWS * d_max);
     L.hidden = cv.take(sizeof(float) * fwd::MAX_ROWS * d_max);
-    L.att = cv.take(sizeof(bf16) * fwd::MAX_ROWS * d_max);
-    L.act = cv.take(sizeof(bf16) * fwd::MAX_ROWS * f_max);
+    L.att = cv.take(sizeof(bf16) * 2 * fwd::MAX_ROWS * d_max);        // values, then rounding remainders
+    L.act = cv.take(sizeof(bf16) * 2 * fwd::MAX_ROWS * f_max);
     L.qkv = cv.take(sizeof(float) * fwd::MAX_ROWS * qrows_max);
-    L.xg = cv.take(sizeof(bf16) * fwd::MAX_ROWS * d_max);
+    L.xg = cv.take(sizeof(bf16) * 2 * fwd::MAX_ROWS * d_max);
     L.ssq = cv.take(sizeof(float) * fwd::MAX_ROWS * (d_max / 16 + 1));
     L.tile_top = cv.take(sizeof(float) * 4 * fwd::MAX_ROWS * ((size_t)V / 16 + 1));
     L.attp = cv.take(sizeof(float) * (size_t)B * h_max * fwd::MAX_SPLIT * rps_max * (hd_max + 2));
@@ -185,7 +186,7 @@ static Layout make_layout(const pacer_cfg &c) {
     L.part = cv.take(L.part_bytes);
     for (int i = 0; i < 3; ++i) {
         const int hd = ms[i]->d_model / ms[i]->n_heads;
-        L.kv_bytes[i] = sizeof(bf16) * (size_t)ms[i]->n_layers * B * ms[i]->n_kv_heads * c.max_ctx * hd;
+        L.kv_bytes[i] = 2 * sizeof(bf16) * (size_t)ms[i]->n_layers * B * ms[i]->n_kv_heads * c.max_ctx * hd;   // values + remainders
         L.kc[i] = cv.take(L.kv_bytes[i]);
         L.vc[i] = cv.take(L.kv_bytes[i]);
         L.rope_bytes[i] = sizeof(float2) * (size_t)c.max_ctx * (hd / 2);
@@ -245,6 +246,8 @@ extern "C" int pacer_create(const pacer_cfg *cfg, void *dev_workspace, size_t wo
     d.q = nullptr; d.hidden = (float *)(w + L.hidden); d.part = (float *)(w + L.part);
     c->fb.qkv = (float *)(w + L.qkv); c->fb.xg = (bf16 *)(w + L.xg); c->fb.ssq = (float *)(w + L.ssq);
     c->fb.part = (float *)(w + L.part);
+    c->fb.xg_lo = c->fb.att_lo = (long long)fwd::MAX_ROWS * L.d_max;
+    c->fb.act_lo = (long long)fwd::MAX_ROWS * L.f_max;
     c->fb.tile_top = (float *)(w + L.tile_top); c->fb.attp = (float *)(w + L.attp);
     c->fb.att_cnt = (int32_t *)(w + L.att_cnt); c->fb.bar = (unsigned long long *)(w + L.bar);
     c->fb.abort_flag = (int32_t *)(w + L.abort_flag);
@@ -264,6 +267,7 @@ extern "C" int pacer_create(const pacer_cfg *cfg, void *dev_workspace, size_t wo
         m.qrows = (m.cfg.n_heads + 2 * m.cfg.n_kv_heads) * m.hd;
         m.kcache = (bf16 *)(w + L.kc[i]);
         m.vcache = (bf16 *)(w + L.vc[i]);
+        m.kv_lo = L.kv_bytes[i] / (2 * sizeof(bf16));
         m.rope = (const float2 *)(w + L.rope[i]);
         const int half = m.hd / 2;
         c->rope_host[i].resize((size_t)cfg->max_ctx * half);

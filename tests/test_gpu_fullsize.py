@@ -1,0 +1,64 @@
+"""GPU parity at the full 7B / 68M sizes, in the launch configuration the benchmark times (one cooperative launch
+per forward, one block per SM, 17 verify rows): all 32 layers at width 4096 with the 32000-entry head, against the
+fp64 oracle reading the same bf16 weights.  The prompt is short so that the oracle's prefill stays within seconds;
+the verify forward itself is the full one.  Logits within 2e-2; drafts bit-exact where the oracle's margins allow."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import pacer_oracle as orc
+from paper_2602_01274_b200 import synth
+from tests.common import oracle_models
+
+pytestmark = pytest.mark.gpu
+
+LOGIT_TOL = 2e-2
+ALPHA_TOL = 2e-3
+
+
+def test_7b_verify_forward_full_size():
+    from paper_2602_01274_b200 import binding as b
+    cfg = dataclasses.replace(synth.CONFIGS["7b_68m"], n_prompt=4, max_new=20)
+    V, gc, bb = cfg.target.vocab, cfg.gamma_cap, cfg.block_b
+    pair_gpu = synth.make_pair(cfg, seed=1, device="cuda:0")
+    pair_cpu = {k: ({n: t.cpu() for n, t in v.items()} if isinstance(v, dict) else v.cpu()) for k, v in pair_gpu.items()}
+    T, D, B = oracle_models(cfg, pair_cpu)
+    max_ctx = cfg.n_prompt + cfg.max_new + gc + 2
+    ctx = b.Context(b.make_cfg(cfg.target, cfg.draft, 1, max_ctx, gc, bb, cfg.rho, 0, cfg.succ_bias))
+    try:
+        b.load_pair(ctx, pair_gpu)
+        del pair_gpu
+        prompt = synth.make_prompts(V, 1, cfg.n_prompt, seed=3)[0].numpy()
+        o = orc.Pacer(T, D, B, max_ctx, b=bb, gamma_cap=gc, t0=-1.0, rho=cfg.rho)
+        o.prefill(prompt)
+        ctx.pacer_prefill(prompt, cfg.max_new, cfg.gamma_max, -1.0)
+        while o.drafting:
+            for _ in range(bb):
+                ctx.pacer_draft_step()
+            o.draft_block()
+            ql = ctx.pacer_read_buffer(b.BUF_DRAFT_LOGITS, np.float32, gc * V).reshape(gc, V)[: o.gamma]
+            assert np.abs(ql - o.qlogits(o.gamma)).max() < LOGIT_TOL
+            y = ctx.pacer_read_buffer(b.BUF_DRAFTS, np.int32, gc)[: o.gamma]
+            np.testing.assert_array_equal(y, o.y())
+            ctx.pacer_preverify()
+            o.preverify()
+            al = ctx.pacer_read_buffer(b.BUF_ALPHA, np.float32, gc)[: o.gamma]
+            assert np.abs(al - o.alpha()).max() < ALPHA_TOL
+        assert o.gamma == gc
+        ctx.pacer_verify()
+        o.verify()
+        pl = ctx.pacer_read_buffer(b.BUF_VERIFY_LOGITS, np.float32, (gc + 1) * V).reshape(gc + 1, V)
+        ref = o.plogits(gc + 1)
+        err = np.abs(pl - ref).max()
+        assert err < LOGIT_TOL, f"verify logits differ by {err}"
+        ctx.pacer_accept_rollback()
+        n = o.accept()
+        st = ctx.pacer_read_state()[0]
+        top2 = np.sort(ref, axis=1)[:, -2:]
+        if (top2[: n + 1, 1] - top2[: n + 1, 0]).min() > 2 * LOGIT_TOL:
+            assert (st["last_n"], st["last_next"], st["P"]) == (n, o.last_next, o.P)
+    finally:
+        ctx.close()
+        torch.cuda.empty_cache()

@@ -29,6 +29,10 @@ SHAPES = {
     "long_ctx": synth.PairConfig("long_ctx", synth.ModelShape(2, 256, 2, 2, 512, 4096),
                                  synth.ModelShape(1, 128, 2, 2, 256, 4096), agree=0.8, n_prompt=700, max_new=16,
                                  gamma_max=12),
+    # many layers: rounding of the activations between layers must not pile up over depth
+    "deep": synth.PairConfig("deep", synth.ModelShape(48, 256, 4, 4, 512, 4096),
+                             synth.ModelShape(1, 128, 2, 2, 256, 4096), agree=0.8, n_prompt=24, max_new=16,
+                             gamma_max=16),
 }
 
 
