@@ -80,6 +80,7 @@ struct ModelDev {
     pacer_model_cfg cfg;
     int32_t hd, qrows;
     const bf16 *embed, *wqkv, *wo, *wgate, *wup, *wdown, *norm1, *norm2, *normf, *head, *head_b, *posemb;
+    const bf16 *wt[5];         // the five projections re-laid for the tensor cores (index: OpKind of the forward kernel)
     const int32_t *succ;
     bf16 *kcache, *vcache;     // [2][L][max_batch][Hkv][max_ctx][hd]: the bf16 values, then their rounding remainders
     size_t kv_lo;              // elements between the two parts

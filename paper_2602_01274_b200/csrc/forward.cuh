@@ -1,54 +1,59 @@
 // One decoder forward as ONE persistent cooperative kernel (one block per SM).
 //
 // The forward is bound by streaming the weights from HBM once, so the kernel is
-// built around an uninterrupted weight stream and a critical path with as few
-// dependent global-memory round trips as possible:
-//   - a producer warp walks the static list of weight units (16 rows x 256 k)
-//     of the block for the WHOLE forward and keeps a shared-memory ring full
-//     with bulk async copies (cp.async.bulk + mbarrier); it runs ahead into the
-//     next projection while the block sits in a grid barrier or in a small
-//     phase, so the HBM queue never drains between projections;
-//   - a block owns whole 16-row tiles of a projection over its k range (no
-//     partial-sum buffers, no arrival counters, no fences), the eight MMA warps
-//     advance over k in lockstep, and the activation rows of each 256-wide k
-//     step arrive through a second small ring, filled by activation-producer warps;
-//   - tensor cores (mma.m16n8k16, bf16 in / fp32 accumulate, weights as the
-//     16-row operand) do the contraction, so the math is invisible;
-//   - the row-wise step that follows a projection in the decoder (residual add,
-//     SwiGLU, bias/arg-max of the LM head) is the epilogue of the warp that owns
-//     the tile; RMSNorm is split: the residual epilogue also writes x * gain as
-//     bf16 in fragment order (the next projection's input) and the tile's share
-//     of sum(x^2), and the 1/rms factor is applied to the OUTPUT rows of the
-//     next projection in its epilogue, so no normalisation pass exists;
+// built around an uninterrupted weight stream with as many bytes in flight as
+// shared memory can hold, and a critical path with as few dependent
+// global-memory round trips as possible:
+//   - the weights are kept in HBM as 8-row x 64-column atoms (1 KB) that already
+//     have the 128-byte-swizzled K-major layout tcgen05.mma reads from shared
+//     memory, ordered [k block][row atom]: the rows a block owns in a projection
+//     are one contiguous run per k block, fetched by ONE bulk async copy
+//     (cp.async.bulk + mbarrier) into a byte ring; a producer thread walks the
+//     static list of these stages for the WHOLE forward and runs ahead into the
+//     next projection while the block sits in a grid barrier or a small phase;
+//   - the contraction runs on the 5th-generation tensor cores: one thread issues
+//     tcgen05.mma (M = 128, N = the block's weight rows, K = 16) with the
+//     ACTIVATION rows as the A operand and the weight stage as the B operand, the
+//     accumulator lives in tensor memory, and tcgen05.commit hands each stage back
+//     to the producer the moment its MMAs are done, so nearly the whole ring is
+//     in flight (a load takes about 3 us under full load: bandwidth = bytes in
+//     flight / latency);
+//   - activations enter as split bf16 (value rows, then remainder rows, stacked
+//     along M), through a second small ring filled by activation-producer warps;
+//   - the eight phase warps read the accumulator back (tcgen05.ld) into shared
+//     memory once per projection and run the row-wise step that follows it in the
+//     decoder (residual add, SwiGLU, bias/arg-max of the LM head) as the epilogue;
+//     RMSNorm is split: the residual epilogue also writes x * gain as split bf16 in
+//     operand order (the next projection's input) and the tile's share of
+//     sum(x^2), and the 1/rms factor is applied to the OUTPUT rows of the next
+//     projection in its epilogue, so no normalisation pass exists;
 //   - phases are separated by grid barriers with bounded waits.
 #pragma once
 #include "common.cuh"
 
 namespace fwd {
 
-constexpr int MMA_WARPS = 8, MMA_THREADS = 256;  // warps 0..7: MMAs, epilogues and all block-wide phases
-constexpr int W_PRODUCERS = 4;                   // warps 8..11 stream weights: unit n by producer n % 4 (one warp alone
-                                                 // cannot issue the bulk copies fast enough)
-constexpr int X_PRODUCERS = 4;                   // warps 12..14 provide the activation chunks (stage s by producer s); warp 15
-                                                 // computes the RMS statistics
-constexpr int W_PRODUCER = MMA_WARPS, X_PRODUCER = W_PRODUCER + W_PRODUCERS;
+constexpr int MMA_WARPS = 8, MMA_THREADS = 256;  // warps 0..7 ("phase warps"): epilogues and all block-wide phases
+constexpr int W_PRODUCER = 8;                    // warp 8, lane 0: the weight stream
+constexpr int MMA_ISSUER = 9;                    // warp 9: owns the tensor memory; its lane 0 issues every tcgen05.mma
+constexpr int X_PRODUCER = 12, X_PRODUCERS = 4;  // warps 12..14 provide the activation stages (stage s by producer s);
+                                                 // warp 15 computes the RMS statistics; warps 10, 11 have no work
 constexpr int THREADS = 32 * (X_PRODUCER + X_PRODUCERS);
-constexpr int KC = 512;                         // k columns of one weight unit: 1 KB per row and copy (DRAM likes long runs)
-constexpr int PITCH = KC * 2 + 64;              // bytes between the rows of a stage (bank-conflict free)
-constexpr int STAGE_BYTES = 16 * PITCH;         // 17408
-constexpr int NS = 8;                           // weight stages in the ring: one wave of the eight MMA warps
-constexpr int RING_BYTES = NS * STAGE_BYTES;    // 139264
-constexpr int XS_MAX = 3;                       // activation stages: as many as fit the scratch, at most 3 (one producer warp each)
-constexpr int XK = 256;                         // k columns of one activation chunk (half a weight unit)
-constexpr int XCH = XK / 32;                    // its 32-wide chunks
-// An activation stage holds one chunk twice: the bf16 value ("hi") and the bf16 rounding remainder ("lo").
-__host__ __device__ constexpr int xstage_bytes(int NT) { return 2 * NT * XCH * 512; }   // hi + lo, row tiles x chunks x 512 B
+constexpr int KB = 64;                          // k columns of a weight stage: one 128-byte swizzle row
+constexpr int KC = 512;                         // k slices of a projection are whole multiples of this
+constexpr int NB = 16;                          // weight stages that can be in flight (barrier pairs)
+constexpr int RING_BYTES = 136 * 1024;          // weight ring (bytes; a stage takes 128 B per weight row of the block)
+constexpr int XS_MAX = 3;                       // activation stages: as many as fit, at most 3 (one producer warp each)
+constexpr int XK = 256;                         // k columns of one activation stage (four k blocks)
+// Per k block an activation stage holds NT atoms of bf16 values and then NT atoms of bf16 rounding remainders.
+__host__ __device__ constexpr int xstage_bytes(int NT) { return (XK / KB) * 2 * NT * 1024; }
 __host__ __device__ constexpr int x_stages(int NT) { return (80 * 1024) / xstage_bytes(NT) < XS_MAX ? (80 * 1024) / xstage_bytes(NT) : XS_MAX; }
-constexpr int SCRATCH_BYTES = 88 * 1024;        // the activation ring lives in its first 48 KB; the attention
-                                                // phase and the tails use all of it (no activations in flight then)
+constexpr int SCRATCH_BYTES = 88 * 1024;        // the activation ring lives in its first 72 KB at most; the epilogues' copy
+                                                // of the accumulator, the attention phase and the tails use all of it
 constexpr int MISC_BYTES = 2048;
 constexpr int SMEM_BYTES = SCRATCH_BYTES + RING_BYTES + MISC_BYTES;
-constexpr int MAX_TILES = 8;                    // tiles of one pass of a block: one per MMA warp, one ring generation per k step
+constexpr int MAX_TILES = 16;                   // 16-row tiles of one pass of a block: N = 256 of one tcgen05.mma
+constexpr int TMEM_COLS = 256;                  // fp32 accumulator columns (one per weight row of the pass)
 constexpr int MAX_ROWS = 32;                    // rows of one forward (all sequences together)
 constexpr int MAX_SPLIT = 16;                   // key-range splits of one attention head
 constexpr unsigned SPIN_LIMIT = 1u << 22;        // polls of a global word or a shared counter
@@ -61,9 +66,8 @@ enum OpKind { OP_QKV = 0, OP_O = 1, OP_GU = 2, OP_DOWN = 3, OP_HEAD = 4, N_OPS =
 // One weight-streaming projection.  Block c owns the contiguous tiles
 // [t0, t0 + T) given by op_range(); it runs them in passes of at most MAX_TILES, evenly sized.
 struct GemmOp {
-    const bf16 *W1, *W2;     // layer-0 base; W2 only for the interleaved gate/up projection
-    const bf16 *X;           // activations, bf16 in fragment order [K/32][row tiles][32 lanes][8]: the values rounded to bf16
-    long long x_lo;          // element offset from X to the same layout holding the rounding remainders (also bf16)
+    const bf16 *W;           // layer-0 base of the tiled weights: [K/64][2*MT atoms][8 rows][64 k, 16-byte chunks XOR-swizzled by row]
+    const bf16 *X;           // activations, split bf16 in operand order (see xatom_index)
     long long lstride;       // elements between layers
     int32_t N;               // weight rows in all (gate/up: 2F)
     int32_t MT;              // 16-row tiles
@@ -71,7 +75,6 @@ struct GemmOp {
     int32_t S;               // k slices: 1, or (attention output / MLP down, which have few tiles) a divisor of the
                              // grid size: the slices' partial tiles are summed by a small pass after a grid barrier
     int32_t rot;             // block that gets the first tile range (spreads the one-tile imbalance)
-    int32_t interleave;      // 1: tile t = gate rows 8t..8t+7 then up rows 8t..8t+7
 };
 
 struct Plan {
@@ -82,8 +85,7 @@ struct Plan {
 // Device buffers of the forward kernel beyond DevPtrs (all in the workspace).
 struct FwdBufs {
     float *qkv;              // [MAX_ROWS][qrows] fp32
-    bf16 *xg;                // x * gain of the next RMSNorm, split bf16 in fragment order (its 1/rms comes later)
-    long long xg_lo, att_lo, act_lo;   // element offsets of the remainder halves of xg, DevPtrs::att, DevPtrs::act
+    bf16 *xg;                // x * gain of the next RMSNorm, split bf16 in operand order (its 1/rms comes later)
     float *ssq;              // [d/16][MAX_ROWS] sum of squares of x over the 16 columns of a tile
     float *part;             // k-slice partial tiles [S][d/16][row tiles * 8][16] of the two residual projections
     float *tile_top;         // [MT(head)][MAX_ROWS][4]: max, argmax (int bits), runner-up, unused
@@ -147,14 +149,51 @@ __device__ __forceinline__ void mma16816(float (&c)[4], uint32_t a0, uint32_t a1
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
+// ---- 5th-generation tensor cores (tcgen05) and tensor memory
+
+// Shared-memory matrix descriptor of a K-major operand in the 128-byte swizzle layout: rows of 128 bytes, groups of
+// eight rows 1024 bytes apart; `saddr` is 1024-byte aligned plus 32 bytes per 16-column step inside the swizzle row.
+__device__ __forceinline__ uint64_t umma_desc(uint32_t saddr) {
+    return (uint64_t)((saddr >> 4) & 0x3FFF) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = n (a multiple of 16, at most 256).
+__device__ __forceinline__ uint32_t umma_idesc(int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | (((uint32_t)n >> 3) << 17) | ((128u >> 4) << 24);
+}
+// D[tmem] (+)= A[smem] * B[smem]^T, issued by one thread.
+__device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t a, uint64_t b, uint32_t idesc, uint32_t accumulate) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}\n"
+                 ::"r"(d_tmem), "l"(a), "l"(b), "r"(idesc), "r"(accumulate), "r"(0u) : "memory");
+}
+// The barrier gets one arrival when every tcgen05.mma this thread issued before has finished.
+__device__ __forceinline__ void umma_commit(uint64_t *bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// 32 consecutive accumulator columns of this thread's lane (lane = 32 * (warp % 4) + lane id).
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]), "=r"(v[9]),
+                   "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]), "=r"(v[17]), "=r"(v[18]),
+                   "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]),
+                   "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+                 : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
 // ------------------------------------------------------------------ block-level context
 
 struct Ctx {
     // shared memory
     unsigned char *scratch;        // SCRATCH_BYTES (activation ring in front)
     unsigned char *ring;           // weight ring
-    uint64_t *wfull, *wempty;      // [NS]
+    uint64_t *wfull, *wempty;      // [NB]
     uint64_t *xfull, *xempty;      // [XS_MAX]
+    uint64_t *acc_full, *acc_empty; // the accumulator of a pass is complete / has been copied out
+    volatile int32_t *pass_done;   // passes whose epilogue is over (the activation ring may be overwritten)
+    uint32_t tmem;                 // tensor-memory address of the accumulator
     int32_t *row_pos, *row_tok;    // [MAX_ROWS]
     int32_t *n_rows;               // [MAX_ROWS] per sequence
     float *inv_rms;                // [MAX_ROWS]
@@ -164,19 +203,28 @@ struct Ctx {
     unsigned long long bar_target; // used by thread 0
     int warp, lane, cta, ncta;
     uint64_t policy;
-    int wn, xn;                    // weight units / activation chunks of this block consumed (or produced) so far
+    int np;                        // passes of this block finished so far (phase warps)
 };
 
 // Activations enter the tensor cores as TWO bf16 numbers, hi = bf16(v) and lo = bf16(v - hi): together they carry
 // 16 mantissa bits, so rounding the inputs of a projection no longer shows in the logits (with single bf16 inputs
 // the error against an fp64 evaluation grows to 0.18 over 32 layers of width 4096).  The weights stay bf16 as given.
-__device__ __forceinline__ void store_split(bf16 *hi_base, long long lo_off, size_t idx, float v) {
+//
+// Operand order of an activation buffer with nt row tiles of 8: [k / 64][2 * nt atoms][8 rows][64 k], an atom being
+// 1 KB in the 128-byte swizzle layout (the 16-byte chunk c of row r sits at chunk c ^ r); atoms 0 .. nt-1 of a
+// k block hold the values of rows 8a .. 8a+7, atoms nt .. 2nt-1 the remainders.  As the A operand of an MMA with
+// M = 128 the values are accumulator lanes 0 .. 8nt-1 and the remainders lanes 8nt .. 16nt-1; the epilogue adds them.
+__device__ __forceinline__ size_t xatom_index(int r, int k, int nt, int plane) {
+    const int kk = k & 63, rr = r & 7;
+    return ((size_t)(k >> 6) * (2 * nt) + plane * nt + (r >> 3)) * 512 + rr * 64 + ((((kk >> 3) ^ rr) << 3) | (kk & 7));
+}
+__device__ __forceinline__ void store_split(bf16 *base, int nt, int r, int k, float v) {
     const bf16 h = __float2bfloat16(v);
-    hi_base[idx] = h;
-    hi_base[idx + lo_off] = __float2bfloat16(v - __bfloat162float(h));
+    base[xatom_index(r, k, nt, 0)] = h;
+    base[xatom_index(r, k, nt, 1)] = __float2bfloat16(v - __bfloat162float(h));
 }
 
-// Barrier of the eight MMA warps (the producer warps never join it).
+// Barrier of the eight phase warps (the producer warps never join it).
 __device__ __forceinline__ void bsync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
 // Work of block `cta` in a projection: tiles [t0, t0 + T) over the k range [k_lo, k_hi).

@@ -9,7 +9,7 @@
 // warp keeps a running (max, sum, output) per row, FlashAttention style.  The
 // warps' results are merged through shared memory into the item's partial; after
 // a grid barrier the splits of every (sequence, head, row) are merged by one warp
-// each into the attention output, in the fragment order the output projection reads.
+// each into the attention output, in the operand order the output projection reads.
 #pragma once
 #include "fwd_phases.cuh"
 
@@ -257,7 +257,7 @@ __device__ __forceinline__ void attention_item(Ctx &c, const Args &a, int layer,
             ov += rw[ch] * f;
         }
         if (nsplit == 1) {
-            store_split(d.att, a.fb.att_lo, xfrag_index(r_base + j, h * HD + ch, nt_total), ov / L);
+            store_split(d.att, nt_total, r_base + j, h * HD + ch, ov / L);
         } else {
             float *op = outp + (size_t)j * PW;
             op[ch] = ov;
@@ -278,7 +278,7 @@ __device__ __forceinline__ int attention_splits(const Ctx &c, const Args &a) {
 
 // All blocks, after the grid barrier that follows the items: the splits of every
 // (sequence, head, row) merged by one warp each, into the bf16 attention output in
-// the fragment order the output projection reads.
+// the operand order the output projection reads.
 __device__ __forceinline__ void phase_attention_merge(Ctx &c, const Args &a, int nsplit, int nt_total) {
     const int H = a.m.cfg.n_heads, hd = a.m.hd, PW = hd + 2, rps = a.g.rps;
     const int tasks = a.g.batch * H * rps;
@@ -302,7 +302,7 @@ __device__ __forceinline__ void phase_attention_merge(Ctx &c, const Args &a, int
 #pragma unroll
         for (int e = 0; e < 4; ++e)
             if (c.lane + 32 * e < hd)
-                store_split(a.d.att, a.fb.att_lo, xfrag_index(seq * rps + j, h * hd + c.lane + 32 * e, nt_total), ov[e] * inv);
+                store_split(a.d.att, nt_total, seq * rps + j, h * hd + c.lane + 32 * e, ov[e] * inv);
     }
 }
 

@@ -137,15 +137,22 @@ __device__ __forceinline__ void tail_ar(Ctx &c, const Args &a, int s) {
 template <int NT>
 __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ Args a, const int which) {
     extern __shared__ __align__(1024) unsigned char smem[];
+    if (smem_u32(smem) & 1023u) {           // the swizzled operand layout needs this alignment (the same in every block)
+        if (threadIdx.x == 0) atomicCAS(a.fb.abort_flag, 0, 13);
+        return;
+    }
     Ctx c;
     c.warp = threadIdx.x >> 5; c.lane = threadIdx.x & 31; c.cta = blockIdx.x; c.ncta = gridDim.x;
     c.scratch = smem;
     c.ring = smem + SCRATCH_BYTES;
     unsigned char *misc = smem + SCRATCH_BYTES + RING_BYTES;
-    c.wfull = reinterpret_cast<uint64_t *>(misc);                            // NS
-    c.wempty = c.wfull + NS;                                                 // NS
-    c.xfull = c.wempty + NS;                                                 // XS_MAX
-    c.xempty = c.xfull + XS_MAX;                                             // XS_MAX  (ends at 8 * (2*NS + 2*XS_MAX) <= 320)
+    c.wfull = reinterpret_cast<uint64_t *>(misc);                            // NB
+    c.wempty = c.wfull + NB;                                                 // NB
+    c.xfull = c.wempty + NB;                                                 // XS_MAX
+    c.xempty = c.xfull + XS_MAX;                                             // XS_MAX
+    c.acc_full = c.xempty + XS_MAX;
+    c.acc_empty = c.acc_full + 1;                                            // ends at 8 * (2*NB + 2*XS_MAX + 2) = 320
+    static_assert(8 * (2 * NB + 2 * XS_MAX + 2) <= 320, "barriers overlap the row tables");
     c.row_pos = reinterpret_cast<int32_t *>(misc + 320);
     c.row_tok = c.row_pos + MAX_ROWS;
     c.n_rows = c.row_tok + MAX_ROWS;
@@ -155,8 +162,11 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
     float **row_dst = reinterpret_cast<float **>(misc + 1024);               // [MAX_ROWS]
     int32_t *bias_at = reinterpret_cast<int32_t *>(misc + 1024 + 256);       // [MAX_ROWS]
     Top2 *top_sm = reinterpret_cast<Top2 *>(misc + 1024 + 384);              // [8]
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(misc + 1536);
+    c.pass_done = reinterpret_cast<volatile int32_t *>(misc + 1540);
     c.bar_target = 0;
-    c.wn = c.xn = 0;
+    c.np = 0;
+    c.tmem = 0;
     c.policy = policy_evict_first();
     const DevPtrs &d = a.d;
     const ModelDev &m = a.m;
@@ -208,16 +218,33 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
     if (threadIdx.x == 0) {
         const unsigned long long v = ld_acquire_u64(a.fb.bar);
         c.bar_target = v / (unsigned long long)c.ncta * (unsigned long long)c.ncta;
-        for (int i = 0; i < NS; ++i) { mbar_init(c.wfull + i, 1); mbar_init(c.wempty + i, 1); }
-        for (int i = 0; i < XS_MAX; ++i) { mbar_init(c.xfull + i, 1); mbar_init(c.xempty + i, MMA_WARPS); }
+        for (int i = 0; i < NB; ++i) { mbar_init(c.wfull + i, 1); mbar_init(c.wempty + i, 1); }
+        for (int i = 0; i < XS_MAX; ++i) { mbar_init(c.xfull + i, 1); mbar_init(c.xempty + i, 1); }
+        mbar_init(c.acc_full, 1); mbar_init(c.acc_empty, 1);
         c.ready_op[0] = 0; c.ready_op[1] = 0;
+        *c.pass_done = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    if (c.warp == MMA_ISSUER) {             // the accumulator's tensor memory, held until the end of the kernel
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
     fence_proxy_async();
+    tc_fence_before();
     __syncthreads();
+    tc_fence_after();
+    c.tmem = *tmem_slot;
 
-    // the two producer warps live in their streams until the forward's last unit
-    if (c.warp >= W_PRODUCER && c.warp < X_PRODUCER) { weight_producer(c, a.fb, a.P, c.warp - W_PRODUCER); return; }
+    // the producer warps live in their streams until the forward's last stage
+    if (c.warp == W_PRODUCER) { if (c.lane == 0) weight_producer(c, a.fb, a.P); return; }
+    if (c.warp == MMA_ISSUER) {
+        if (c.lane == 0) mma_issuer<NT>(c, a.fb, a.P);
+        __syncwarp();
+        asm volatile("bar.sync 2, 288;" ::: "memory");        // the phase warps have read their last accumulator
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(c.tmem), "r"(TMEM_COLS) : "memory");
+        return;
+    }
+    if (c.warp > MMA_ISSUER && c.warp < X_PRODUCER) return;
     if (c.warp == X_PRODUCER + X_PRODUCERS - 1) { helper_warp(c, a.fb, a.P, m.cfg.d_model, m.cfg.rms_eps); return; }
     if (c.warp >= X_PRODUCER) {
         uint64_t keep;
@@ -316,6 +343,8 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
         else if (kind == KIND_PREFILL || kind == KIND_PREFILL_B) tail_prefill(c, a, c.cta, which);
     }
     stamp();
+    tc_fence_before();
+    asm volatile("bar.sync 2, 288;" ::: "memory");            // lets the owner release the tensor memory
 }
 
 }  // namespace fwd
@@ -330,10 +359,10 @@ static inline Plan make_plan(const ModelDev &m, const DevPtrs &d, const FwdBufs 
     const pacer_model_cfg &k = m.cfg;
     const long long dm = k.d_model, F = k.d_ffn, hh = (long long)k.n_heads * m.hd;
     int rot = 0;
-    auto set = [&](int i, const bf16 *w1, const bf16 *w2, const bf16 *x, long long x_lo, long long lstride, int N, int K, int MT,
-                   int inter) {
+    auto set = [&](int i, const bf16 *w, const bf16 *x, int N, int K, int MT) {
         GemmOp &o = P.op[i];
-        o.W1 = w1; o.W2 = w2 ? w2 : w1; o.X = x; o.x_lo = x_lo; o.lstride = lstride; o.N = N; o.K = K; o.MT = MT; o.interleave = inter;
+        o.W = w; o.X = x; o.N = N; o.K = K; o.MT = MT;
+        o.lstride = (long long)(K / KB) * (2 * MT) * 512;
         o.S = 1;
         // few tiles and enough bytes to be bandwidth bound: also cut along k, so that a block needs less of the
         // activations (a small projection is latency bound and better off without the extra pass and barrier)
@@ -345,11 +374,12 @@ static inline Plan make_plan(const ModelDev &m, const DevPtrs &d, const FwdBufs 
         o.rot = rot;
         rot = (rot + (MT % (ncta / o.S)) * o.S) % ncta;       // the next projection's extra tiles go to other blocks
     };
-    set(OP_QKV, m.wqkv, nullptr, fb.xg, fb.xg_lo, (long long)m.qrows * dm, m.qrows, (int)dm, (m.qrows + 15) / 16, 0);
-    set(OP_O, m.wo, nullptr, d.att, fb.att_lo, dm * hh, (int)dm, (int)hh, ((int)dm + 15) / 16, 0);
-    set(OP_GU, m.wgate, m.wup, fb.xg, fb.xg_lo, F * dm, (int)(2 * F), (int)dm, ((int)F + 7) / 8, 1);
-    set(OP_DOWN, m.wdown, nullptr, d.act, fb.act_lo, dm * F, (int)dm, (int)F, ((int)dm + 15) / 16, 0);
-    set(OP_HEAD, m.head, nullptr, fb.xg, fb.xg_lo, 0, k.vocab, (int)dm, (k.vocab + 15) / 16, 0);
+    set(OP_QKV, m.wt[OP_QKV], fb.xg, m.qrows, (int)dm, (m.qrows + 15) / 16);
+    set(OP_O, m.wt[OP_O], d.att, (int)dm, (int)hh, ((int)dm + 15) / 16);
+    set(OP_GU, m.wt[OP_GU], fb.xg, (int)(2 * F), (int)dm, ((int)F + 7) / 8);
+    set(OP_DOWN, m.wt[OP_DOWN], d.act, (int)dm, (int)F, ((int)dm + 15) / 16);
+    set(OP_HEAD, m.wt[OP_HEAD], fb.xg, k.vocab, (int)dm, (k.vocab + 15) / 16);
+    P.op[OP_HEAD].lstride = 0;
     P.n_layers = k.n_layers;
     P.has_head = has_head ? 1 : 0;
     return P;

@@ -72,8 +72,8 @@ __device__ __forceinline__ RowDesc row_desc(int kind, const DevPtrs &d, int s, i
 
 // x = embedding row (or h + e for the pre-verification model, or the draft's
 // hidden row during its prefill), spread over the MMA warps of the grid by
-// 16-column tiles.  Leaves x (fp32), x * gain of the first RMSNorm (bf16,
-// fragment order) and the per-tile sums of squares.
+// 16-column tiles.  Leaves x (fp32), x * gain of the first RMSNorm (split bf16,
+// operand order) and the per-tile sums of squares.
 __device__ __forceinline__ void phase_begin(Ctx &c, const Args &a, int nt_total) {
     const DevPtrs &d = a.d;
     const ModelDev &m = a.m;
@@ -98,7 +98,7 @@ __device__ __forceinline__ void phase_begin(Ctx &c, const Args &a, int nt_total)
                 }
             }
             d.xres[(size_t)r * dm + col] = v;          // idle rows hold zeros: they stay finite through the layers
-            store_split(a.fb.xg, a.fb.xg_lo, xfrag_index(r, col, nt_total), v * gain);
+            store_split(a.fb.xg, nt_total, r, col, v * gain);
             float ss = v * v;
 #pragma unroll
             for (int o = 8; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
@@ -127,7 +127,7 @@ __device__ __forceinline__ void epi_qkv(Ctx &c, const Args &a, int tile, float (
 
 // Tile of the attention-output / down projection.  The accumulators started from
 // the residual rows, so they hold the new x: store it, store x * gain of the
-// RMSNorm that follows as bf16 in fragment order (the next projection's input),
+// RMSNorm that follows as split bf16 in operand order (the next projection's input),
 // and the tile's share of sum(x^2) per row.
 template <int NT>
 __device__ __forceinline__ void epi_residual(Ctx &c, const Args &a, const bf16 *gain_next, int tile, float (&acc)[NT][4]) {
@@ -144,12 +144,12 @@ __device__ __forceinline__ void epi_residual(Ctx &c, const Args &a, const bf16 *
             if (n0 < dm) {
                 const float v = acc[nt][i];
                 x[n0] = v; ss[i] += v * v;
-                store_split(a.fb.xg, a.fb.xg_lo, xfrag_index(r, n0, NT), v * g0);
+                store_split(a.fb.xg, NT, r, n0, v * g0);
             }
             if (n1 < dm) {
                 const float v = acc[nt][2 + i];
                 x[n1] = v; ss[i] += v * v;
-                store_split(a.fb.xg, a.fb.xg_lo, xfrag_index(r, n1, NT), v * g1);
+                store_split(a.fb.xg, NT, r, n1, v * g1);
             }
         }
 #pragma unroll
@@ -181,7 +181,7 @@ __device__ __forceinline__ void epi_partial(Ctx &c, const Args &a, const GemmOp 
 
 // After the grid barrier that completes the partials of a k-sliced residual
 // projection: x += the slices' sums (slice order, so the result does not depend
-// on timing); x * gain of the next RMSNorm as bf16 fragments; sum(x^2) per tile.
+// on timing); x * gain of the next RMSNorm as split bf16; sum(x^2) per tile.
 // Spread over the MMA warps of the grid by 16-column tiles.
 template <int NT>
 __device__ __forceinline__ void phase_residual(Ctx &c, const Args &a, const GemmOp &op, const bf16 *gain_next) {
@@ -211,7 +211,7 @@ __device__ __forceinline__ void phase_residual(Ctx &c, const Args &a, const Gemm
         for (int it = 0; it < NIT; ++it) {
             const int r = 2 * it + half;
             a.d.xres[(size_t)r * dm + col] = v[it];
-            store_split(a.fb.xg, a.fb.xg_lo, xfrag_index(r, col, NT), v[it] * gain);
+            store_split(a.fb.xg, NT, r, col, v[it] * gain);
             float ss = v[it] * v[it];
 #pragma unroll
             for (int o = 8; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
@@ -222,7 +222,7 @@ __device__ __forceinline__ void phase_residual(Ctx &c, const Args &a, const Gemm
 
 // Interleaved gate/up tile: rows 0..7 are gate rows f = 8*tile + g, rows 8..15 the
 // up rows of the same f, so a lane holds both; 1/rms of the input RMSNorm, then
-// silu(gate) * up as bf16 in the fragment order the down projection reads.
+// silu(gate) * up as split bf16 in the operand order the down projection reads.
 template <int NT>
 __device__ __forceinline__ void epi_swiglu(Ctx &c, const Args &a, int tile, float (&acc)[NT][4]) {
     const int g = c.lane >> 2, t = c.lane & 3, F = a.m.cfg.d_ffn;
@@ -236,7 +236,7 @@ __device__ __forceinline__ void epi_swiglu(Ctx &c, const Args &a, int tile, floa
             const float inv = c.inv_rms[r];
             const float gt = acc[nt][i] * inv, up = acc[nt][2 + i] * inv;
             const float v = (r < a.g.rtot && c.row_pos[r] >= 0) ? gt / (1.f + expf(-gt)) * up : 0.f;
-            store_split(a.d.act, a.fb.act_lo, xfrag_index(r, f, NT), v);
+            store_split(a.d.act, NT, r, f, v);
         }
     }
 }

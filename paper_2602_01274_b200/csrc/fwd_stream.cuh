@@ -1,11 +1,13 @@
-// Weight and activation streams of the forward kernel: the two producer warps
-// and the projection loop of the MMA warps.
+// Weight and activation streams of the forward kernel: the producer threads, the
+// thread that issues the tensor-core instructions, and the projection loop of the
+// phase warps.
 //
-// Order of everything, identical on both sides: projections q = 0, 1, ... of the
+// Order of everything, identical on all sides: projections q = 0, 1, ... of the
 // forward (four per layer, then the LM head); inside a projection the passes of
-// this block (at most MAX_TILES tiles each, evenly sized); inside a pass the k steps of KC
-// columns; inside a k step the tiles of the pass.  Weight unit number n of the
-// block lives in ring stage n % NS, activation chunk number m in stage m % XS.
+// this block (at most MAX_TILES tiles each, evenly sized); inside a pass the k
+// blocks of KB columns.  Weight stage number n of the block (one k block of the
+// pass's rows) uses barrier pair n % NB and the next free bytes of the ring;
+// activation stage number m (XK columns) lives in stage m % XS.
 #pragma once
 #include "forward.cuh"
 
@@ -45,39 +47,77 @@ __device__ __forceinline__ int n_ops(const Plan &P) { return 4 * P.n_layers + (P
 __device__ __forceinline__ int op_index(const Plan &P, int q) { return q < 4 * P.n_layers ? (q & 3) : OP_HEAD; }
 __device__ __forceinline__ int op_layer(const Plan &P, int q) { return q < 4 * P.n_layers ? (q >> 2) : 0; }
 
-// Warps W_PRODUCER ..: every weight unit of the block, for the whole forward, in
-// order; producer `me` issues the units n with n % W_PRODUCERS == me.
-__device__ __forceinline__ void weight_producer(Ctx &c, const FwdBufs &fb, const Plan &P, int me) {
-    int n = 0;
+// Placement of the stages in the byte ring: each takes the next `bytes` (a multiple of 1 KB), starting over at
+// the ring's base when it would run past the end.  The producer and the MMA thread replay the same sequence.
+__device__ __forceinline__ int ring_place(int &head, int bytes) {
+    if (head + bytes > RING_BYTES) head = 0;
+    const int at = head;
+    head += bytes;
+    return at;
+}
+
+// Lane 0 of warp W_PRODUCER: every weight stage of the block, for the whole forward, in order.  A stage may
+// be written once every earlier stage that overlaps its bytes has been released (stages are released in order).
+__device__ __forceinline__ void weight_producer(Ctx &c, const FwdBufs &fb, const Plan &P) {
+    int n = 0, tail = 0, head = 0;
+    int q_s[NB], q_e[NB];
     for (int q = 0; q < n_ops(P); ++q) {
         const GemmOp &op = P.op[op_index(P, q)];
-        const size_t lbase = (size_t)op_layer(P, q) * op.lstride;
+        const bf16 *wl = op.W + (size_t)op_layer(P, q) * op.lstride;
         int t0, T, k_lo, k_hi;
         op_range(op, c.cta, c.ncta, t0, T, k_lo, k_hi);
         for (int p = 0; p < n_passes(T); ++p) {
             int p0, Tp;
             pass_range(T, p, p0, Tp);
-            for (int k = k_lo; k < k_hi; k += KC) {
-                const uint32_t bytes = (uint32_t)min(KC, k_hi - k) * 2u;
-                for (int i = 0; i < Tp; ++i, ++n) {
-                    if (n % W_PRODUCERS != me) continue;
-                    const int slot = n % NS, tile = t0 + p0 + i;
-                    if (!wait_bar(fb, c.wempty + slot, (((uint32_t)(n / NS)) & 1u) ^ 1u, 5, n)) return;   // stop feeding
-                    if (c.lane == 0) mbar_expect_tx(c.wfull + slot, 16u * bytes);
-                    __syncwarp();
-                    if (c.lane < 16) {
-                        const bf16 *src;
-                        if (op.interleave) {
-                            const int f = min(tile * 8 + (c.lane & 7), (op.N >> 1) - 1);
-                            src = (c.lane < 8 ? op.W1 : op.W2) + lbase + (size_t)f * op.K + k;
-                        } else {
-                            const int nrow = min(tile * 16 + c.lane, op.N - 1);
-                            src = op.W1 + lbase + (size_t)nrow * op.K + k;
-                        }
-                        bulk_g2s(c.ring + slot * STAGE_BYTES + c.lane * PITCH, src, bytes, c.wfull + slot, c.policy);
-                    }
-                }
+            const int bytes = Tp * 2048;                 // two 8-row atoms per tile
+            for (int k = k_lo; k < k_hi; k += KB, ++n) {
+                const int at = ring_place(head, bytes), end = at + bytes;
+                int need = n - tail >= NB ? tail + 1 : tail;
+                for (int j = tail; j < n; ++j)
+                    if (q_s[j % NB] < end && at < q_e[j % NB]) need = j + 1;
+                for (; tail < need; ++tail)
+                    if (!wait_bar(fb, c.wempty + tail % NB, ((uint32_t)(tail / NB)) & 1u, 5, tail)) return;   // stop feeding
+                q_s[n % NB] = at; q_e[n % NB] = end;
+                mbar_expect_tx(c.wfull + n % NB, (uint32_t)bytes);
+                bulk_g2s(c.ring + at, wl + ((size_t)(k >> 6) * (2 * op.MT) + 2 * (t0 + p0)) * 512, (uint32_t)bytes, c.wfull + n % NB,
+                         c.policy);
             }
+        }
+    }
+}
+
+// Lane 0 of warp MMA_ISSUER: the tensor-core instructions of every stage.  Per k block four MMAs of K = 16; the
+// A operand is the activation stage (128 rows are read from its base: values, remainders, then whatever follows
+// in shared memory, which only reaches accumulator lanes nobody reads), the B operand the weight stage.
+template <int NT>
+__device__ __forceinline__ void mma_issuer(Ctx &c, const FwdBufs &fb, const Plan &P) {
+    constexpr int XS = x_stages(NT), XSTAGE_BYTES = xstage_bytes(NT), XKB_BYTES = 2 * NT * 1024;
+    int n = 0, head = 0, m = 0, np = 0;
+    for (int q = 0; q < n_ops(P); ++q) {
+        const GemmOp &op = P.op[op_index(P, q)];
+        int t0, T, k_lo, k_hi;
+        op_range(op, c.cta, c.ncta, t0, T, k_lo, k_hi);
+        for (int p = 0; p < n_passes(T); ++p, ++np) {
+            int p0, Tp;
+            pass_range(T, p, p0, Tp);
+            const int bytes = Tp * 2048;
+            const uint32_t idesc = umma_idesc(Tp * 16);
+            // the phase warps have copied the previous pass's accumulator out
+            if (!wait_bar(fb, c.acc_empty, (((uint32_t)np) & 1u) ^ 1u, 11, np)) return;
+            for (int k = k_lo; k < k_hi; k += KB, ++n) {
+                const int kx = (k - k_lo) % XK, xslot = m % XS;
+                if (kx == 0 && !wait_bar(fb, c.xfull + xslot, ((uint32_t)(m / XS)) & 1u, 8, m)) return;
+                const int at = ring_place(head, bytes);
+                if (!wait_bar(fb, c.wfull + n % NB, ((uint32_t)(n / NB)) & 1u, 9, n)) return;
+                tc_fence_after();
+                const uint32_t a0 = smem_u32(c.scratch + xslot * XSTAGE_BYTES + (kx / KB) * XKB_BYTES), b0 = smem_u32(c.ring + at);
+#pragma unroll
+                for (int k16 = 0; k16 < 4; ++k16)
+                    umma(c.tmem, umma_desc(a0 + k16 * 32), umma_desc(b0 + k16 * 32), idesc, (k > k_lo || k16 > 0) ? 1u : 0u);
+                umma_commit(c.wempty + n % NB);
+                if (kx == XK - KB || k + KB >= k_hi) { umma_commit(c.xempty + xslot); ++m; }
+            }
+            umma_commit(c.acc_full);
         }
     }
 }
@@ -105,15 +145,15 @@ __device__ __forceinline__ void compute_inv(Ctx &c, const FwdBufs &fb, int dm, f
     __syncwarp();
 }
 
-// Warps X_PRODUCER .. X_PRODUCER + XS - 1: the activation chunk of every k step,
-// once the projection's inputs are complete (the MMA warps raise ready_op[0] after
-// the grid barrier): a bulk copy of a bf16 buffer that already has fragment order.
-// Stage s is fed by producer s, so its generations stay in order.
+// Warps X_PRODUCER .. X_PRODUCER + XS - 1: the activation stage of every XK columns, once the projection's
+// inputs are complete (the phase warps raise ready_op[0] after the grid barrier): one bulk copy of a buffer that
+// already has operand order.  Stage s is fed by producer s, so its generations stay in order.  A later pass of
+// the same projection starts once the epilogue of the pass before is over (it uses the ring's bytes).
 template <int NT>
 __device__ __forceinline__ void activation_producer(Ctx &c, const FwdBufs &fb, const Plan &P, int me, uint64_t keep_policy) {
     constexpr int XS = x_stages(NT), XSTAGE_BYTES = xstage_bytes(NT);
     if (me >= XS) return;
-    int m = 0;
+    int m = 0, np = 0;
     for (int q = 0; q < n_ops(P); ++q) {
         const GemmOp &op = P.op[op_index(P, q)];
         int t0, T, k_lo, k_hi;
@@ -122,18 +162,20 @@ __device__ __forceinline__ void activation_producer(Ctx &c, const FwdBufs &fb, c
         wait_count(fb, c.ready_op, q + 1, 6);
         __threadfence_block();
         asm volatile("fence.proxy.async;" ::: "memory");
-        for (int p = 0; p < n_passes(T); ++p) {
+        for (int p = 0; p < n_passes(T); ++p, ++np) {
+            if (p > 0) {
+                wait_count(fb, c.pass_done, np, 12);
+                __threadfence_block();
+                asm volatile("fence.proxy.async;" ::: "memory");
+            }
             for (int k = k_lo; k < k_hi; k += XK, ++m) {
                 if (m % XS != me) continue;
-                const int slot = m % XS, nch = min(XK, k_hi - k) >> 5;
+                const int slot = m % XS, nkb = min(XK, k_hi - k) / KB;
                 if (!wait_bar(fb, c.xempty + slot, (((uint32_t)(m / XS)) & 1u) ^ 1u, 7, m)) return;
-                if (c.lane == 0) {                       // the chunk's bf16 values, then its rounding remainders
-                    const uint32_t bytes = (uint32_t)nch * (uint32_t)NT * 512u;
-                    const bf16 *src = op.X + (size_t)(k >> 5) * NT * 256;
-                    unsigned char *dst = c.scratch + slot * XSTAGE_BYTES;
-                    mbar_expect_tx(c.xfull + slot, 2u * bytes);
-                    bulk_g2s(dst, src, bytes, c.xfull + slot, keep_policy);
-                    bulk_g2s(dst + XSTAGE_BYTES / 2, src + op.x_lo, bytes, c.xfull + slot, keep_policy);
+                if (c.lane == 0) {
+                    const uint32_t bytes = (uint32_t)nkb * 2u * NT * 1024u;
+                    mbar_expect_tx(c.xfull + slot, bytes);
+                    bulk_g2s(c.scratch + slot * XSTAGE_BYTES, op.X + (size_t)(k >> 6) * (2 * NT * 512), bytes, c.xfull + slot, keep_policy);
                 }
                 __syncwarp();
             }
@@ -159,33 +201,11 @@ __device__ __forceinline__ void helper_warp(Ctx &c, const FwdBufs &fb, const Pla
     }
 }
 
-// acc[nt] += W(16 rows x 32*nchunks k, from chunk `chunk0` of the stage) * (X_hi + X_lo).  Lane (g, t) reads the
-// 8 consecutive weights of rows g and g+8 at k = 32c + 8t and uses them as the k slots {2t, 2t+1, 2t+8, 2t+9}
-// of two MMAs; the activation fragments are stored with the same rule, so the products pair up.
-template <int NT>
-__device__ __forceinline__ void consume_unit(const unsigned char *stage, int chunk0, const uint4 *xhi, const uint4 *xlo, int nchunks,
-                                             float (&acc)[NT][4], int lane) {
-    const int g = lane >> 2, t = lane & 3;
-    const unsigned char *p0 = stage + g * PITCH + t * 16 + chunk0 * 64, *p1 = p0 + 8 * PITCH;
-#pragma unroll 2
-    for (int cix = 0; cix < nchunks; ++cix) {
-        const uint4 a0 = *reinterpret_cast<const uint4 *>(p0 + cix * 64);
-        const uint4 a1 = *reinterpret_cast<const uint4 *>(p1 + cix * 64);
-#pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {
-            const uint4 bh = xhi[(cix * NT + nt) * 32 + lane], bl = xlo[(cix * NT + nt) * 32 + lane];
-            mma16816(acc[nt], a0.x, a1.x, a0.y, a1.y, bh.x, bh.y);
-            mma16816(acc[nt], a0.z, a1.z, a0.w, a1.w, bh.z, bh.w);
-            mma16816(acc[nt], a0.x, a1.x, a0.y, a1.y, bl.x, bl.y);
-            mma16816(acc[nt], a0.z, a1.z, a0.w, a1.w, bl.z, bl.w);
-        }
-    }
-}
-
-// One projection, run by the eight MMA warps after the grid barrier that
-// completed its inputs.  Warp w owns tile w of every pass, over the block's k
-// range; epi(tile, acc) gets the sums.
-// Accumulator element (nt, i): token row nt*8 + 2t + (i & 1), tile column g + 8*(i >> 1).
+// One projection, run by the eight phase warps after the grid barrier that completed its inputs: per pass they
+// wait for the accumulator, copy its lanes (values part, remainders part) from tensor memory to shared memory,
+// and run epi(tile, acc) for the pass's 16-row tiles, warp w taking tiles w, w + 8.
+// Accumulator element (nt, i) as the epilogues see it: token row nt*8 + 2t + (i & 1), tile column g + 8*(i >> 1),
+// with g = lane / 4, t = lane % 4.  resid: rows added to the sums (the residual stream), or NULL.
 template <int NT, class Epi>
 __device__ __forceinline__ void gemm_op(Ctx &c, const FwdBufs &fb, const Plan &P, int q, const float *resid, int resid_ld,
                                         Epi epi) {
@@ -198,58 +218,55 @@ __device__ __forceinline__ void gemm_op(Ctx &c, const FwdBufs &fb, const Plan &P
     const bool normed = opi == OP_QKV || opi == OP_GU || opi == OP_HEAD;
     int t0, T, k_lo, k_hi;
     op_range(op, c.cta, c.ncta, t0, T, k_lo, k_hi);
-    constexpr int XS = x_stages(NT), XSTAGE_BYTES = xstage_bytes(NT);
+    float *stage = reinterpret_cast<float *>(c.scratch);
+    const int g = c.lane >> 2, t = c.lane & 3;
     for (int p = 0; p < n_passes(T); ++p) {
         int p0, Tp;
         pass_range(T, p, p0, Tp);
-        const bool has = c.warp < Tp;
-        // Accumulators start from the residual rows when the projection adds into the residual stream: the
-        // loads are issued before the k loop, so the epilogue has no global round trip of its own.
-        float acc[NT][4];
+        const int C = Tp * 16, pitch = C + 1;               // odd pitch: a warp's 32 lanes (rows) hit 32 banks
+        wait_bar(fb, c.acc_full, ((uint32_t)c.np) & 1u, 10, c.np);
+        tc_fence_after();
         {
-            const int g = c.lane >> 2, t = c.lane & 3;
+            const int quad = c.warp & 3;                     // the accumulator lanes this warp can read: 32 quad ..
+            if (quad * 32 < 16 * NT) {
+                for (int cg = c.warp >> 2; cg * 32 < C; cg += 2) {
+                    uint32_t v[32];
+                    tmem_ld32(c.tmem + ((uint32_t)(quad * 32) << 16) + (uint32_t)(cg * 32), v);
+                    float *row = stage + (size_t)(quad * 32 + c.lane) * pitch + cg * 32;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (cg * 32 + j < C) row[j] = __uint_as_float(v[j]);
+                }
+            }
+        }
+        tc_fence_before();
+        bsync();
+        if (threadIdx.x == 0) mbar_arrive(c.acc_empty);       // the next pass may overwrite the accumulator
+        if (normed) {
+            wait_count(fb, c.ready_op + 1, q + 1, 10);                 // 1/rms of this projection's input rows
+            __threadfence_block();
+        }
+        for (int ti = c.warp; ti < Tp; ti += MMA_WARPS) {
+            const int tile = t0 + p0 + ti;
+            float acc[NT][4];
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
-                    acc[nt][i] = 0.f;
-                    if (resid && has) {
-                        const int r = nt * 8 + 2 * t + (i & 1), n0 = (t0 + p0 + c.warp) * 16 + g + 8 * (i >> 1);
-                        if (n0 < op.N) acc[nt][i] = __ldcg(resid + (size_t)r * resid_ld + n0);
+                    const int r = nt * 8 + 2 * t + (i & 1), cc = ti * 16 + g + 8 * (i >> 1);
+                    float v = stage[(size_t)r * pitch + cc] + stage[(size_t)(8 * NT + r) * pitch + cc];
+                    if (resid) {
+                        const int n0 = tile * 16 + g + 8 * (i >> 1);
+                        if (n0 < op.N) v += __ldcg(resid + (size_t)r * resid_ld + n0);
                     }
+                    acc[nt][i] = v;
                 }
+            epi(tile, acc);
         }
-        for (int k = k_lo; k < k_hi; k += KC) {
-            const int nch = min(KC, k_hi - k) >> 5;
-            int slot = 0;
-            if (has) {
-                const int n = c.wn + c.warp;
-                slot = n % NS;
-                wait_bar(fb, c.wfull + slot, ((uint32_t)(n / NS)) & 1u, 9, n);
-            }
-            for (int c0 = 0; c0 < nch; c0 += XCH) {           // the activations come in chunks of XK columns
-                const int xslot = c.xn % XS;
-                wait_bar(fb, c.xfull + xslot, ((uint32_t)(c.xn / XS)) & 1u, 8, c.xn);
-                if (has) {
-                    const uint4 *xhi = reinterpret_cast<const uint4 *>(c.scratch + xslot * XSTAGE_BYTES);
-                    consume_unit<NT>(c.ring + slot * STAGE_BYTES, c0, xhi, xhi + XSTAGE_BYTES / 32, min(XCH, nch - c0), acc, c.lane);
-                }
-                __syncwarp();
-                if (c.lane == 0) mbar_arrive(c.xempty + xslot);
-                ++c.xn;
-            }
-            if (has && c.lane == 0) mbar_arrive(c.wempty + slot);
-            // Lockstep over k.  A ring stage is shared by different warps over time, and a parity wait is exact
-            // only while the waiter is less than one stage generation ahead: a k step has at most NS units (and
-            // at most two activation chunks), so after this barrier the stage's previous user is done.
-            bsync();
-            c.wn += Tp;
-        }
-        if (normed && has) {
-            wait_count(fb, c.ready_op + 1, q + 1, 10);                 // 1/rms of this projection's input rows
-            __threadfence_block();
-        }
-        if (has) epi(t0 + p0 + c.warp, acc);
+        fence_proxy_async();                   // the copy in shared memory is read; bulk copies may overwrite it
+        bsync();
+        ++c.np;
+        if (threadIdx.x == 0) { __threadfence_block(); *c.pass_done = c.np; }
     }
 }
 

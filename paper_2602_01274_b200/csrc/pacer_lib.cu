@@ -82,7 +82,7 @@ static bool model_cfg_ok(const pacer_model_cfg &m) {
     const int hd = m.d_model / m.n_heads;
     if (hd != 64 && hd != 128) return false;
     if (m.n_heads % m.n_kv_heads) return false;
-    if (m.d_model % 32 || m.d_ffn % 32) return false;
+    if (m.d_model % 64 || m.d_ffn % 64) return false;     // the weight stages are 64 k columns wide
     return true;
 }
 
@@ -118,6 +118,7 @@ struct Layout {
     size_t row_pos, row_tok, n_rows, row_arg, row_margin, xres, att, act, hidden, part;
     size_t att_cnt, bar, abort_flag, qkv, xg, ssq, tile_top, attp, prof;
     size_t kc[3], vc[3], rope[3];
+    size_t wt[3][5], wt_bytes[3][5];   // the projections re-laid for the tensor cores
     size_t kv_bytes[3], rope_bytes[3];
     size_t total;
     int rtot_max, nt_max, max_steps, d_max, f_max;
@@ -192,6 +193,18 @@ static Layout make_layout(const pacer_cfg &c) {
         L.rope_bytes[i] = sizeof(float2) * (size_t)c.max_ctx * (hd / 2);
         L.rope[i] = cv.take(L.rope_bytes[i]);
     }
+    for (int i = 0; i < 3; ++i) {
+        const pacer_model_cfg &k = *ms[i];
+        const size_t hd = k.d_model / k.n_heads, qrows = (k.n_heads + 2 * (size_t)k.n_kv_heads) * hd, hh = k.n_heads * hd;
+        const size_t rows16[5] = {(qrows + 15) / 16, ((size_t)k.d_model + 15) / 16, ((size_t)k.d_ffn + 7) / 8,
+                                  ((size_t)k.d_model + 15) / 16, ((size_t)k.vocab + 15) / 16};       // 16-row tiles
+        const size_t kdim[5] = {(size_t)k.d_model, hh, (size_t)k.d_model, (size_t)k.d_ffn, (size_t)k.d_model};
+        for (int j = 0; j < 5; ++j) {
+            const size_t layers = j == 4 ? (i == 2 ? 0 : 1) : (size_t)k.n_layers;
+            L.wt_bytes[i][j] = layers * (kdim[j] / 64) * (2 * rows16[j]) * 1024;
+            L.wt[i][j] = cv.take(L.wt_bytes[i][j]);
+        }
+    }
     L.total = cv.off;
     return L;
 }
@@ -246,8 +259,6 @@ extern "C" int pacer_create(const pacer_cfg *cfg, void *dev_workspace, size_t wo
     d.q = nullptr; d.hidden = (float *)(w + L.hidden); d.part = (float *)(w + L.part);
     c->fb.qkv = (float *)(w + L.qkv); c->fb.xg = (bf16 *)(w + L.xg); c->fb.ssq = (float *)(w + L.ssq);
     c->fb.part = (float *)(w + L.part);
-    c->fb.xg_lo = c->fb.att_lo = (long long)fwd::MAX_ROWS * L.d_max;
-    c->fb.act_lo = (long long)fwd::MAX_ROWS * L.f_max;
     c->fb.tile_top = (float *)(w + L.tile_top); c->fb.attp = (float *)(w + L.attp);
     c->fb.att_cnt = (int32_t *)(w + L.att_cnt); c->fb.bar = (unsigned long long *)(w + L.bar);
     c->fb.abort_flag = (int32_t *)(w + L.abort_flag);
@@ -268,6 +279,7 @@ extern "C" int pacer_create(const pacer_cfg *cfg, void *dev_workspace, size_t wo
         m.kcache = (bf16 *)(w + L.kc[i]);
         m.vcache = (bf16 *)(w + L.vc[i]);
         m.kv_lo = L.kv_bytes[i] / (2 * sizeof(bf16));
+        for (int j = 0; j < 5; ++j) m.wt[j] = L.wt_bytes[i][j] ? (const bf16 *)(w + L.wt[i][j]) : nullptr;
         m.rope = (const float2 *)(w + L.rope[i]);
         const int half = m.hd / 2;
         c->rope_host[i].resize((size_t)cfg->max_ctx * half);
@@ -320,6 +332,27 @@ extern "C" int pacer_destroy(pacer_ctx *c) {
 
 // ------------------------------------------------------------------ weights
 
+// Re-lays one stack of [layers][N][K] row-major matrices into the order the forward kernel streams:
+// [layer][K/64][atoms][8 rows][64 k], an atom being 1 KB in the 128-byte swizzle layout of a K-major tensor-core
+// operand (the 16-byte chunk c of row r sits at chunk c ^ r).  Atom a holds rows 8a .. 8a+7 of W1, or, when W2 is
+// given (gate/up), rows 8(a/2) .. of W1 for even a and of W2 for odd a.  Rows past N are zeros.
+__global__ void k_retile(const bf16 *W1, const bf16 *W2, bf16 *out, int layers, int N, int K, int atoms) {
+    const size_t total = (size_t)layers * (K / 64) * atoms * 64;          // 16-byte chunks
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        const int ch = (int)(i & 7), r = (int)((i >> 3) & 7);
+        const size_t atom_lin = i >> 6;
+        const int a = (int)(atom_lin % atoms);
+        const size_t lk = atom_lin / atoms;
+        const int kb = (int)(lk % (K / 64)), layer = (int)(lk / (K / 64));
+        const bf16 *src = W1;
+        int row = a * 8 + r;
+        if (W2) { row = (a >> 1) * 8 + r; if (a & 1) src = W2; }
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (row < N) v = *reinterpret_cast<const uint4 *>(src + ((size_t)layer * N + row) * K + kb * 64 + ch * 8);
+        *reinterpret_cast<uint4 *>(out + atom_lin * 512 + r * 64 + ((ch ^ r) << 3)) = v;
+    }
+}
+
 extern "C" int pacer_load_weights(pacer_ctx *c, int which, const pacer_tensor *tbl, int n, const int32_t *succ) {
     if (!c || !tbl || which < 0 || which > 2 || n < 1) return fail(c, PACER_EINVAL, "pacer_load_weights: bad argument");
     ModelDev &m = c->model[which];
@@ -352,6 +385,23 @@ extern "C" int pacer_load_weights(pacer_ctx *c, int which, const pacer_tensor *t
     }
     for (auto &wn : want)
         if (wn.needed && !*wn.slot) return fail(c, PACER_EINVAL, std::string("pacer_load_weights: missing tensor ") + wn.name);
+    {
+        // the library's own copy of the five projections, in streaming order (the caller's matrices are not read again)
+        const int F = k.d_ffn;
+        struct Job { const bf16 *w1, *w2; int j, layers, N, K, atoms; };
+        const Job jobs[5] = {
+            {m.wqkv, nullptr, 0, (int)L, m.qrows, (int)d, 2 * ((m.qrows + 15) / 16)},
+            {m.wo, nullptr, 1, (int)L, (int)d, (int)hh, 2 * (((int)d + 15) / 16)},
+            {m.wgate, m.wup, 2, (int)L, F, (int)d, 2 * ((F + 7) / 8)},
+            {m.wdown, nullptr, 3, (int)L, (int)d, F, 2 * (((int)d + 15) / 16)},
+            {m.head, nullptr, 4, 1, (int)V, (int)d, 2 * (((int)V + 15) / 16)},
+        };
+        for (const Job &jb : jobs) {
+            if (!jb.w1 || !m.wt[jb.j]) continue;
+            k_retile<<<148 * 8, 256, 0, c->stream>>>(jb.w1, jb.w2, const_cast<bf16 *>(m.wt[jb.j]), jb.layers, jb.N, jb.K, jb.atoms);
+            CK(cudaGetLastError());
+        }
+    }
     m.succ = isB ? nullptr : succ;
     m.loaded = 1;
     c->plans.clear();
