@@ -34,10 +34,10 @@
 namespace fwd {
 
 constexpr int MMA_WARPS = 8, MMA_THREADS = 256;  // warps 0..7 ("phase warps"): epilogues and all block-wide phases
-constexpr int W_PRODUCER = 8;                    // warp 8, lane 0: the weight stream
+constexpr int W_PRODUCER = 8, W_PRODUCERS = 3;   // lane 0 of warps 8, 10, 11: the weight stream, stage n by producer n % 3
 constexpr int MMA_ISSUER = 9;                    // warp 9: owns the tensor memory; its lane 0 issues every tcgen05.mma
 constexpr int X_PRODUCER = 12, X_PRODUCERS = 4;  // warps 12..14 provide the activation stages (stage s by producer s);
-                                                 // warp 15 computes the RMS statistics; warps 10, 11 have no work
+                                                 // warp 15 computes the RMS statistics
 constexpr int THREADS = 32 * (X_PRODUCER + X_PRODUCERS);
 constexpr int KB = 64;                          // k columns of a weight stage: one 128-byte swizzle row
 constexpr int KC = 512;                         // k slices of a projection are whole multiples of this
@@ -84,7 +84,7 @@ struct Plan {
 
 // Device buffers of the forward kernel beyond DevPtrs (all in the workspace).
 struct FwdBufs {
-    float *qkv;              // [MAX_ROWS][qrows] fp32
+    float *qkv;              // [k slices][MAX_ROWS][qrows] fp32
     bf16 *xg;                // x * gain of the next RMSNorm, split bf16 in operand order (its 1/rms comes later)
     float *ssq;              // [d/16][MAX_ROWS] sum of squares of x over the 16 columns of a tile
     float *part;             // k-slice partial tiles [S][d/16][row tiles * 8][16] of the two residual projections

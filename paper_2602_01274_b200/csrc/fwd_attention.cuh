@@ -58,37 +58,61 @@ __device__ __forceinline__ void attention_rows(Ctx &c, const Args &a, int layer,
     bf16 *kn = reinterpret_cast<bf16 *>(c.scratch + SM::KN_OFF), *vn = reinterpret_cast<bf16 *>(c.scratch + SM::VN_OFF);
     const size_t cbase = (((size_t)layer * d.max_batch + seq) * Hkv + kh) * (size_t)d.max_ctx * HD;
     const float scale = rsqrtf((float)HD);
-    for (int i = threadIdx.x; i < 32 * half; i += MMA_THREADS) {
-        const int j = i / half, ii = i - j * half;
-        bf16 *qrow = reinterpret_cast<bf16 *>(c.scratch + SM::Q_OFF + j * SM::QP);
-        bf16 *qrow_lo = reinterpret_cast<bf16 *>(c.scratch + SM::Q_OFF + (32 + j) * SM::QP);
-        if (j < n_r) {
-            const int pos = pos0 + j;
-            const float *row = a.fb.qkv + (size_t)(r_base + j) * qrows;
-            const float2 cs = m.rope[(size_t)pos * half + ii];
-            const float qa = __ldcg(row + h * HD + ii), qb = __ldcg(row + h * HD + ii + half);
-            split_bf16((qa * cs.x - qb * cs.y) * scale, qrow[ii], qrow_lo[ii]);
-            split_bf16((qb * cs.x + qa * cs.y) * scale, qrow[ii + half], qrow_lo[ii + half]);
-            const float ka = __ldcg(row + (H + kh) * HD + ii), kb = __ldcg(row + (H + kh) * HD + ii + half);
-            bf16 k0, k0l, k1, k1l, v0, v0l, v1, v1l;
-            split_bf16(ka * cs.x - kb * cs.y, k0, k0l);
-            split_bf16(kb * cs.x + ka * cs.y, k1, k1l);
-            split_bf16(__ldcg(row + (H + Hkv + kh) * HD + ii), v0, v0l);
-            split_bf16(__ldcg(row + (H + Hkv + kh) * HD + ii + half), v1, v1l);
-            kn[j * HD + ii] = k0; kn[j * HD + ii + half] = k1;
-            kn[(32 + j) * HD + ii] = k0l; kn[(32 + j) * HD + ii + half] = k1l;
-            vn[j * HD + ii] = v0; vn[j * HD + ii + half] = v1;
-            vn[(32 + j) * HD + ii] = v0l; vn[(32 + j) * HD + ii + half] = v1l;
-            if (writer) {
-                bf16 *kc = m.kcache + cbase + (size_t)pos * HD, *vc = m.vcache + cbase + (size_t)pos * HD;
-                kc[ii] = k0; kc[ii + half] = k1;
-                kc[m.kv_lo + ii] = k0l; kc[m.kv_lo + ii + half] = k1l;
-                vc[ii] = v0; vc[ii + half] = v1;
-                vc[m.kv_lo + ii] = v0l; vc[m.kv_lo + ii + half] = v1l;
+    // The projection may have been cut along k: every value is the sum of the slices' shares.  Two elements per
+    // thread at a time, all their loads issued before the first use (the phase is bound by load latency).
+    const int S = a.P.op[OP_QKV].S;
+    const size_t sl = (size_t)MAX_ROWS * qrows;
+    constexpr int U = 2;
+    for (int i0 = threadIdx.x; i0 < 32 * half; i0 += U * MMA_THREADS) {
+        float part[U][4][6];
+        float2 cs[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int i = i0 + u * MMA_THREADS, j = i / half, ii = i - j * half;
+            const bool on = i < 32 * half && j < n_r;
+            const float *row = a.fb.qkv + (size_t)(r_base + (on ? j : 0)) * qrows;
+            const int col[6] = {h * HD + ii, h * HD + ii + half, (H + kh) * HD + ii, (H + kh) * HD + ii + half,
+                                (H + Hkv + kh) * HD + ii, (H + Hkv + kh) * HD + ii + half};
+            cs[u] = on ? m.rope[(size_t)(pos0 + j) * half + ii] : make_float2(0.f, 0.f);
+#pragma unroll
+            for (int s = 0; s < 4; ++s)
+#pragma unroll
+                for (int e = 0; e < 6; ++e) part[u][s][e] = (on && s < S) ? __ldcg(row + s * sl + col[e]) : 0.f;
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int i = i0 + u * MMA_THREADS, j = i / half, ii = i - j * half;
+            if (i >= 32 * half) continue;
+            bf16 *qrow = reinterpret_cast<bf16 *>(c.scratch + SM::Q_OFF + j * SM::QP);
+            bf16 *qrow_lo = reinterpret_cast<bf16 *>(c.scratch + SM::Q_OFF + (32 + j) * SM::QP);
+            if (j < n_r) {
+                const int pos = pos0 + j;
+                float in[6];
+#pragma unroll
+                for (int e = 0; e < 6; ++e) in[e] = (part[u][0][e] + part[u][1][e]) + (part[u][2][e] + part[u][3][e]);
+                const float qa = in[0], qb = in[1], ka = in[2], kb = in[3];
+                split_bf16((qa * cs[u].x - qb * cs[u].y) * scale, qrow[ii], qrow_lo[ii]);
+                split_bf16((qb * cs[u].x + qa * cs[u].y) * scale, qrow[ii + half], qrow_lo[ii + half]);
+                bf16 k0, k0l, k1, k1l, v0, v0l, v1, v1l;
+                split_bf16(ka * cs[u].x - kb * cs[u].y, k0, k0l);
+                split_bf16(kb * cs[u].x + ka * cs[u].y, k1, k1l);
+                split_bf16(in[4], v0, v0l);
+                split_bf16(in[5], v1, v1l);
+                kn[j * HD + ii] = k0; kn[j * HD + ii + half] = k1;
+                kn[(32 + j) * HD + ii] = k0l; kn[(32 + j) * HD + ii + half] = k1l;
+                vn[j * HD + ii] = v0; vn[j * HD + ii + half] = v1;
+                vn[(32 + j) * HD + ii] = v0l; vn[(32 + j) * HD + ii + half] = v1l;
+                if (writer) {
+                    bf16 *kc = m.kcache + cbase + (size_t)pos * HD, *vc = m.vcache + cbase + (size_t)pos * HD;
+                    kc[ii] = k0; kc[ii + half] = k1;
+                    kc[m.kv_lo + ii] = k0l; kc[m.kv_lo + ii + half] = k1l;
+                    vc[ii] = v0; vc[ii + half] = v1;
+                    vc[m.kv_lo + ii] = v0l; vc[m.kv_lo + ii + half] = v1l;
+                }
+            } else {
+                qrow[ii] = qrow_lo[ii] = __float2bfloat16(0.f);
+                qrow[ii + half] = qrow_lo[ii + half] = __float2bfloat16(0.f);
             }
-        } else {
-            qrow[ii] = qrow_lo[ii] = __float2bfloat16(0.f);
-            qrow[ii + half] = qrow_lo[ii + half] = __float2bfloat16(0.f);
         }
     }
 }

@@ -236,7 +236,10 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
     c.tmem = *tmem_slot;
 
     // the producer warps live in their streams until the forward's last stage
-    if (c.warp == W_PRODUCER) { if (c.lane == 0) weight_producer(c, a.fb, a.P); return; }
+    if (c.warp == W_PRODUCER || c.warp == 10 || c.warp == 11) {
+        if (c.lane == 0) weight_producer(c, a.fb, a.P, c.warp == W_PRODUCER ? 0 : c.warp - 9);
+        return;
+    }
     if (c.warp == MMA_ISSUER) {
         if (c.lane == 0) mma_issuer<NT>(c, a.fb, a.P);
         __syncwarp();
@@ -244,7 +247,6 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(c.tmem), "r"(TMEM_COLS) : "memory");
         return;
     }
-    if (c.warp > MMA_ISSUER && c.warp < X_PRODUCER) return;
     if (c.warp == X_PRODUCER + X_PRODUCERS - 1) { helper_warp(c, a.fb, a.P, m.cfg.d_model, m.cfg.rms_eps); return; }
     if (c.warp >= X_PRODUCER) {
         uint64_t keep;
@@ -267,7 +269,11 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
 
     const int L = a.P.n_layers;
     for (int l = 0; l < L; ++l) {
-        gemm_op<NT>(c, a.fb, a.P, 4 * l + OP_QKV, nullptr, 0, [&](int tile, float (&acc)[NT][4]) { epi_qkv<NT>(c, a, tile, acc); });
+        {
+            const int slice = op_slice(a.P.op[OP_QKV], c.cta, c.ncta);
+            gemm_op<NT>(c, a.fb, a.P, 4 * l + OP_QKV, nullptr, 0,
+                        [&](int tile, float (&acc)[NT][4]) { epi_qkv<NT>(c, a, slice, tile, acc); });
+        }
         stamp();
         grid_barrier(c, a.fb);
         stamp();
@@ -366,10 +372,12 @@ static inline Plan make_plan(const ModelDev &m, const DevPtrs &d, const FwdBufs 
         o.S = 1;
         // few tiles and enough bytes to be bandwidth bound: also cut along k, so that a block needs less of the
         // activations (a small projection is latency bound and better off without the extra pass and barrier)
-        if ((i == OP_O || i == OP_DOWN) && (long long)N * K * 2 >= (16ll << 20)) {
+        // (the wider a block's row range, the larger its stages: a stage costs the issuing threads about 0.4 us
+        // whatever its size).  As many slices as keep a block's share within one pass, four at most.
+        if ((i == OP_QKV || i == OP_O || i == OP_DOWN) && (long long)N * K * 2 >= (16ll << 20)) {
             const int nks = (K + KC - 1) / KC;
-            for (int sdiv = 2; sdiv <= 8; ++sdiv)
-                if (ncta % sdiv == 0 && sdiv <= nks && MT * (sdiv / 2) < 4 * ncta) o.S = sdiv;
+            for (int sdiv = 2; sdiv <= 4; ++sdiv)
+                if (ncta % sdiv == 0 && sdiv <= nks && (MT + ncta / sdiv - 1) / (ncta / sdiv) <= MAX_TILES) o.S = sdiv;
         }
         o.rot = rot;
         rot = (rot + (MT % (ncta / o.S)) * o.S) % ncta;       // the next projection's extra tiles go to other blocks

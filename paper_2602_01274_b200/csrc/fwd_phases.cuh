@@ -110,16 +110,17 @@ __device__ __forceinline__ void phase_begin(Ctx &c, const Args &a, int nt_total)
 // ------------------------------------------------------------------ tile epilogues
 // acc element (nt, i): token row nt*8 + 2t + (i & 1), tile column g + 8*(i >> 1), with g = lane / 4, t = lane % 4.
 
-// q/k/v tile: the deferred 1/rms of the input RMSNorm, then qkv[row][column].
+// q/k/v tile: the deferred 1/rms of the input RMSNorm, then qkv[k slice][row][column] (the attention phase
+// adds the k slices' shares when it reads the rows).
 template <int NT>
-__device__ __forceinline__ void epi_qkv(Ctx &c, const Args &a, int tile, float (&acc)[NT][4]) {
+__device__ __forceinline__ void epi_qkv(Ctx &c, const Args &a, int slice, int tile, float (&acc)[NT][4]) {
     const int g = c.lane >> 2, t = c.lane & 3, N = a.m.qrows;
     const int n0 = tile * 16 + g, n1 = n0 + 8;
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
         const int r0 = nt * 8 + 2 * t;
         const float i0 = c.inv_rms[r0], i1 = c.inv_rms[r0 + 1];
-        float *q0 = a.fb.qkv + (size_t)r0 * N, *q1 = q0 + N;
+        float *q0 = a.fb.qkv + ((size_t)slice * MAX_ROWS + r0) * N, *q1 = q0 + N;
         if (n0 < N) { q0[n0] = acc[nt][0] * i0; q1[n0] = acc[nt][1] * i1; }
         if (n1 < N) { q0[n1] = acc[nt][2] * i0; q1[n1] = acc[nt][3] * i1; }
     }

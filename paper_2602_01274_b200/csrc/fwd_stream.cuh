@@ -56,9 +56,11 @@ __device__ __forceinline__ int ring_place(int &head, int bytes) {
     return at;
 }
 
-// Lane 0 of warp W_PRODUCER: every weight stage of the block, for the whole forward, in order.  A stage may
-// be written once every earlier stage that overlaps its bytes has been released (stages are released in order).
-__device__ __forceinline__ void weight_producer(Ctx &c, const FwdBufs &fb, const Plan &P) {
+// Lane 0 of the W_PRODUCERS weight warps: every weight stage of the block, for the whole forward, in order;
+// producer `me` issues the stages n with n % W_PRODUCERS == me (one thread alone issues a bulk copy only every
+// 0.4 us or so) and replays the placement of the others.  A stage may be written once every earlier stage that
+// overlaps its bytes has been released; stages are released in order, and stage n - NB before stage n is issued.
+__device__ __forceinline__ void weight_producer(Ctx &c, const FwdBufs &fb, const Plan &P, int me) {
     int n = 0, tail = 0, head = 0;
     int q_s[NB], q_e[NB];
     for (int q = 0; q < n_ops(P); ++q) {
@@ -72,15 +74,18 @@ __device__ __forceinline__ void weight_producer(Ctx &c, const FwdBufs &fb, const
             const int bytes = Tp * 2048;                 // two 8-row atoms per tile
             for (int k = k_lo; k < k_hi; k += KB, ++n) {
                 const int at = ring_place(head, bytes), end = at + bytes;
-                int need = n - tail >= NB ? tail + 1 : tail;
-                for (int j = tail; j < n; ++j)
-                    if (q_s[j % NB] < end && at < q_e[j % NB]) need = j + 1;
-                for (; tail < need; ++tail)
-                    if (!wait_bar(fb, c.wempty + tail % NB, ((uint32_t)(tail / NB)) & 1u, 5, tail)) return;   // stop feeding
+                if (n % W_PRODUCERS == me) {
+                    if (tail < n - NB) tail = n - NB;       // older stages were released before stage n - NB
+                    int need = n - tail >= NB ? tail + 1 : tail;
+                    for (int j = tail; j < n; ++j)
+                        if (q_s[j % NB] < end && at < q_e[j % NB]) need = j + 1;
+                    for (; tail < need; ++tail)
+                        if (!wait_bar(fb, c.wempty + tail % NB, ((uint32_t)(tail / NB)) & 1u, 5, tail)) return;   // stop feeding
+                    mbar_expect_tx(c.wfull + n % NB, (uint32_t)bytes);
+                    bulk_g2s(c.ring + at, wl + ((size_t)(k >> 6) * (2 * op.MT) + 2 * (t0 + p0)) * 512, (uint32_t)bytes,
+                             c.wfull + n % NB, c.policy);
+                }
                 q_s[n % NB] = at; q_e[n % NB] = end;
-                mbar_expect_tx(c.wfull + n % NB, (uint32_t)bytes);
-                bulk_g2s(c.ring + at, wl + ((size_t)(k >> 6) * (2 * op.MT) + 2 * (t0 + p0)) * 512, (uint32_t)bytes, c.wfull + n % NB,
-                         c.policy);
             }
         }
     }

@@ -178,7 +178,7 @@ static Layout make_layout(const pacer_cfg &c) {
     L.hidden = cv.take(sizeof(float) * fwd::MAX_ROWS * d_max);
     L.att = cv.take(sizeof(bf16) * 2 * fwd::MAX_ROWS * d_max);        // values, then rounding remainders
     L.act = cv.take(sizeof(bf16) * 2 * fwd::MAX_ROWS * f_max);
-    L.qkv = cv.take(sizeof(float) * fwd::MAX_ROWS * qrows_max);
+    L.qkv = cv.take(sizeof(float) * 4 * fwd::MAX_ROWS * qrows_max);     // up to four k slices
     L.xg = cv.take(sizeof(bf16) * 2 * fwd::MAX_ROWS * d_max);
     L.ssq = cv.take(sizeof(float) * fwd::MAX_ROWS * (d_max / 16 + 1));
     L.tile_top = cv.take(sizeof(float) * 4 * fwd::MAX_ROWS * ((size_t)V / 16 + 1));
