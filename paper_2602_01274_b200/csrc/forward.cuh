@@ -40,7 +40,6 @@ constexpr int X_PRODUCER = 12, X_PRODUCERS = 4;  // warps 12..14 provide the act
                                                  // warp 15 computes the RMS statistics
 constexpr int THREADS = 32 * (X_PRODUCER + X_PRODUCERS);
 constexpr int KB = 64;                          // k columns of a weight stage: one 128-byte swizzle row
-constexpr int KC = 512;                         // k slices of a projection are whole multiples of this
 constexpr int NB = 16;                          // weight stages that can be in flight (barrier pairs)
 constexpr int RING_BYTES = 136 * 1024;          // weight ring (bytes; a stage takes 128 B per weight row of the block)
 constexpr int XS_MAX = 3;                       // activation stages: as many as fit, at most 3 (one producer warp each)
@@ -229,7 +228,7 @@ __device__ __forceinline__ void bsync() { asm volatile("bar.sync 1, 256;" ::: "m
 
 // Work of block `cta` in a projection: tiles [t0, t0 + T) over the k range [k_lo, k_hi).
 // With S slices the blocks form ncta / S groups; a group shares a tile range and its S
-// blocks take one k slice each (slices are whole KC steps).
+// blocks take one k slice each (slices are whole 64-column k blocks, as even as they come).
 __device__ __host__ __forceinline__ void op_range(const GemmOp &op, int cta, int ncta, int &t0, int &T, int &k_lo, int &k_hi) {
     int ci = cta - op.rot;
     if (ci < 0) ci += ncta;
@@ -237,9 +236,9 @@ __device__ __host__ __forceinline__ void op_range(const GemmOp &op, int cta, int
     const int base = op.MT / groups, rem = op.MT % groups;
     T = g < groups ? base + (g < rem ? 1 : 0) : 0;
     t0 = g * base + (g < rem ? g : rem);
-    const int nks = (op.K + KC - 1) / KC, sb = nks / op.S, sr = nks % op.S;
-    k_lo = (s * sb + (s < sr ? s : sr)) * KC;
-    k_hi = k_lo + (sb + (s < sr ? 1 : 0)) * KC;
+    const int nks = op.K / KB, sb = nks / op.S, sr = nks % op.S;
+    k_lo = (s * sb + (s < sr ? s : sr)) * KB;
+    k_hi = k_lo + (sb + (s < sr ? 1 : 0)) * KB;
     if (k_hi > op.K) k_hi = op.K;
     if (k_lo >= k_hi) T = 0;
 }

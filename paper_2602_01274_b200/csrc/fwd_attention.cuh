@@ -58,13 +58,13 @@ __device__ __forceinline__ void attention_rows(Ctx &c, const Args &a, int layer,
     bf16 *kn = reinterpret_cast<bf16 *>(c.scratch + SM::KN_OFF), *vn = reinterpret_cast<bf16 *>(c.scratch + SM::VN_OFF);
     const size_t cbase = (((size_t)layer * d.max_batch + seq) * Hkv + kh) * (size_t)d.max_ctx * HD;
     const float scale = rsqrtf((float)HD);
-    // The projection may have been cut along k: every value is the sum of the slices' shares.  Two elements per
+    // The projection may have been cut along k: every value is the sum of the slices' shares.  Four elements per
     // thread at a time, all their loads issued before the first use (the phase is bound by load latency).
     const int S = a.P.op[OP_QKV].S;
     const size_t sl = (size_t)MAX_ROWS * qrows;
-    constexpr int U = 2;
+    constexpr int U = 4;
     for (int i0 = threadIdx.x; i0 < 32 * half; i0 += U * MMA_THREADS) {
-        float part[U][4][6];
+        float part[U][2][6];
         float2 cs[U];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
@@ -75,9 +75,16 @@ __device__ __forceinline__ void attention_rows(Ctx &c, const Args &a, int layer,
                                 (H + Hkv + kh) * HD + ii, (H + Hkv + kh) * HD + ii + half};
             cs[u] = on ? m.rope[(size_t)(pos0 + j) * half + ii] : make_float2(0.f, 0.f);
 #pragma unroll
-            for (int s = 0; s < 4; ++s)
+            for (int s = 0; s < 2; ++s)
 #pragma unroll
                 for (int e = 0; e < 6; ++e) part[u][s][e] = (on && s < S) ? __ldcg(row + s * sl + col[e]) : 0.f;
+            if (S > 2 && on) {                                   // slices 2, 3: a second wave of loads
+#pragma unroll
+                for (int e = 0; e < 6; ++e) {
+                    const float p2 = __ldcg(row + 2 * sl + col[e]), p3 = S > 3 ? __ldcg(row + 3 * sl + col[e]) : 0.f;
+                    part[u][0][e] += p2; part[u][1][e] += p3;
+                }
+            }
         }
 #pragma unroll
         for (int u = 0; u < U; ++u) {
@@ -89,7 +96,7 @@ __device__ __forceinline__ void attention_rows(Ctx &c, const Args &a, int layer,
                 const int pos = pos0 + j;
                 float in[6];
 #pragma unroll
-                for (int e = 0; e < 6; ++e) in[e] = (part[u][0][e] + part[u][1][e]) + (part[u][2][e] + part[u][3][e]);
+                for (int e = 0; e < 6; ++e) in[e] = part[u][0][e] + part[u][1][e];
                 const float qa = in[0], qb = in[1], ka = in[2], kb = in[3];
                 split_bf16((qa * cs[u].x - qb * cs[u].y) * scale, qrow[ii], qrow_lo[ii]);
                 split_bf16((qb * cs[u].x + qa * cs[u].y) * scale, qrow[ii + half], qrow_lo[ii + half]);
@@ -230,6 +237,21 @@ __device__ __forceinline__ void attention_keys(Ctx &c, const bf16 *kcache, const
     }
 }
 
+// L2 prefetch of the cached K and V rows (values and remainders) this warp's steps will read, issued before the
+// new rows are prepared: the key loop is a chain of dependent loads, which then hit L2 instead of HBM.
+template <int HD>
+__device__ __forceinline__ void attention_prefetch(const Ctx &c, const bf16 *kcache, const bf16 *vcache, size_t kv_lo, int lo,
+                                                   int hi, int kw, int KW) {
+    constexpr int LPK = HD / 64;                         // 128-byte lines per key row
+    const int steps_c = (hi - lo + 7) >> 3;
+    for (int st = kw; st < steps_c; st += KW)
+        for (int idx = c.lane; idx < 32 * LPK; idx += 32) {
+            const int line = idx % LPK, key = (idx / LPK) & 7, plane = (idx / (LPK * 8)) & 1, tens = idx / (LPK * 16);
+            const bf16 *ptr = (tens ? vcache : kcache) + plane * kv_lo + (size_t)min(lo + st * 8 + key, hi - 1) * HD + line * 64;
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr));
+        }
+}
+
 template <int HD>
 __device__ __forceinline__ void attention_item(Ctx &c, const Args &a, int layer, int seq, int h, int split, int nsplit,
                                                int nt_total) {
@@ -240,13 +262,13 @@ __device__ __forceinline__ void attention_item(Ctx &c, const Args &a, int layer,
     const int H = m.cfg.n_heads, Hkv = m.cfg.n_kv_heads, group = H / Hkv, kh = h / group;
     const int n_r = c.n_rows[seq], r_base = seq * a.g.rps, pos0 = c.row_pos[r_base];
     const size_t cbase = (((size_t)layer * d.max_batch + seq) * Hkv + kh) * (size_t)d.max_ctx * HD;
-    attention_rows<HD>(c, a, layer, seq, h, split == 0 && h == kh * group);
-    bsync();
-
     const int lo = (int)((long long)pos0 * split / nsplit), hi = (int)((long long)pos0 * (split + 1) / nsplit);
     const int two = n_r > 16 ? 1 : 0;                    // two query tiles: warps 0..3 take rows 0..15, warps 4..7 rows 16..31
     const int mt = two ? (c.warp >> 2) : 0, kw = two ? (c.warp & 3) : c.warp, KW = two ? 4 : 8;
     const int g = c.lane >> 2, t = c.lane & 3;
+    if (hi > lo) attention_prefetch<HD>(c, m.kcache + cbase, m.vcache + cbase, m.kv_lo, lo, hi, kw, KW);
+    attention_rows<HD>(c, a, layer, seq, h, split == 0 && h == kh * group);
+    bsync();
     float mx[2] = {-INFINITY, -INFINITY}, lsum[2] = {0.f, 0.f};
     float o[NOT][4];
 #pragma unroll

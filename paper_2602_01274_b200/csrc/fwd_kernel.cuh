@@ -375,7 +375,7 @@ static inline Plan make_plan(const ModelDev &m, const DevPtrs &d, const FwdBufs 
         // (the wider a block's row range, the larger its stages: a stage costs the issuing threads about 0.4 us
         // whatever its size).  As many slices as keep a block's share within one pass, four at most.
         if ((i == OP_QKV || i == OP_O || i == OP_DOWN) && (long long)N * K * 2 >= (16ll << 20)) {
-            const int nks = (K + KC - 1) / KC;
+            const int nks = K / (8 * KB);                    // a slice keeps at least 512 columns
             for (int sdiv = 2; sdiv <= 4; ++sdiv)
                 if (ncta % sdiv == 0 && sdiv <= nks && (MT + ncta / sdiv - 1) / (ncta / sdiv) <= MAX_TILES) o.S = sdiv;
         }
