@@ -12,14 +12,19 @@
  *   - "device" pointers are CUDA device addresses on the current device, "host"
  *     pointers are ordinary memory.  All device memory is CALLER-OWNED: the
  *     library never allocates or frees device memory.  It carves the workspace
- *     given to pacer_create and reads weights in place.
+ *     given to pacer_create; pacer_load_weights copies the projection matrices
+ *     into it in the order the forward kernel streams them (the workspace holds
+ *     one copy of every layer matrix and LM head) and reads the other tensors in
+ *     place.
  *   - Calls enqueue work on the context's stream and return without waiting
  *     unless marked [sync].  A context is not thread-safe.
  *   - Models are Llama-style decoders: RMSNorm, rotary embedding (rotate-half,
  *     absolute positions), causal attention with n_kv_heads <= n_heads, SwiGLU
  *     MLP, untied embedding and LM head, no biases.  Weights are bf16, matrices
  *     are [out][in] row-major and stacked over layers; accumulation, the residual
- *     stream, norms and softmax are fp32; KV caches are bf16.
+ *     stream, norms and softmax are fp32.  Activations enter the tensor cores as
+ *     a bf16 value plus a bf16 rounding remainder (16 mantissa bits), and the KV
+ *     caches hold both parts.
  *   - Batch rows are independent sequences.  Token ids are int32.
  */
 #ifndef PACER_H_
@@ -44,6 +49,7 @@ enum {
 
 typedef struct pacer_ctx pacer_ctx;
 
+/* d_model and d_ffn are multiples of 64 (the width of a weight stage), d_model / n_heads is 64 or 128. */
 typedef struct {
     int32_t n_layers, d_model, n_heads, n_kv_heads, d_ffn, vocab;
     float rope_theta;        /* 10000 */
@@ -67,7 +73,9 @@ typedef struct {
  *   wo [L][d][H*hd]         wgate, wup [L][F][d]       wdown [L][d][F]
  *   norm1, norm2 [L][d]     normf [d]                  head [V][d]
  * M_B (which = 2) has no embed/head but  head_b [2][d]  and  posemb [gamma_cap][d].
- * The tensors are used in place and must outlive the context. */
+ * wqkv, wo, wgate, wup, wdown and head are copied (re-laid for the tensor cores) by
+ * pacer_load_weights and may be freed once the stream has run it; embed, the norm
+ * gains, head_b and posemb are used in place and must outlive the context. */
 typedef struct {
     const char *name;
     const void *dev_ptr;
@@ -125,9 +133,9 @@ enum {
 const char *pacer_strerror(int code);
 const char *pacer_last_error(const pacer_ctx *ctx);
 
-/* Bytes of device workspace a context with this configuration needs (KV caches
- * of the three models, activations, logits, per-sequence state).  0 on a bad
- * configuration. */
+/* Bytes of device workspace a context with this configuration needs (the
+ * re-laid projection matrices and KV caches of the three models, activations,
+ * logits, per-sequence state).  0 on a bad configuration. */
 size_t pacer_workspace_bytes(const pacer_cfg *cfg);
 
 /* Creates a context on the current device.  dev_workspace: device, at least

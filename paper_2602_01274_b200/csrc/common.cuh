@@ -1,5 +1,5 @@
 // Shared definitions of the Pacer CUDA library (device state, row geometry,
-// fragment-major activation layout).  sm_100a only.
+// activation layout of the standalone GEMM).  sm_100a only.
 #pragma once
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -65,9 +65,9 @@ struct DevPtrs {
     int32_t *row_arg;    // [rtot] argmax of the LM-head row
     float *row_margin;   // [rtot] top1 - top2
     float *xres;         // [rtot][d] fp32 residual stream
-    bf16 *xn;            // fragment-major bf16 [K=d][rows]: GEMM input after a norm
-    bf16 *att;           // fragment-major bf16 [K=H*hd][rows]
-    bf16 *act;           // fragment-major bf16 [K=F][rows]
+    bf16 *xn;            // unused by the forward kernel (its x * gain buffer is FwdBufs::xg)
+    bf16 *att;           // attention output, split bf16 in tensor-core operand order (K = H*hd)
+    bf16 *act;           // SwiGLU output, split bf16 in tensor-core operand order (K = F)
     float *q;            // [rtot][H*hd] fp32 rotated queries
     float *hidden;       // [rtot][d] fp32 final-norm output
     float *part;         // split-K partial sums [S][nt*8][N]
@@ -88,7 +88,7 @@ struct ModelDev {
     int32_t loaded;
 };
 
-// Offset (in elements) of X[r][k] in the fragment-major layout the GEMM reads:
+// Offset (in elements) of X[r][k] in the fragment-major layout the standalone GEMM (pacer_linear) reads:
 // [k/32][row tile][lane = (r%8)*4 + (k%32)/8][k%8].  A warp's 128-bit loads of
 // one (32-wide k chunk, row tile) are 512 contiguous bytes, already in the
 // register order of mma.m16n8k16's B operand (with the k permutation the GEMM

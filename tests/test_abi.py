@@ -37,8 +37,9 @@ def test_workspace_bytes_host_logic():
     from paper_2602_01274_b200 import binding as b
     cfg = synth.CONFIGS["7b_68m"]
     n = b.pacer_workspace_bytes(b.make_cfg(cfg.target, cfg.draft, 1, 1024, 16))
-    kv = cfg.target.kv_bytes_per_token() * 1024
-    assert kv < n < kv + (1 << 30)
+    # the target's cache (values + remainders) and the library's own copy of its projection matrices dominate
+    big = 2 * cfg.target.kv_bytes_per_token() * 1024 + cfg.target.streamed_weight_bytes()
+    assert big < n < big + (1 << 30)
     assert b.pacer_workspace_bytes(b.make_cfg(cfg.target, cfg.draft, 0, 1024, 16)) == 0
     assert b.pacer_workspace_bytes(b.make_cfg(cfg.target, cfg.draft, 1, 1024, 16, block_b=3)) == 0
     assert b.pacer_strerror if hasattr(b, "pacer_strerror") else True
