@@ -156,7 +156,7 @@ __device__ __forceinline__ void attention_keys(Ctx &c, const bf16 *kcache, const
         }
         // scores S = Q K^T for 8 keys: lane (g, t) reads 8 consecutive channels of key g and uses them as the
         // k slots {2t, 2t+1, 2t+8, 2t+9} of two MMAs; q is read with the same rule
-        float s[4] = {0.f, 0.f, 0.f, 0.f};
+        float s[4];
         {
             const bf16 *krow = kb + (size_t)min(key0 + g, kend - 1) * HD + t * 8;
             uint4 kf[NCH], kl[NCH];
@@ -165,18 +165,24 @@ __device__ __forceinline__ void attention_keys(Ctx &c, const bf16 *kcache, const
                 kf[cc] = *reinterpret_cast<const uint4 *>(krow + cc * 32);
                 kl[cc] = *reinterpret_cast<const uint4 *>(krow + plane + cc * 32);
             }
+            // two independent accumulators halve the chain of dependent MMAs (more of them spill registers)
+            float sa[2][4];
+#pragma unroll
+            for (int e = 0; e < 2; ++e) sa[e][0] = sa[e][1] = sa[e][2] = sa[e][3] = 0.f;
 #pragma unroll
             for (int cc = 0; cc < NCH; ++cc) {
                 const uint4 qa = *reinterpret_cast<const uint4 *>(q0 + cc * 64), qb = *reinterpret_cast<const uint4 *>(q1 + cc * 64);
-                mma16816(s, qa.x, qb.x, qa.y, qb.y, kf[cc].x, kf[cc].y);
-                mma16816(s, qa.z, qb.z, qa.w, qb.w, kf[cc].z, kf[cc].w);
-                mma16816(s, qa.x, qb.x, qa.y, qb.y, kl[cc].x, kl[cc].y);
-                mma16816(s, qa.z, qb.z, qa.w, qb.w, kl[cc].z, kl[cc].w);
+                mma16816(sa[0], qa.x, qb.x, qa.y, qb.y, kf[cc].x, kf[cc].y);
+                mma16816(sa[1], qa.z, qb.z, qa.w, qb.w, kf[cc].z, kf[cc].w);
+                mma16816(sa[0], qa.x, qb.x, qa.y, qb.y, kl[cc].x, kl[cc].y);
+                mma16816(sa[1], qa.z, qb.z, qa.w, qb.w, kl[cc].z, kl[cc].w);
                 const uint4 la = *reinterpret_cast<const uint4 *>(q0 + 32 * QP + cc * 64);
                 const uint4 lb = *reinterpret_cast<const uint4 *>(q1 + 32 * QP + cc * 64);
-                mma16816(s, la.x, lb.x, la.y, lb.y, kf[cc].x, kf[cc].y);
-                mma16816(s, la.z, lb.z, la.w, lb.w, kf[cc].z, kf[cc].w);
+                mma16816(sa[0], la.x, lb.x, la.y, lb.y, kf[cc].x, kf[cc].y);
+                mma16816(sa[1], la.z, lb.z, la.w, lb.w, kf[cc].z, kf[cc].w);
             }
+#pragma unroll
+            for (int i = 0; i < 4; ++i) s[i] = sa[0][i] + sa[1][i];
         }
         // mask: keys past the end; among the keys of this forward, row j sees keys 0..j
         float rmax[2] = {-INFINITY, -INFINITY};
