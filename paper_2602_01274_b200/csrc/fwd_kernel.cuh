@@ -378,6 +378,10 @@ static inline Plan make_plan(const ModelDev &m, const DevPtrs &d, const FwdBufs 
             const int nks = K / (8 * KB);                    // a slice keeps at least 512 columns
             for (int sdiv = 2; sdiv <= 4; ++sdiv)
                 if (ncta % sdiv == 0 && sdiv <= nks && (MT + ncta / sdiv - 1) / (ncta / sdiv) <= MAX_TILES) o.S = sdiv;
+        } else if (i == OP_DOWN && K >= 32 * KB && MT < ncta && ncta % 4 == 0) {
+            // a small model's down projection: one or two tiles per block over a long k range is a chain of
+            // K / 64 stages of 0.3 - 0.4 us each, longer than the reduction pass that four k slices cost
+            o.S = 4;
         }
         o.rot = rot;
         rot = (rot + (MT % (ncta / o.S)) * o.S) % ncta;       // the next projection's extra tiles go to other blocks
