@@ -36,7 +36,7 @@ struct AttSmem {
     static constexpr int VS_OFF = VN_OFF + 2 * 32 * HD * 2;   // [8 warps][16][VP] V of the current step: 8 keys x 2 planes
     static constexpr int END = VS_OFF + MMA_WARPS * 16 * VP;
     static_assert(END <= SCRATCH_BYTES, "attention staging does not fit the scratch");
-    static_assert(MMA_WARPS * 16 * PW * 4 <= SCRATCH_BYTES, "attention merge buffer does not fit the scratch");
+    static_assert((MMA_WARPS * 16 * PW + 32 * MMA_WARPS + 64) * 4 <= SCRATCH_BYTES, "attention merge buffer does not fit the scratch");
 };
 
 __device__ __forceinline__ void split_bf16(float v, bf16 &hi, bf16 &lo) {
@@ -58,18 +58,26 @@ __device__ __forceinline__ void attention_rows(Ctx &c, const Args &a, int layer,
     bf16 *kn = reinterpret_cast<bf16 *>(c.scratch + SM::KN_OFF), *vn = reinterpret_cast<bf16 *>(c.scratch + SM::VN_OFF);
     const size_t cbase = (((size_t)layer * d.max_batch + seq) * Hkv + kh) * (size_t)d.max_ctx * HD;
     const float scale = rsqrtf((float)HD);
-    // The projection may have been cut along k: every value is the sum of the slices' shares.  Four elements per
+    // The projection may have been cut along k: every value is the sum of the slices' shares.  Five elements per
     // thread at a time, all their loads issued before the first use (the phase is bound by load latency).
     const int S = a.P.op[OP_QKV].S;
     const size_t sl = (size_t)MAX_ROWS * qrows;
-    constexpr int U = 4;
-    for (int i0 = threadIdx.x; i0 < 32 * half; i0 += U * MMA_THREADS) {
+    constexpr int U = 5;                                 // 17 rows of 128 channels are one batch
+    const int n_act = n_r * half;
+    for (int i = n_act + threadIdx.x; i < 32 * half; i += MMA_THREADS) {     // idle query rows are zeros
+        const int j = i / half, ii = i - j * half;
+        bf16 *qrow = reinterpret_cast<bf16 *>(c.scratch + SM::Q_OFF + j * SM::QP);
+        bf16 *qrow_lo = reinterpret_cast<bf16 *>(c.scratch + SM::Q_OFF + (32 + j) * SM::QP);
+        qrow[ii] = qrow_lo[ii] = __float2bfloat16(0.f);
+        qrow[ii + half] = qrow_lo[ii + half] = __float2bfloat16(0.f);
+    }
+    for (int i0 = threadIdx.x; i0 < n_act; i0 += U * MMA_THREADS) {
         float part[U][2][6];
         float2 cs[U];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const int i = i0 + u * MMA_THREADS, j = i / half, ii = i - j * half;
-            const bool on = i < 32 * half && j < n_r;
+            const bool on = i < n_act;
             const float *row = a.fb.qkv + (size_t)(r_base + (on ? j : 0)) * qrows;
             const int col[6] = {h * HD + ii, h * HD + ii + half, (H + kh) * HD + ii, (H + kh) * HD + ii + half,
                                 (H + Hkv + kh) * HD + ii, (H + Hkv + kh) * HD + ii + half};
@@ -89,10 +97,10 @@ __device__ __forceinline__ void attention_rows(Ctx &c, const Args &a, int layer,
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const int i = i0 + u * MMA_THREADS, j = i / half, ii = i - j * half;
-            if (i >= 32 * half) continue;
+            if (i >= n_act) continue;
             bf16 *qrow = reinterpret_cast<bf16 *>(c.scratch + SM::Q_OFF + j * SM::QP);
             bf16 *qrow_lo = reinterpret_cast<bf16 *>(c.scratch + SM::Q_OFF + (32 + j) * SM::QP);
-            if (j < n_r) {
+            {
                 const int pos = pos0 + j;
                 float in[6];
 #pragma unroll
@@ -116,9 +124,6 @@ __device__ __forceinline__ void attention_rows(Ctx &c, const Args &a, int layer,
                     vc[ii] = v0; vc[ii + half] = v1;
                     vc[m.kv_lo + ii] = v0l; vc[m.kv_lo + ii + half] = v1l;
                 }
-            } else {
-                qrow[ii] = qrow_lo[ii] = __float2bfloat16(0.f);
-                qrow[ii + half] = qrow_lo[ii + half] = __float2bfloat16(0.f);
             }
         }
     }
@@ -296,24 +301,34 @@ __device__ __forceinline__ void attention_item(Ctx &c, const Args &a, int layer,
     // merge the warps of each query tile -> the item's partial in global memory; with a single split the
     // result is final and goes straight to the output projection's input buffer
     float *outp = a.fb.attp + (((size_t)(seq * H + h) * MAX_SPLIT + split) * a.g.rps) * PW;
-    for (int i = threadIdx.x; i < n_r * HD; i += MMA_THREADS) {
-        const int j = i / HD, ch = i - j * HD;
-        const int w0 = two ? (j >> 4) * 4 : 0, rr = j & 15;
+    // per (row, warp) the factor exp(max_w - max) once, then one multiply-add per warp and output channel
+    float *fw = red + MMA_WARPS * 16 * PW;               // [row][8] factors, then [row] max, [row] sum
+    float *rowM = fw + 32 * MMA_WARPS, *rowL = rowM + 32;
+    if (threadIdx.x < n_r) {
+        const int j = threadIdx.x, w0 = two ? (j >> 4) * 4 : 0, rr = j & 15;
         float M = -INFINITY;
         for (int w = 0; w < KW; ++w) M = fmaxf(M, red[((size_t)(w0 + w) * 16 + rr) * PW + HD]);
-        float L = 0.f, ov = 0.f;
+        float L = 0.f;
         for (int w = 0; w < KW; ++w) {
             const float *rw = red + ((size_t)(w0 + w) * 16 + rr) * PW;
             const float f = rw[HD] == -INFINITY ? 0.f : __expf(rw[HD] - M);
+            fw[j * MMA_WARPS + w] = f;
             L += rw[HD + 1] * f;
-            ov += rw[ch] * f;
         }
+        rowM[j] = M; rowL[j] = L;
+    }
+    bsync();
+    for (int i = threadIdx.x; i < n_r * HD; i += MMA_THREADS) {
+        const int j = i / HD, ch = i - j * HD;
+        const int w0 = two ? (j >> 4) * 4 : 0, rr = j & 15;
+        float ov = 0.f;
+        for (int w = 0; w < KW; ++w) ov += red[((size_t)(w0 + w) * 16 + rr) * PW + ch] * fw[j * MMA_WARPS + w];
         if (nsplit == 1) {
-            store_split(d.att, nt_total, r_base + j, h * HD + ch, ov / L);
+            store_split(d.att, nt_total, r_base + j, h * HD + ch, ov / rowL[j]);
         } else {
             float *op = outp + (size_t)j * PW;
             op[ch] = ov;
-            if (ch == 0) { op[HD] = M; op[HD + 1] = L; }
+            if (ch == 0) { op[HD] = rowM[j]; op[HD + 1] = rowL[j]; }
         }
     }
     bsync();
