@@ -129,6 +129,23 @@ __device__ __forceinline__ void attention_rows(Ctx &c, const Args &a, int layer,
     }
 }
 
+// L2 prefetch of the cached K and V rows (values and remainders) of step st of this warp.  The first ATT_PF steps
+// are prefetched before the new rows are prepared, every later step ATT_PF steps ahead inside the key loop: the
+// loop is a chain of dependent loads, which then hit L2 instead of HBM (a burst of prefetches for a long key
+// range costs microseconds to issue and is partly dropped).
+constexpr int ATT_PF = 3;
+template <int HD>
+__device__ __forceinline__ void attention_prefetch(const Ctx &c, const bf16 *kcache, const bf16 *vcache, size_t kv_lo, int lo,
+                                                   int hi, int st) {
+    constexpr int LPK = HD / 64;                         // 128-byte lines per key row
+    if (st >= ((hi - lo + 7) >> 3)) return;
+    for (int idx = c.lane; idx < 32 * LPK; idx += 32) {
+        const int line = idx % LPK, key = (idx / LPK) & 7, plane = (idx / (LPK * 8)) & 1, tens = idx / (LPK * 16);
+        const bf16 *ptr = (tens ? vcache : kcache) + plane * kv_lo + (size_t)min(lo + st * 8 + key, hi - 1) * HD + line * 64;
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr));
+    }
+}
+
 // The key loop of one warp: keys in steps of 8 (step st, st + KW, ...), first the
 // cached keys [lo, hi), then (last split only) the n_r keys of this forward, which
 // row j sees up to key j.  mt: the warp's 16-row query tile.  Leaves running max,
@@ -159,6 +176,7 @@ __device__ __forceinline__ void attention_keys(Ctx &c, const bf16 *kcache, const
             if (fresh) *reinterpret_cast<uint4 *>(vslot + kr * VP + piece * 16) = *reinterpret_cast<const uint4 *>(src);
             else cp_async16(vslot + kr * VP + piece * 16, src);
         }
+        if (hi > lo) attention_prefetch<HD>(c, kcache, vcache, kv_lo, lo, hi, st + ATT_PF * KW);
         // scores S = Q K^T for 8 keys: lane (g, t) reads 8 consecutive channels of key g and uses them as the
         // k slots {2t, 2t+1, 2t+8, 2t+9} of two MMAs; q is read with the same rule
         float s[4];
@@ -248,21 +266,6 @@ __device__ __forceinline__ void attention_keys(Ctx &c, const bf16 *kcache, const
     }
 }
 
-// L2 prefetch of the cached K and V rows (values and remainders) this warp's steps will read, issued before the
-// new rows are prepared: the key loop is a chain of dependent loads, which then hit L2 instead of HBM.
-template <int HD>
-__device__ __forceinline__ void attention_prefetch(const Ctx &c, const bf16 *kcache, const bf16 *vcache, size_t kv_lo, int lo,
-                                                   int hi, int kw, int KW) {
-    constexpr int LPK = HD / 64;                         // 128-byte lines per key row
-    const int steps_c = (hi - lo + 7) >> 3;
-    for (int st = kw; st < steps_c; st += KW)
-        for (int idx = c.lane; idx < 32 * LPK; idx += 32) {
-            const int line = idx % LPK, key = (idx / LPK) & 7, plane = (idx / (LPK * 8)) & 1, tens = idx / (LPK * 16);
-            const bf16 *ptr = (tens ? vcache : kcache) + plane * kv_lo + (size_t)min(lo + st * 8 + key, hi - 1) * HD + line * 64;
-            asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr));
-        }
-}
-
 template <int HD>
 __device__ __forceinline__ void attention_item(Ctx &c, const Args &a, int layer, int seq, int h, int split, int nsplit,
                                                int nt_total) {
@@ -277,7 +280,8 @@ __device__ __forceinline__ void attention_item(Ctx &c, const Args &a, int layer,
     const int two = n_r > 16 ? 1 : 0;                    // two query tiles: warps 0..3 take rows 0..15, warps 4..7 rows 16..31
     const int mt = two ? (c.warp >> 2) : 0, kw = two ? (c.warp & 3) : c.warp, KW = two ? 4 : 8;
     const int g = c.lane >> 2, t = c.lane & 3;
-    if (hi > lo) attention_prefetch<HD>(c, m.kcache + cbase, m.vcache + cbase, m.kv_lo, lo, hi, kw, KW);
+    if (hi > lo)
+        for (int i = 0; i < ATT_PF; ++i) attention_prefetch<HD>(c, m.kcache + cbase, m.vcache + cbase, m.kv_lo, lo, hi, kw + i * KW);
     attention_rows<HD>(c, a, layer, seq, h, split == 0 && h == kh * group);
     bsync();
     float mx[2] = {-INFINITY, -INFINITY}, lsum[2] = {0.f, 0.f};
