@@ -51,8 +51,10 @@ constexpr int SCRATCH_BYTES = 88 * 1024;        // the activation ring lives in 
                                                 // of the accumulator, the attention phase and the tails use all of it
 constexpr int MISC_BYTES = 2048;
 constexpr int SMEM_BYTES = SCRATCH_BYTES + RING_BYTES + MISC_BYTES;
-constexpr int MAX_TILES = 16;                   // 16-row tiles of one pass of a block: N = 256 of one tcgen05.mma
-constexpr int TMEM_COLS = 256;                  // fp32 accumulator columns (one per weight row of the pass)
+constexpr int MMA_TILES = 16;                   // 16-row tiles one tcgen05.mma covers (N = 256)
+constexpr int MAX_TILES = 2 * MMA_TILES;        // tiles of one pass of a block: two accumulators, two MMAs per 16 k columns
+                                                // (a block that has one tile too many for N = 256 still reads the activations once)
+constexpr int ACC_COLS = 256;                   // fp32 accumulator columns of one accumulator (one per weight row)
 constexpr int MAX_ROWS = 32;                    // rows of one forward (all sequences together)
 constexpr int MAX_SPLIT = 16;                   // key-range splits of one attention head
 constexpr unsigned SPIN_LIMIT = 1u << 22;        // polls of a global word or a shared counter
@@ -79,6 +81,7 @@ struct GemmOp {
 struct Plan {
     GemmOp op[N_OPS];
     int32_t n_layers, has_head;
+    int32_t max_tiles;       // tiles of one pass: MMA_TILES, or MAX_TILES in the kernel variant with two accumulators
 };
 
 // Device buffers of the forward kernel beyond DevPtrs (all in the workspace).
@@ -245,9 +248,9 @@ __device__ __host__ __forceinline__ void op_range(const GemmOp &op, int cta, int
 
 // Passes of a block over its T tiles: as few as possible, evenly sized (the activations are streamed
 // once per pass, and an even split keeps every pass bandwidth bound rather than latency bound).
-__device__ __host__ __forceinline__ int n_passes(int T) { return (T + MAX_TILES - 1) / MAX_TILES; }
-__device__ __host__ __forceinline__ void pass_range(int T, int p, int &p0, int &Tp) {
-    const int np = n_passes(T), base = T / np, rem = T % np;
+__device__ __host__ __forceinline__ int n_passes(int T, int cap) { return (T + cap - 1) / cap; }
+__device__ __host__ __forceinline__ void pass_range(int T, int p, int cap, int &p0, int &Tp) {
+    const int np = n_passes(T, cap), base = T / np, rem = T % np;
     Tp = base + (p < rem ? 1 : 0);
     p0 = p * base + (p < rem ? p : rem);
 }

@@ -134,7 +134,7 @@ __device__ __forceinline__ void tail_ar(Ctx &c, const Args &a, int s) {
 
 // ------------------------------------------------------------------ the kernel
 
-template <int NT>
+template <int NT, bool TWO>
 __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ Args a, const int which) {
     extern __shared__ __align__(1024) unsigned char smem[];
     if (smem_u32(smem) & 1023u) {           // the swizzled operand layout needs this alignment (the same in every block)
@@ -226,7 +226,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (c.warp == MMA_ISSUER) {             // the accumulator's tensor memory, held until the end of the kernel
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TWO ? 2 * ACC_COLS : ACC_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     fence_proxy_async();
@@ -241,10 +241,10 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
         return;
     }
     if (c.warp == MMA_ISSUER) {
-        if (c.lane == 0) mma_issuer<NT>(c, a.fb, a.P);
+        if (c.lane == 0) mma_issuer<NT, TWO>(c, a.fb, a.P);
         __syncwarp();
         asm volatile("bar.sync 2, 288;" ::: "memory");        // the phase warps have read their last accumulator
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(c.tmem), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(c.tmem), "r"(TWO ? 2 * ACC_COLS : ACC_COLS) : "memory");
         return;
     }
     if (c.warp == X_PRODUCER + X_PRODUCERS - 1) { helper_warp(c, a.fb, a.P, m.cfg.d_model, m.cfg.rms_eps); return; }
@@ -271,7 +271,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
     for (int l = 0; l < L; ++l) {
         {
             const int slice = op_slice(a.P.op[OP_QKV], c.cta, c.ncta);
-            gemm_op<NT>(c, a.fb, a.P, 4 * l + OP_QKV, nullptr, 0,
+            gemm_op<NT, TWO>(c, a.fb, a.P, 4 * l + OP_QKV, nullptr, 0,
                         [&](int tile, float (&acc)[NT][4]) { epi_qkv<NT>(c, a, slice, tile, acc); });
         }
         stamp();
@@ -290,11 +290,11 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
             const GemmOp &op = a.P.op[OP_O];
             const bf16 *gain_next = m.norm2 + (size_t)l * dm;
             if (op.S == 1) {
-                gemm_op<NT>(c, a.fb, a.P, 4 * l + OP_O, d.xres, dm,
+                gemm_op<NT, TWO>(c, a.fb, a.P, 4 * l + OP_O, d.xres, dm,
                             [&](int tile, float (&acc)[NT][4]) { epi_residual<NT>(c, a, gain_next, tile, acc); });
             } else {
                 const int slice = op_slice(op, c.cta, c.ncta);
-                gemm_op<NT>(c, a.fb, a.P, 4 * l + OP_O, nullptr, 0,
+                gemm_op<NT, TWO>(c, a.fb, a.P, 4 * l + OP_O, nullptr, 0,
                             [&](int tile, float (&acc)[NT][4]) { epi_partial<NT>(c, a, op, slice, tile, acc); });
             }
             stamp();
@@ -305,7 +305,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
             }
             stamp();
         }
-        gemm_op<NT>(c, a.fb, a.P, 4 * l + OP_GU, nullptr, 0, [&](int tile, float (&acc)[NT][4]) { epi_swiglu<NT>(c, a, tile, acc); });
+        gemm_op<NT, TWO>(c, a.fb, a.P, 4 * l + OP_GU, nullptr, 0, [&](int tile, float (&acc)[NT][4]) { epi_swiglu<NT>(c, a, tile, acc); });
         stamp();
         grid_barrier(c, a.fb);
         stamp();
@@ -313,11 +313,11 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
             const GemmOp &op = a.P.op[OP_DOWN];
             const bf16 *gain_next = l + 1 < L ? m.norm1 + (size_t)(l + 1) * dm : m.normf;
             if (op.S == 1) {
-                gemm_op<NT>(c, a.fb, a.P, 4 * l + OP_DOWN, d.xres, dm,
+                gemm_op<NT, TWO>(c, a.fb, a.P, 4 * l + OP_DOWN, d.xres, dm,
                             [&](int tile, float (&acc)[NT][4]) { epi_residual<NT>(c, a, gain_next, tile, acc); });
             } else {
                 const int slice = op_slice(op, c.cta, c.ncta);
-                gemm_op<NT>(c, a.fb, a.P, 4 * l + OP_DOWN, nullptr, 0,
+                gemm_op<NT, TWO>(c, a.fb, a.P, 4 * l + OP_DOWN, nullptr, 0,
                             [&](int tile, float (&acc)[NT][4]) { epi_partial<NT>(c, a, op, slice, tile, acc); });
             }
             stamp();
@@ -330,7 +330,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
         }
     }
     if (a.P.has_head) {
-        gemm_op<NT>(c, a.fb, a.P, 4 * L, nullptr, 0,
+        gemm_op<NT, TWO>(c, a.fb, a.P, 4 * L, nullptr, 0,
                     [&](int tile, float (&acc)[NT][4]) { epi_head<NT>(c, a, row_dst, bias_at, tile, acc); });
         stamp();
         grid_barrier(c, a.fb);
@@ -377,7 +377,7 @@ static inline Plan make_plan(const ModelDev &m, const DevPtrs &d, const FwdBufs 
         if ((i == OP_QKV || i == OP_O || i == OP_DOWN) && (long long)N * K * 2 >= (16ll << 20)) {
             const int nks = K / (8 * KB);                    // a slice keeps at least 512 columns
             for (int sdiv = 2; sdiv <= 4; ++sdiv)
-                if (ncta % sdiv == 0 && sdiv <= nks && (MT + ncta / sdiv - 1) / (ncta / sdiv) <= MAX_TILES) o.S = sdiv;
+                if (ncta % sdiv == 0 && sdiv <= nks && (MT + ncta / sdiv - 1) / (ncta / sdiv) <= MMA_TILES) o.S = sdiv;
         } else if (i == OP_DOWN && K >= 32 * KB && MT < ncta && ncta % 4 == 0) {
             // a small model's down projection: one or two tiles per block over a long k range is a chain of
             // K / 64 stages of 0.3 - 0.4 us each, longer than the reduction pass that four k slices cost
@@ -392,29 +392,40 @@ static inline Plan make_plan(const ModelDev &m, const DevPtrs &d, const FwdBufs 
     set(OP_DOWN, m.wt[OP_DOWN], d.act, (int)dm, (int)F, ((int)dm + 15) / 16);
     set(OP_HEAD, m.wt[OP_HEAD], fb.xg, k.vocab, (int)dm, (k.vocab + 15) / 16);
     P.op[OP_HEAD].lstride = 0;
+    // one pass per projection where N = 256 allows it; a model in which some block has up to twice as many tiles
+    // runs the kernel variant with two accumulators (the activations are then still read once)
+    P.max_tiles = MMA_TILES;
+    for (int i = 0; i < N_OPS; ++i) {
+        if (i == OP_HEAD && !has_head) continue;
+        const GemmOp &o = P.op[i];
+        const int groups = ncta / o.S, per_block = (o.MT + groups - 1) / groups;
+        if (per_block > MMA_TILES && per_block <= MAX_TILES) P.max_tiles = MAX_TILES;
+    }
     P.n_layers = k.n_layers;
     P.has_head = has_head ? 1 : 0;
     return P;
 }
 
-template <int NT>
+template <int NT, bool TWO>
 static inline cudaError_t launch_nt(const Args &a, int which, int ncta, cudaStream_t st) {
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(k_forward<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+        cudaError_t e = cudaFuncSetAttribute(k_forward<NT, TWO>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
     void *params[] = {(void *)&a, (void *)&which};
-    return cudaLaunchCooperativeKernel((const void *)k_forward<NT>, dim3(ncta), dim3(THREADS), params, SMEM_BYTES, st);
+    return cudaLaunchCooperativeKernel((const void *)k_forward<NT, TWO>, dim3(ncta), dim3(THREADS), params, SMEM_BYTES, st);
 }
 
+// The variant with two accumulators runs the models in which some block has more than MMA_TILES tiles of a projection.
 static inline cudaError_t launch(const Args &a, int which, int ncta, cudaStream_t st) {
+    const bool two = a.P.max_tiles > MMA_TILES;
     switch (a.g.nt) {
-        case 1: return launch_nt<1>(a, which, ncta, st);
-        case 2: return launch_nt<2>(a, which, ncta, st);
-        case 3: return launch_nt<3>(a, which, ncta, st);
-        case 4: return launch_nt<4>(a, which, ncta, st);
+        case 1: return two ? launch_nt<1, true>(a, which, ncta, st) : launch_nt<1, false>(a, which, ncta, st);
+        case 2: return two ? launch_nt<2, true>(a, which, ncta, st) : launch_nt<2, false>(a, which, ncta, st);
+        case 3: return two ? launch_nt<3, true>(a, which, ncta, st) : launch_nt<3, false>(a, which, ncta, st);
+        case 4: return two ? launch_nt<4, true>(a, which, ncta, st) : launch_nt<4, false>(a, which, ncta, st);
     }
     return cudaErrorInvalidValue;
 }

@@ -68,9 +68,9 @@ __device__ __forceinline__ void weight_producer(Ctx &c, const FwdBufs &fb, const
         const bf16 *wl = op.W + (size_t)op_layer(P, q) * op.lstride;
         int t0, T, k_lo, k_hi;
         op_range(op, c.cta, c.ncta, t0, T, k_lo, k_hi);
-        for (int p = 0; p < n_passes(T); ++p) {
+        for (int p = 0; p < n_passes(T, P.max_tiles); ++p) {
             int p0, Tp;
-            pass_range(T, p, p0, Tp);
+            pass_range(T, p, P.max_tiles, p0, Tp);
             const int bytes = Tp * 2048;                 // two 8-row atoms per tile
             for (int k = k_lo; k < k_hi; k += KB, ++n) {
                 const int at = ring_place(head, bytes), end = at + bytes;
@@ -94,7 +94,7 @@ __device__ __forceinline__ void weight_producer(Ctx &c, const FwdBufs &fb, const
 // Lane 0 of warp MMA_ISSUER: the tensor-core instructions of every stage.  Per k block four MMAs of K = 16; the
 // A operand is the activation stage (128 rows are read from its base: values, remainders, then whatever follows
 // in shared memory, which only reaches accumulator lanes nobody reads), the B operand the weight stage.
-template <int NT>
+template <int NT, bool TWO>
 __device__ __forceinline__ void mma_issuer(Ctx &c, const FwdBufs &fb, const Plan &P) {
     constexpr int XS = x_stages(NT), XSTAGE_BYTES = xstage_bytes(NT), XKB_BYTES = 2 * NT * 1024;
     int n = 0, head = 0, m = 0, np = 0;
@@ -102,11 +102,12 @@ __device__ __forceinline__ void mma_issuer(Ctx &c, const FwdBufs &fb, const Plan
         const GemmOp &op = P.op[op_index(P, q)];
         int t0, T, k_lo, k_hi;
         op_range(op, c.cta, c.ncta, t0, T, k_lo, k_hi);
-        for (int p = 0; p < n_passes(T); ++p, ++np) {
+        for (int p = 0; p < n_passes(T, P.max_tiles); ++p, ++np) {
             int p0, Tp;
-            pass_range(T, p, p0, Tp);
+            pass_range(T, p, P.max_tiles, p0, Tp);
             const int bytes = Tp * 2048;
-            const uint32_t idesc = umma_idesc(Tp * 16);
+            const int T0 = TWO ? min(Tp, MMA_TILES) : Tp, T1 = Tp - T0;      // tiles of the first / second accumulator
+            const uint32_t idesc = umma_idesc(T0 * 16), idesc1 = umma_idesc(T1 ? T1 * 16 : 16);
             // the phase warps have copied the previous pass's accumulator out
             if (!wait_bar(fb, c.acc_empty, (((uint32_t)np) & 1u) ^ 1u, 11, np)) return;
             for (int k = k_lo; k < k_hi; k += KB, ++n) {
@@ -119,6 +120,13 @@ __device__ __forceinline__ void mma_issuer(Ctx &c, const FwdBufs &fb, const Plan
 #pragma unroll
                 for (int k16 = 0; k16 < 4; ++k16)
                     umma(c.tmem, umma_desc(a0 + k16 * 32), umma_desc(b0 + k16 * 32), idesc, (k > k_lo || k16 > 0) ? 1u : 0u);
+                if (TWO && T1) {                         // (only in the kernel variant with two accumulators: the common
+                                                         // variant's loop is the kernel's critical path and stays minimal)
+#pragma unroll
+                    for (int k16 = 0; k16 < 4; ++k16)
+                        umma(c.tmem + ACC_COLS, umma_desc(a0 + k16 * 32), umma_desc(b0 + T0 * 2048 + k16 * 32), idesc1,
+                             (k > k_lo || k16 > 0) ? 1u : 0u);
+                }
                 umma_commit(c.wempty + n % NB);
                 if (kx == XK - KB || k + KB >= k_hi) { umma_commit(c.xempty + xslot); ++m; }
             }
@@ -167,7 +175,7 @@ __device__ __forceinline__ void activation_producer(Ctx &c, const FwdBufs &fb, c
         wait_count(fb, c.ready_op, q + 1, 6);
         __threadfence_block();
         asm volatile("fence.proxy.async;" ::: "memory");
-        for (int p = 0; p < n_passes(T); ++p, ++np) {
+        for (int p = 0; p < n_passes(T, P.max_tiles); ++p, ++np) {
             if (p > 0) {
                 wait_count(fb, c.pass_done, np, 12);
                 __threadfence_block();
@@ -211,7 +219,7 @@ __device__ __forceinline__ void helper_warp(Ctx &c, const FwdBufs &fb, const Pla
 // and run epi(tile, acc) for the pass's 16-row tiles, warp w taking tiles w, w + 8.
 // Accumulator element (nt, i) as the epilogues see it: token row nt*8 + 2t + (i & 1), tile column g + 8*(i >> 1),
 // with g = lane / 4, t = lane % 4.  resid: rows added to the sums (the residual stream), or NULL.
-template <int NT, class Epi>
+template <int NT, bool TWO, class Epi>
 __device__ __forceinline__ void gemm_op(Ctx &c, const FwdBufs &fb, const Plan &P, int q, const float *resid, int resid_ld,
                                         Epi epi) {
     const GemmOp &op = P.op[op_index(P, q)];
@@ -225,48 +233,56 @@ __device__ __forceinline__ void gemm_op(Ctx &c, const FwdBufs &fb, const Plan &P
     op_range(op, c.cta, c.ncta, t0, T, k_lo, k_hi);
     float *stage = reinterpret_cast<float *>(c.scratch);
     const int g = c.lane >> 2, t = c.lane & 3;
-    for (int p = 0; p < n_passes(T); ++p) {
+    for (int p = 0; p < n_passes(T, P.max_tiles); ++p) {
         int p0, Tp;
-        pass_range(T, p, p0, Tp);
-        const int C = Tp * 16, pitch = C + 1;               // odd pitch: a warp's 32 lanes (rows) hit 32 banks
+        pass_range(T, p, P.max_tiles, p0, Tp);
         wait_bar(fb, c.acc_full, ((uint32_t)c.np) & 1u, 10, c.np);
         tc_fence_after();
-        {
-            const int quad = c.warp & 3;                     // the accumulator lanes this warp can read: 32 quad ..
-            if (quad * 32 < 16 * NT) {
-                for (int cg = c.warp >> 2; cg * 32 < C; cg += 2) {
-                    uint32_t v[32];
-                    tmem_ld32(c.tmem + ((uint32_t)(quad * 32) << 16) + (uint32_t)(cg * 32), v);
-                    float *row = stage + (size_t)(quad * 32 + c.lane) * pitch + cg * 32;
 #pragma unroll
-                    for (int j = 0; j < 32; ++j)
-                        if (cg * 32 + j < C) row[j] = __uint_as_float(v[j]);
+        for (int half = 0; half < (TWO ? 2 : 1); ++half) {                // one accumulator (at most 16 tiles) at a time
+            const int hbase = half * MMA_TILES;
+            if (TWO && hbase >= Tp) break;
+            const int Th = TWO ? min(MMA_TILES, Tp - hbase) : Tp;
+            const int C = Th * 16, pitch = C + 1;           // odd pitch: a warp's 32 lanes (rows) hit 32 banks
+            const uint32_t acc_at = c.tmem + (TWO && hbase ? ACC_COLS : 0);
+            if (TWO && hbase) bsync();                       // the first accumulator's copy has been read
+            {
+                const int quad = c.warp & 3;                 // the accumulator lanes this warp can read: 32 quad ..
+                if (quad * 32 < 16 * NT) {
+                    for (int cg = c.warp >> 2; cg * 32 < C; cg += 2) {
+                        uint32_t v[32];
+                        tmem_ld32(acc_at + ((uint32_t)(quad * 32) << 16) + (uint32_t)(cg * 32), v);
+                        float *row = stage + (size_t)(quad * 32 + c.lane) * pitch + cg * 32;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (cg * 32 + j < C) row[j] = __uint_as_float(v[j]);
+                    }
                 }
             }
-        }
-        tc_fence_before();
-        bsync();
-        if (threadIdx.x == 0) mbar_arrive(c.acc_empty);       // the next pass may overwrite the accumulator
-        if (normed) {
-            wait_count(fb, c.ready_op + 1, q + 1, 10);                 // 1/rms of this projection's input rows
-            __threadfence_block();
-        }
-        for (int ti = c.warp; ti < Tp; ti += MMA_WARPS) {
-            const int tile = t0 + p0 + ti;
-            float acc[NT][4];
+            tc_fence_before();
+            bsync();
+            if (threadIdx.x == 0 && (!TWO || hbase + MMA_TILES >= Tp)) mbar_arrive(c.acc_empty);   // the next pass may overwrite them
+            if (normed && (!TWO || hbase == 0)) {
+                wait_count(fb, c.ready_op + 1, q + 1, 10);             // 1/rms of this projection's input rows
+                __threadfence_block();
+            }
+            for (int ti = c.warp; ti < Th; ti += MMA_WARPS) {
+                const int tile = t0 + p0 + hbase + ti;
+                float acc[NT][4];
 #pragma unroll
-            for (int nt = 0; nt < NT; ++nt)
+                for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int r = nt * 8 + 2 * t + (i & 1), cc = ti * 16 + g + 8 * (i >> 1);
-                    float v = stage[(size_t)r * pitch + cc] + stage[(size_t)(8 * NT + r) * pitch + cc];
-                    if (resid) {
-                        const int n0 = tile * 16 + g + 8 * (i >> 1);
-                        if (n0 < op.N) v += __ldcg(resid + (size_t)r * resid_ld + n0);
+                    for (int i = 0; i < 4; ++i) {
+                        const int r = nt * 8 + 2 * t + (i & 1), cc = ti * 16 + g + 8 * (i >> 1);
+                        float v = stage[(size_t)r * pitch + cc] + stage[(size_t)(8 * NT + r) * pitch + cc];
+                        if (resid) {
+                            const int n0 = tile * 16 + g + 8 * (i >> 1);
+                            if (n0 < op.N) v += __ldcg(resid + (size_t)r * resid_ld + n0);
+                        }
+                        acc[nt][i] = v;
                     }
-                    acc[nt][i] = v;
-                }
-            epi(tile, acc);
+                epi(tile, acc);
+            }
         }
         fence_proxy_async();                   // the copy in shared memory is read; bulk copies may overwrite it
         bsync();
