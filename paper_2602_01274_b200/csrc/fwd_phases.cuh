@@ -82,10 +82,12 @@ __device__ __forceinline__ void phase_begin(Ctx &c, const Args &a, int nt_total)
     for (int tile = c.cta * MMA_WARPS + c.warp; tile < ntiles; tile += c.ncta * MMA_WARPS) {
         const int col = tile * 16 + col16;
         const float gain = __bfloat162float(m.norm1[col]);
-        for (int rr = 0; rr < rpad; rr += 2) {
-            const int r = rr + half;
+        float vv[MAX_ROWS / 2];                         // all rows' loads in flight together (the phase is a latency chain)
+#pragma unroll
+        for (int it = 0; it < MAX_ROWS / 2; ++it) {
+            const int r = 2 * it + half;
             float v = 0.f;
-            if (r < a.g.rtot && c.row_pos[r] >= 0) {
+            if (2 * it < rpad && r < a.g.rtot && c.row_pos[r] >= 0) {
                 const int s = r / a.g.rps, j = r - s * a.g.rps;
                 if (a.kind == KIND_MB) {
                     v = d.hpend[((size_t)s * (d.block_b + 1) + j) * dm + col];
@@ -97,6 +99,13 @@ __device__ __forceinline__ void phase_begin(Ctx &c, const Args &a, int nt_total)
                     v = __bfloat162float(m.embed[(size_t)c.row_tok[r] * dm + col]);
                 }
             }
+            vv[it] = v;
+        }
+#pragma unroll
+        for (int it = 0; it < MAX_ROWS / 2; ++it) {
+            if (2 * it >= rpad) break;
+            const int r = 2 * it + half;
+            const float v = vv[it];
             d.xres[(size_t)r * dm + col] = v;          // idle rows hold zeros: they stay finite through the layers
             store_split(a.fb.xg, nt_total, r, col, v * gain);
             float ss = v * v;
