@@ -159,7 +159,13 @@ __device__ __forceinline__ void attention_keys(Ctx &c, const bf16 *kcache, const
     constexpr int NCH = HD / 32, NOT = HD / 8, QP = SM::QP, VP = SM::VP;
     const int g = c.lane >> 2, t = c.lane & 3;
     const bf16 *kn = reinterpret_cast<const bf16 *>(c.scratch + SM::KN_OFF), *vn = reinterpret_cast<const bf16 *>(c.scratch + SM::VN_OFF);
-    unsigned char *vslot = c.scratch + SM::VS_OFF + c.warp * (16 * VP);
+    // With two query tiles, warps w and w + 4 walk the same key steps: warp w stages the V rows for both (they
+    // meet at a named barrier of 64 threads before and after the P V products).
+    const bool shared_v = KW == 4, loader = !shared_v || c.warp < 4;
+    unsigned char *vslot = c.scratch + SM::VS_OFF + (shared_v ? (c.warp & 3) : c.warp) * (16 * VP);
+    auto pair_sync = [&]() {
+        if (shared_v) asm volatile("bar.sync %0, 64;" ::"r"(3 + (c.warp & 3)) : "memory");
+    };
     const unsigned char *q0 = c.scratch + SM::Q_OFF + (mt * 16 + g) * QP + t * 16, *q1 = q0 + 8 * QP;
     const int steps_c = (hi - lo + 7) >> 3, steps_n = (n_new + 7) >> 3;
     for (int st = kw; st < steps_c + steps_n; st += KW) {
@@ -170,7 +176,7 @@ __device__ __forceinline__ void attention_keys(Ctx &c, const bf16 *kcache, const
         const size_t plane = fresh ? (size_t)32 * HD : kv_lo;
         // V of the step into this warp's slot: rows 0..7 the values of the 8 keys, rows 8..15 their remainders
         // (keys past the end repeat the last valid key: finite, and masked)
-        for (int i = c.lane; i < 16 * (HD / 8); i += 32) {
+        for (int i = c.lane; loader && i < 16 * (HD / 8); i += 32) {
             const int kr = i / (HD / 8), piece = i - kr * (HD / 8);
             const bf16 *src = vb + (kr >> 3) * plane + (size_t)min(key0 + (kr & 7), kend - 1) * HD + piece * 8;
             if (fresh) *reinterpret_cast<uint4 *>(vslot + kr * VP + piece * 16) = *reinterpret_cast<const uint4 *>(src);
@@ -247,6 +253,7 @@ __device__ __forceinline__ void attention_keys(Ctx &c, const bf16 *kcache, const
         // appear twice in the first product; the second adds (remainder of P) x (values of V).
         cp_async_wait_all();
         __syncwarp();
+        pair_sync();                                     // the slot is filled, for both warps of a pair
         const unsigned char *vrow = vslot + ((c.lane & 7) + ((c.lane >> 3) & 1) * 8) * VP + (c.lane >> 4) * 16;
 #pragma unroll
         for (int np = 0; np < NOT / 2; ++np) {
@@ -258,6 +265,7 @@ __device__ __forceinline__ void attention_keys(Ctx &c, const bf16 *kcache, const
             mma16816(o[2 * np + 1], pl[0], pl[1], 0u, 0u, vf[2], vf[3]);
         }
         __syncwarp();                                    // the slot is read; the next step may overwrite it
+        pair_sync();
     }
 #pragma unroll
     for (int hr = 0; hr < 2; ++hr) {
