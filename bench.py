@@ -123,7 +123,7 @@ def oracle_sample(cfg: synth.PairConfig, pair_cpu, prompt, n_prompt_s, max_new_s
 # dram__bytes_read.sum + dram__bytes_write.sum of a k_forward verify launch divided by its algorithmic bytes, from
 # the ncu capture summarised under profiles/ (traffic grows with the layer count like the algorithmic bytes do).
 # Taken with the kernel as it is now; None would be right after any later change to the kernel.
-NCU_TRAFFIC_RATIO = 1.007
+NCU_TRAFFIC_RATIO = 1.008
 
 
 def verify_forward_numbers(ctx, cfg, prompt, n_ver, n_warm):
@@ -158,7 +158,7 @@ def verify_forward_numbers(ctx, cfg, prompt, n_ver, n_warm):
     roofline = {"bound": "hbm", "kernel": "k_forward (one launch = one verify forward)", "achieved": gbs, "peak": peak,
                 "unit": "GB/s", "frac": gbs / peak, "peak_kind": f"of {peak_kind}", "traffic": vbytes * NCU_TRAFFIC_RATIO,
                 "traffic_note": "dram read + write bytes of one launch from the ncu capture of the 4-layer cut "
-                                "(profiles/k_forward_7b_l4_verify17.md: 1.007 x its algorithmic bytes), scaled to this "
+                                "(profiles/k_forward_7b_l4_verify17.md: 1.008 x its algorithmic bytes), scaled to this "
                                 "launch by its algorithmic bytes",
                 "launches_timed": fwd_n, "bytes_per_launch": vbytes, "weight_bytes_per_launch": weight_bytes / max(1, fwd_n),
                 "ms_per_launch": launch_ms}
