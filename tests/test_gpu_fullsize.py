@@ -1,8 +1,10 @@
 """GPU parity at the full 7B / 68M, 13B / 68M and 33B / 1.3B sizes, in the launch configuration the benchmark times
 (one cooperative launch per forward, one block per SM, 17 or 25 verify rows): all 32 / 40 / 62 layers at width
 4096 / 5120 / 7168 (the last with grouped-query attention) and the full LM head, against the fp64 oracle reading
-the same bf16 weights.  The prompt is short so that the oracle's prefill stays within seconds;
-the verify forward itself is the full one.  Logits within 2e-2; drafts bit-exact where the oracle's margins allow."""
+the same bf16 weights.  The prompt is short so that the oracle's prefill stays within seconds; the verify forward
+itself is the full one.  One more case runs the 7B pair behind a 520-token prompt (the oracle's prefill then takes a
+few minutes): that verify forward has the benchmark's attention shape too, 17 rows against 519 cached keys in 4
+key-range splits per head.  Logits within 2e-2; drafts bit-exact where the oracle's margins allow."""
 import dataclasses
 
 import numpy as np
@@ -19,14 +21,14 @@ LOGIT_TOL = 2e-2
 ALPHA_TOL = 2e-3
 
 
-@pytest.mark.parametrize("name", ["7b_68m", "13b_68m", "33b_1b3"])
-def test_verify_forward_full_size(name):
+@pytest.mark.parametrize("name,n_prompt", [("7b_68m", 4), ("13b_68m", 4), ("33b_1b3", 4), ("7b_68m", 520)])
+def test_verify_forward_full_size(name, n_prompt):
     import psutil
     from paper_2602_01274_b200 import binding as b
     need = 2.5 * synth.CONFIGS[name].target.streamed_weight_bytes()      # host copy of the weights + the oracle's buffers
     if psutil.virtual_memory().available < need:
         pytest.skip("not enough host memory for the oracle at this size")
-    cfg = dataclasses.replace(synth.CONFIGS[name], n_prompt=4, max_new=20)
+    cfg = dataclasses.replace(synth.CONFIGS[name], n_prompt=n_prompt, max_new=20)
     V, gc, bb = cfg.target.vocab, cfg.gamma_cap, cfg.block_b
     pair_gpu = synth.make_pair(cfg, seed=1, device="cuda:0")
     pair_cpu = {k: ({n: t.cpu() for n, t in v.items()} if isinstance(v, dict) else v.cpu()) for k, v in pair_gpu.items()}

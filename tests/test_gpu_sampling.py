@@ -60,11 +60,17 @@ def test_sampled_generate_matches_oracle(tiny, t0):
 
 def test_sampled_autoregressive_matches_oracle(tiny):
     b, cfg, ctx = tiny["b"], tiny["cfg"], tiny["ctx"]
-    out_o, margin = orc.generate_ar(tiny["T"], tiny["prompt"], 32, mode=1, seed=7)
-    tok, _ = ctx.pacer_generate_ar(tiny["prompt"], 32, mode=b.PACER_SAMPLE, seed=7)
-    if margin <= 2 * LOGIT_TOL:
-        pytest.skip("a perturbed top-1/top-2 gap lies within the tolerance on this seed")
-    np.testing.assert_array_equal(tok[0], out_o)
+    comparable = 0
+    for seed in range(7, 40):                      # seeds whose perturbed top-1/top-2 gaps all clear the tolerance
+        out_o, margin = orc.generate_ar(tiny["T"], tiny["prompt"], 32, mode=1, seed=seed)
+        if margin <= 2 * LOGIT_TOL:
+            continue
+        tok, _ = ctx.pacer_generate_ar(tiny["prompt"], 32, mode=b.PACER_SAMPLE, seed=seed)
+        np.testing.assert_array_equal(tok[0], out_o, err_msg=f"seed {seed}")
+        comparable += 1
+        if comparable == 3:
+            break
+    assert comparable >= 1, "no seed in 7..39 keeps every draw clear of a tie"
 
 
 def test_different_seeds_give_different_samples(tiny):

@@ -1,4 +1,5 @@
-"""GPU parity on shapes the tiny pair does not reach: 17 verify rows (two 16-row query tiles in attention, three
+"""GPU parity on shapes the tiny pair does not reach: 17 and 25 verify rows together with key-range splits of a head
+(the attention path of the full-size benchmark forwards), 17 verify rows (two 16-row query tiles in attention, three
 row tiles in the projections), head dimension 128, grouped-query attention, k-sliced residual projections, and a
 vocabulary large enough that a block runs the LM head in more than one pass.  Same rules as test_gpu_parity.py:
 logits within 2e-2 of the fp64 oracle reading the same bf16 weights; tokens and per-step lengths bit-exact,
@@ -29,6 +30,20 @@ SHAPES = {
     "long_ctx": synth.PairConfig("long_ctx", synth.ModelShape(2, 256, 2, 2, 512, 4096),
                                  synth.ModelShape(1, 128, 2, 2, 256, 4096), agree=0.8, n_prompt=700, max_new=16,
                                  gamma_max=12),
+    # the attention path of the 7B benchmark forward: 17 rows (two 16-row query tiles, the paired warps share the
+    # V staging) AND 4 key-range splits per head (merge pass after the grid barrier), hd 128
+    "tiles2_split4": synth.PairConfig("tiles2_split4", synth.ModelShape(2, 512, 4, 4, 1024, 4096),
+                                      synth.ModelShape(1, 128, 2, 2, 256, 4096), agree=0.8, n_prompt=300, max_new=20,
+                                      gamma_max=16),
+    # the attention path of the 33B benchmark forward: 25 rows, 2 key-range splits, grouped-query attention with
+    # 4 query heads per kv head, hd 128, and an LM head with 17 tiles per block (the two-accumulator kernel variant)
+    "gqa4_split2_rows25": synth.PairConfig("gqa4_split2_rows25", synth.ModelShape(2, 1024, 8, 2, 2048, 40000),
+                                           synth.ModelShape(1, 128, 2, 2, 256, 40000), agree=0.8, n_prompt=150,
+                                           max_new=28, gamma_max=24),
+    # the largest number of key-range splits (16), 17 rows, hd 128
+    "tiles2_split16": synth.PairConfig("tiles2_split16", synth.ModelShape(1, 256, 2, 2, 512, 4096),
+                                       synth.ModelShape(1, 128, 2, 2, 256, 4096), agree=0.8, n_prompt=1100, max_new=20,
+                                       gamma_max=16),
     # many layers: rounding of the activations between layers must not pile up over depth
     "deep": synth.PairConfig("deep", synth.ModelShape(48, 256, 4, 4, 512, 4096),
                              synth.ModelShape(1, 128, 2, 2, 256, 4096), agree=0.8, n_prompt=24, max_new=16,
@@ -88,15 +103,23 @@ def test_generate_matches_oracle(pair, t0):
     cfg, ctx = pair["cfg"], pair["ctx"]
     o = orc.Pacer(pair["T"], pair["D"], pair["B"], pair["max_ctx"], b=cfg.block_b, gamma_cap=cfg.gamma_cap, t0=t0,
                   rho=cfg.rho)
-    out_o, dl_o, al_o, st_o = o.generate(pair["prompt"], cfg.max_new)
-    safe = st_o["min_margin_target"] > 2 * LOGIT_TOL and st_o["min_margin_draft"] > 2 * LOGIT_TOL and \
-        (t0 < 0 or st_o["min_margin_stop"] > ALPHA_TOL)
-    tok, ns, dl, al, st = ctx.pacer_generate(pair["prompt"], cfg.max_new, cfg.gamma_max, t0)
-    ar, _ = ctx.pacer_generate_ar(pair["prompt"], cfg.max_new)
-    if not safe:
-        pytest.skip("an oracle decision lies within the tolerance of a tie on this seed")
-    np.testing.assert_array_equal(tok[0], out_o)
-    np.testing.assert_array_equal(ar[0], out_o)            # lossless: speculative output == autoregressive output
-    assert ns[0] == len(dl_o)
-    np.testing.assert_array_equal(dl[0, : ns[0]], dl_o)
-    np.testing.assert_array_equal(al[0, : ns[0]], al_o)
+    # The comparison is exact only where no decision of the oracle lies within the tolerance of a tie: take the
+    # first prompt seeds on which that holds (never skip: at least one seed must be comparable).
+    comparable = 0
+    for seed in range(3, 11):
+        prompt = pair["prompt"] if seed == 3 else synth.make_prompts(cfg.target.vocab, 1, cfg.n_prompt, seed=seed)[0].numpy()
+        out_o, dl_o, al_o, st_o = o.generate(prompt, cfg.max_new)
+        safe = st_o["min_margin_target"] > 2 * LOGIT_TOL and st_o["min_margin_draft"] > 2 * LOGIT_TOL and \
+            (t0 < 0 or st_o["min_margin_stop"] > ALPHA_TOL)
+        if not safe:
+            continue
+        tok, ns, dl, al, st = ctx.pacer_generate(prompt, cfg.max_new, cfg.gamma_max, t0)
+        ar, _ = ctx.pacer_generate_ar(prompt, cfg.max_new)
+        np.testing.assert_array_equal(tok[0], out_o)
+        np.testing.assert_array_equal(ar[0], out_o)            # lossless: speculative output == autoregressive output
+        assert ns[0] == len(dl_o)
+        np.testing.assert_array_equal(dl[0, : ns[0]], dl_o)
+        np.testing.assert_array_equal(al[0, : ns[0]], al_o)
+        comparable += 1
+        break
+    assert comparable >= 1, "no prompt seed in 3..10 keeps every oracle decision clear of a tie"

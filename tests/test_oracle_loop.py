@@ -298,6 +298,43 @@ def test_sampled_output_follows_the_target_distribution(loop):
     assert chi2 < chi2_dist.ppf(0.999, len(e) - 1), (chi2, len(e))
 
 
+def test_sampled_autoregressive_output_follows_the_target_distribution():
+    """Eq. 1 under temperature-1 sampling: the first two tokens the oracle's autoregressive loop draws over 20000
+    seeds against the target's exactly enumerated joint distribution (V = 8; sparse cells pooled).  The joint
+    comes from the separately pinned forward by teacher forcing, so a wrong position, tag or logit row in the
+    sampled loop fails the chi-square."""
+    V = 8
+    T_s = synth.ModelShape(1, 16, 2, 2, 32, V)
+    wt = synth.make_model(T_s, "target", seed=31, std=0.6)
+    T = orc.OracleModel(T_s, wt)
+    prompt = np.array([4, 0, 6], np.int32)
+    sm = lambda v: np.exp(v - v.max()) / np.exp(v - v.max()).sum()
+    _, lg = orc.forward(T, orc.Cache(T, 8), tokens=prompt)
+    p1 = sm(lg[-1])
+    joint = np.zeros((V, V))
+    for a in range(V):
+        _, lg2 = orc.forward(T, orc.Cache(T, 8), tokens=np.append(prompt, a).astype(np.int32))
+        joint[a] = p1[a] * sm(lg2[-1])
+    assert joint.max() < 0.6, "the distribution should not be degenerate"
+    N = 20000
+    counts = np.zeros((V, V))
+    for s in range(N):
+        out, _ = orc.generate_ar(T, prompt, 2, mode=1, seed=9000 + s)
+        counts[out[0], out[1]] += 1
+    exp = (N * joint).ravel()
+    cnt = counts.ravel()
+    big = exp >= 10.0
+    e = np.append(exp[big], exp[~big].sum())
+    c = np.append(cnt[big], cnt[~big].sum())
+    assert len(e) >= 8
+    from scipy.stats import chi2 as chi2_dist
+    chi2 = ((c - e) ** 2 / e).sum()
+    assert chi2 < chi2_dist.ppf(0.999, len(e) - 1), (chi2, len(e))
+    # greedy mode of the same loop is the arg-max chain of the same forward
+    out_g, _ = orc.generate_ar(T, prompt, 2, mode=0)
+    assert out_g[0] == int(np.argmax(p1)) and out_g[1] == int(np.argmax(joint[out_g[0]]))
+
+
 def test_preverify_inputs_are_hidden_plus_position_embedding_of_the_draft_index():
     """Eq. 7 wiring: row of draft i (1-based within the step, continuing over
     blocks) gets e_i = PosEmb row i-1; a catch-up history row gets none; alpha_hat
