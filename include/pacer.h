@@ -66,6 +66,10 @@ typedef struct {
     int32_t criterion;       /* block statistic: 0 mean (the method), 1 minimum ("any"), 2 last token */
     float succ_bias;         /* added to logit succ[input token] of every LM-head row; 0 = off */
     int32_t use_posemb;      /* 1: add the draft position embedding e_i (the method); 0: ablation */
+    int32_t mb_scope;        /* attention context of M_B ("attention context" ablation): 0 full = its whole KV cache
+                                (the method), 1 local draft = the drafts of the current step, 2 local block = the
+                                drafts of the current block.  A restricted context starts at the first draft row of
+                                the step / block; history rows are outside it and attend to themselves only. */
 } pacer_cfg;
 
 /* One named weight tensor, bf16, contiguous, on the device.  Names per model:
@@ -106,7 +110,7 @@ typedef struct {
     int32_t n_steps;            /* draft-and-verify steps completed */
     int32_t last_n, last_next;  /* accepted drafts and the follow-up token of the last step */
     int32_t n_pend;             /* draft hidden rows not yet given to M_B */
-    int32_t err;                /* device status word of this sequence, 0 = fine */
+    int32_t err;                /* unused, 0 (the device status word is per context: PACER_EDEVICE) */
     int64_t n_draft_fwd, n_mb_calls, n_target_fwd;
 } pacer_seq_state;
 
@@ -183,20 +187,36 @@ int pacer_preverify(pacer_ctx *ctx);
  * (Eq. 4), appending their K/V rows and leaving logits p_1..p_{gamma+1}. */
 int pacer_verify(pacer_ctx *ctx);
 
-/* Acceptance (Eq. 5; greedy = prefix match with the target's argmax), commit of
+/* Acceptance after a pacer_verify call (Eq. 5; greedy = prefix match with the target's argmax), commit of
  * [y_1..y_n, next], truncation of the three caches to the accepted rows, reset of
  * the per-step state, logging of (gamma, n). Uses the mode and seed of pacer_prefill. */
 int pacer_accept_rollback(pacer_ctx *ctx);
 
-/* [sync] Copies the per-sequence scalars of sequences 0..batch-1 to host memory. */
+/* Test hook for the error path: writes the device status word exactly as a kernel's
+ * bounded wait that ran out would (code != 0, and the block, warp and detail it
+ * records).  Until the next pacer_prefill / pacer_generate* resets the word, every
+ * [sync] entry point returns PACER_EDEVICE with the decoded text, and forwards
+ * launched meanwhile fall through their waits.  No kernel is launched.  [sync] */
+int pacer_debug_set_device_status(pacer_ctx *ctx, int code, int block, int warp, int detail);
+
+/* [sync] Copies the per-sequence scalars of sequences 0..batch-1 to host memory.
+ * Returns PACER_EDEVICE (after filling `out`) when the device status word is set. */
 int pacer_read_state(pacer_ctx *ctx, pacer_seq_state *out, int batch);
 
-/* [sync] Copies `bytes` bytes from the start of one device buffer (PACER_BUF_*) to host memory. */
+/* [sync] Copies `bytes` bytes from the start of one device buffer (PACER_BUF_*) to host memory.
+ * Returns PACER_EDEVICE (after the copy) when the device status word is set. */
 int pacer_read_buffer(pacer_ctx *ctx, int which, void *host_dst, size_t bytes);
 
 /* [sync] Algorithm 1 end to end: prefill, then draft-and-verify steps until every
- * sequence has max_new new tokens, all steps enqueued as device-side controlled
- * work (no host decision per token or per step).  Outputs, all host, caller-owned:
+ * sequence has max_new new tokens.  Every decision of the loop (rows of a forward,
+ * stop of the drafting, acceptance, rollback, end of generation) is taken on the
+ * device; the host enqueues whole steps (every block of the window, each a no-op
+ * for a sequence that has stopped drafting) and stays two steps ahead of the device:
+ * it reads the finished flags of an EARLIER step from pinned memory (copied there
+ * behind an event) to know when to stop enqueuing, and never waits for the step it
+ * has just enqueued.  Greedy runs take the acceptance (Eq. 5) in the tail of the
+ * verify forward; sampling runs in a kernel of its own.
+ * Outputs, all host, caller-owned:
  *   out_tokens     int32 [batch][max_new]
  *   out_n_steps    int32 [batch]
  *   out_draft_len  int32 [batch][max_new]  gamma of step s, -1 beyond n_steps
@@ -205,6 +225,20 @@ int pacer_read_buffer(pacer_ctx *ctx, int which, void *host_dst, size_t bytes);
 int pacer_generate(pacer_ctx *ctx, const int32_t *prompt, int batch, int n_prompt, int max_new, int gamma_max,
                    float threshold, int mode, uint64_t seed, int32_t *out_tokens, int32_t *out_n_steps,
                    int32_t *out_draft_len, int32_t *out_accept_len, pacer_stats *stats);
+
+/* [sync] Speculative decoding (Section 2.2) with the draft window of every step
+ * PRESCRIBED instead of decided by the pre-verification model: step s of sequence q
+ * drafts windows[q][s] tokens (host int32 [batch][n_windows], each in [0, gamma_cap];
+ * 0 = a plain target step; steps beyond n_windows reuse the last entry).  With
+ * windows = the accepted lengths of a large-window run of the same prompt this is
+ * decoding with the optimal draft length gamma* of Section 3.1 (the upper bound an
+ * oracle-knowledge window reaches).  M_B is not run.  The draft model catches up, in
+ * the first forward of its next window, on the rows it has not seen; such a forward
+ * holds at most 16 rows per sequence (32 / batch if that is less), and when the
+ * backlog reaches that number a prescribed 0 becomes 1.  Outputs as pacer_generate. */
+int pacer_generate_sched(pacer_ctx *ctx, const int32_t *prompt, int batch, int n_prompt, int max_new,
+                         const int32_t *windows, int n_windows, int mode, uint64_t seed, int32_t *out_tokens,
+                         int32_t *out_n_steps, int32_t *out_draft_len, int32_t *out_accept_len, pacer_stats *stats);
 
 /* [sync] Autoregressive decoding of the target alone on the same kernels (Eq. 1):
  * the baseline, and under greedy decoding the definition of the lossless output. */
@@ -222,8 +256,9 @@ int pacer_generate_ar(pacer_ctx *ctx, const int32_t *prompt, int batch, int n_pr
 int pacer_profile_begin(pacer_ctx *ctx);
 int pacer_profile_end(pacer_ctx *ctx, double *fwd_ms, double *fwd_weight_bytes, int64_t *fwd_launches);
 
-/* Y[r][n] = sum_k X[r][k] * W[n][k]: the skinny weight-streaming product used by
- * every projection, exposed for kernel-level checks and timing.  x: device bf16
+/* Y[r][n] = sum_k X[r][k] * W[n][k]: a stand-alone skinny weight-streaming product
+ * (a split-k kernel on mma.sync with plain bf16 activations; the projections inside
+ * the forwards run on a different, tcgen05 path with split activations).  x: device bf16
  * [rows][K] row-major; w: device bf16 [N][K]; y: device f32 [rows][N];
  * scratch: device, at least pacer_linear_scratch_bytes(rows, N, K) bytes.
  * rows <= 32, K a multiple of 32.  Enqueues on `cuda_stream`. */

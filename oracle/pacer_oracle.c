@@ -20,6 +20,9 @@
  *                         case is the same rule with one-hot distributions.
  *   orc_generate_pacer    Algorithm 1 as a whole.
  *   orc_generate_sd       Section 2.2 (fixed window), written separately.
+ *   orc_generate_sched    Section 2.2 with a window given per step; with the windows
+ *                         L_A* of a large-window run it is the gamma* decoding of
+ *                         Section 3.1 (the oracle-knowledge upper bound).
  *   orc_generate_ar       Eq. 1 on the target: the definition of the lossless output.
  *
  * Readings of the paper taken where it is silent (each also listed in the design
@@ -30,7 +33,9 @@
  * with a two-row forward after a fully accepted step; M_B is one decoder layer at
  * draft width with its own KV cache, RMSNorm and a 2-way linear head, alpha_hat =
  * softmax(.)[1]; rows of accepted history carry no position embedding; M_B's
- * cache is truncated together with the draft's.
+ * cache is truncated together with the draft's.  The restricted attention
+ * contexts of the ablation ("local draft", "local block") start at the first
+ * draft row of the step / of the block; a history row then sees itself only.
  *
  * Parity pins live in tests/test_oracle_*.py.  Unpinned: the architecture of M_B
  * against the authors' trained module (no checkpoint exists here) - "parity
@@ -69,6 +74,8 @@ typedef struct {
     uint64_t seed;
     int32_t seq_id;
     int32_t use_posemb;  /* 1: add e_i to draft rows (the method); 0: ablation */
+    int32_t scope;       /* attention context of M_B: 0 full (the method), 1 local draft, 2 local block */
+    int32_t pad_;
 } orc_params;
 
 typedef struct {
@@ -98,6 +105,7 @@ typedef struct {
     real *alpha;         /* [gamma_cap] alpha_hat of the drafts of this step */
     real *plogits;       /* [gamma_cap+1][V] target logits of the last verify */
     int32_t last_n, last_next;
+    int32_t mb_start;    /* M_B cache position of the first draft row of this step (scope 1) */
     const real *alpha_override; int32_t n_alpha_override, alpha_override_pos; /* test hook */
     orc_stats st;
 } orc_state;
@@ -178,8 +186,25 @@ void orc_cache_truncate(orc_cache *c, int len) { c->len = len; }
  * written to the cache at their positions and the cache length becomes pos0+n.
  * hidden_out [n][d]: output of the final RMSNorm.  logits_out [n][V]: LM head,
  * plus succ_bias on token succ[tokens[j]] of row j when a table is present. */
+static void forward_from(const orc_model *m, orc_cache *c, const int32_t *tokens, const real *x_in,
+                         int n, int pos0, int key_start, real *hidden_out, real *logits_out);
+
 void orc_forward(const orc_model *m, orc_cache *c, const int32_t *tokens, const real *x_in,
                  int n, int pos0, real *hidden_out, real *logits_out) {
+    forward_from(m, c, tokens, x_in, n, pos0, 0, hidden_out, logits_out);
+}
+
+/* The same forward with a restricted attention context (the "attention context"
+ * ablation of the pre-verification layer): the row at position pos attends to the
+ * cache positions key_start..pos; a row that lies before key_start attends to
+ * itself only.  key_start = 0 is ordinary causal attention. */
+void orc_forward_scoped(const orc_model *m, orc_cache *c, const int32_t *tokens, const real *x_in,
+                        int n, int pos0, int key_start, real *hidden_out, real *logits_out) {
+    forward_from(m, c, tokens, x_in, n, pos0, key_start, hidden_out, logits_out);
+}
+
+static void forward_from(const orc_model *m, orc_cache *c, const int32_t *tokens, const real *x_in,
+                         int n, int pos0, int key_start, real *hidden_out, real *logits_out) {
     const int d = m->d_model, H = m->n_heads, Hkv = m->n_kv_heads, hd = d / H, F = m->d_ffn;
     const int kvd = Hkv * hd, qrows = (H + 2 * Hkv) * hd, group = H / Hkv;
     real *x = (real *)malloc(sizeof(real) * (size_t)n * d);
@@ -209,12 +234,13 @@ void orc_forward(const orc_model *m, orc_cache *c, const int32_t *tokens, const 
             memcpy(cv + (size_t)pos * kvd, vv, sizeof(real) * kvd);
         }
         for (int r = 0; r < n; ++r) {
-            int pos = pos0 + r;               /* causal: keys 0..pos */
+            int pos = pos0 + r;               /* causal: keys first..pos (first = 0 unless the context is restricted) */
+            int first = key_start < pos ? key_start : pos;
             for (int h = 0; h < H; ++h) {
                 const real *q = qkv + (size_t)r * qrows + h * hd;
                 int kh = h / group;
                 real mx = -INFINITY;
-                for (int p = 0; p <= pos; ++p) {
+                for (int p = first; p <= pos; ++p) {
                     const real *kp = ck + (size_t)p * kvd + kh * hd;
                     real s = 0;
                     for (int i = 0; i < hd; ++i) s += q[i] * kp[i];
@@ -222,10 +248,10 @@ void orc_forward(const orc_model *m, orc_cache *c, const int32_t *tokens, const 
                     if (sc[p] > mx) mx = sc[p];
                 }
                 real den = 0;
-                for (int p = 0; p <= pos; ++p) { sc[p] = exp(sc[p] - mx); den += sc[p]; }
+                for (int p = first; p <= pos; ++p) { sc[p] = exp(sc[p] - mx); den += sc[p]; }
                 real *out = att + (size_t)r * H * hd + h * hd;
                 for (int i = 0; i < hd; ++i) out[i] = 0;
-                for (int p = 0; p <= pos; ++p) {
+                for (int p = first; p <= pos; ++p) {
                     const real *vp = cv + (size_t)p * kvd + kh * hd;
                     real w = sc[p] / den;
                     for (int i = 0; i < hd; ++i) out[i] += w * vp[i];
@@ -481,7 +507,14 @@ double orc_preverify(orc_state *s) {
             xin[(size_t)r * d + i] = v;
         }
     }
-    orc_forward(B, s->cB, NULL, xin, n, s->cB->len, hid, NULL);
+    /* attention context (Section 5, "attention context" ablation): full = the whole cache (the method);
+     * local draft = the drafts of this step; local block = the drafts of this block.  History rows
+     * (a catch-up row comes first in the step's first call) are never part of a restricted context. */
+    int n_hist = 0;
+    while (n_hist < n && s->hpend_e[n_hist] == 0) n_hist += 1;
+    if (s->gamma == b) s->mb_start = s->cB->len + n_hist;      /* first call of the step */
+    int key_start = s->prm.scope == 2 ? s->cB->len + n_hist : s->prm.scope == 1 ? s->mb_start : 0;
+    forward_from(B, s->cB, NULL, xin, n, s->cB->len, key_start, hid, NULL);
     s->st.n_mb_calls += 1;
     for (int r = 0; r < n; ++r) {
         int e = s->hpend_e[r];
@@ -617,6 +650,63 @@ int orc_generate_sd(const orc_model *T, const orc_model *D, const int32_t *promp
     for (int i = 0; i < max_new; ++i) out_tokens[i] = x[n_prompt + i];
     if (stats) *stats = st;
     orc_cache_free(cT); orc_cache_free(cD); free(x); free(y); free(in); free(ql); free(pl); free(lg);
+    return steps;
+}
+
+/* Speculative decoding (Section 2.2) whose window is prescribed per step: step s
+ * drafts windows[s] tokens (0 = a plain target step), steps past n_windows reuse
+ * the last entry.  With windows[s] = the accepted length L_A* of step s of a
+ * large-window run this is decoding with the optimal draft length gamma* of
+ * Section 3.1 (every draft is accepted, no forward is wasted).  The draft model
+ * catches up on the rows it has not seen (one forward) when it next drafts. */
+int orc_generate_sched(const orc_model *T, const orc_model *D, const int32_t *prompt, int n_prompt, int max_new,
+                       const int32_t *windows, int n_windows, int mode, uint64_t seed, int seq, int max_ctx,
+                       int32_t *out_tokens, int32_t *draft_len, int32_t *accept_len, orc_stats *stats) {
+    const int V = T->vocab;
+    int gmax = 1;
+    for (int i = 0; i < n_windows; ++i) if (windows[i] > gmax) gmax = windows[i];
+    orc_cache *cT = orc_cache_new(T, max_ctx), *cD = orc_cache_new(D, max_ctx);
+    int32_t *x = (int32_t *)calloc(max_ctx, sizeof(int32_t)), *y = (int32_t *)calloc(gmax, sizeof(int32_t));
+    int32_t *in = (int32_t *)calloc(gmax + 1, sizeof(int32_t));
+    real *ql = (real *)malloc(sizeof(real) * (size_t)gmax * V), *pl = (real *)malloc(sizeof(real) * (size_t)(gmax + 1) * V);
+    orc_stats st; stats_reset(&st);
+    memcpy(x, prompt, sizeof(int32_t) * n_prompt);
+    int P = n_prompt, steps = 0;
+    if (P > 1) { orc_forward(T, cT, x, NULL, P - 1, 0, NULL, NULL); orc_forward(D, cD, x, NULL, P - 1, 0, NULL, NULL); }
+    while (P - n_prompt < max_new) {
+        const int gamma = windows[steps < n_windows ? steps : n_windows - 1];
+        for (int i = 0; i < gamma; ++i) {
+            int pos0 = cD->len, n_in = (i == 0) ? (P - pos0) : 1;   /* all rows the draft has not seen yet */
+            const int32_t *src = (i == 0) ? (x + pos0) : (y + i - 1);
+            real *lg = (real *)malloc(sizeof(real) * (size_t)n_in * V);
+            orc_forward(D, cD, src, NULL, n_in, pos0, NULL, lg);
+            st.n_draft_fwd += 1;
+            const real *lrow = lg + (size_t)(n_in - 1) * V;
+            real mg;
+            y[i] = (mode == 0) ? argmax_margin(lrow, V, &mg) : sample_gumbel(lrow, V, seed, P + i, seq, TAG_DRAFT, &mg);
+            if (mg < st.min_margin_draft) st.min_margin_draft = mg;
+            memcpy(ql + (size_t)i * V, lrow, sizeof(real) * V);
+            free(lg);
+        }
+        in[0] = x[P - 1];
+        for (int i = 0; i < gamma; ++i) in[i + 1] = y[i];
+        orc_forward(T, cT, in, NULL, gamma + 1, P - 1, NULL, pl);
+        st.n_target_fwd += 1;
+        int32_t next; double mt, ma;
+        int n = orc_accept_rule(pl, ql, y, gamma, V, mode, seed, P, seq, &next, &mt, &ma);
+        if (mt < st.min_margin_target) st.min_margin_target = mt;
+        if (ma < st.min_margin_accept) st.min_margin_accept = ma;
+        for (int i = 0; i < n; ++i) x[P + i] = y[i];
+        x[P + n] = next;
+        cT->len = P + n;
+        if (gamma > 0) cD->len = (n < gamma) ? P + n : P + gamma - 1;   /* a step without drafts leaves the draft cache alone */
+        P += n + 1;
+        draft_len[steps] = gamma; accept_len[steps] = n;
+        steps += 1; st.n_steps += 1;
+    }
+    for (int i = 0; i < max_new; ++i) out_tokens[i] = x[n_prompt + i];
+    if (stats) *stats = st;
+    orc_cache_free(cT); orc_cache_free(cD); free(x); free(y); free(in); free(ql); free(pl);
     return steps;
 }
 

@@ -43,7 +43,7 @@ class Model(C.Structure):
 class Params(C.Structure):
     _fields_ = [("b", C.c_int32), ("gamma_cap", C.c_int32), ("t0", C.c_float), ("rho", C.c_float),
                 ("criterion", C.c_int32), ("mode", C.c_int32), ("seed", C.c_uint64),
-                ("seq_id", C.c_int32), ("use_posemb", C.c_int32)]
+                ("seq_id", C.c_int32), ("use_posemb", C.c_int32), ("scope", C.c_int32), ("pad_", C.c_int32)]
 
 
 class Stats(C.Structure):
@@ -70,6 +70,8 @@ def lib():
         L.orc_cache_truncate.argtypes = [C.c_void_p, C.c_int]
         L.orc_forward.argtypes = [C.POINTER(Model), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int,
                                   C.c_void_p, C.c_void_p]
+        L.orc_forward_scoped.argtypes = [C.POINTER(Model), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int,
+                                         C.c_void_p, C.c_void_p]
         L.orc_linear.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_int, C.c_void_p]
         L.orc_philox4x32_10.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
         L.orc_uniform.restype = C.c_double
@@ -90,6 +92,9 @@ def lib():
         L.orc_generate_sd.argtypes = [C.POINTER(Model), C.POINTER(Model), C.c_void_p, C.c_int, C.c_int, C.c_int,
                                       C.c_int, C.c_uint64, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p,
                                       C.POINTER(Stats)]
+        L.orc_generate_sched.argtypes = [C.POINTER(Model), C.POINTER(Model), C.c_void_p, C.c_int, C.c_int, C.c_void_p,
+                                         C.c_int, C.c_int, C.c_uint64, C.c_int, C.c_int, C.c_void_p, C.c_void_p,
+                                         C.c_void_p, C.POINTER(Stats)]
         L.orc_generate_ar.argtypes = [C.POINTER(Model), C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_uint64,
                                       C.c_int, C.c_int, C.c_void_p, C.c_void_p]
         for name in ("orc_get_P", "orc_get_gamma", "orc_get_drafting", "orc_get_last_n", "orc_get_last_next",
@@ -187,8 +192,9 @@ class Cache:
 
 
 def forward(model: OracleModel, cache: Cache, tokens=None, x_in=None, pos0: Optional[int] = None,
-            want_hidden=True, want_logits=True):
-    """Decoder forward on n new rows; returns (hidden [n][d], logits [n][V])."""
+            want_hidden=True, want_logits=True, key_start: int = 0):
+    """Decoder forward on n new rows; returns (hidden [n][d], logits [n][V]).  key_start > 0 restricts the
+    attention context to the cache positions key_start.. (a row before key_start sees itself only)."""
     if tokens is not None:
         tok = np.ascontiguousarray(np.asarray(tokens, dtype=np.int32))
         n = tok.shape[0]
@@ -202,7 +208,10 @@ def forward(model: OracleModel, cache: Cache, tokens=None, x_in=None, pos0: Opti
     s = model.shape
     hid = np.empty((n, s.d_model), np.float64) if want_hidden else None
     lg = np.empty((n, s.vocab), np.float64) if (want_logits and model.c.head) else None
-    lib().orc_forward(model.ref(), cache.h, _ptr(tok), _ptr(xin), n, pos0, _ptr(hid), _ptr(lg))
+    if key_start:
+        lib().orc_forward_scoped(model.ref(), cache.h, _ptr(tok), _ptr(xin), n, pos0, key_start, _ptr(hid), _ptr(lg))
+    else:
+        lib().orc_forward(model.ref(), cache.h, _ptr(tok), _ptr(xin), n, pos0, _ptr(hid), _ptr(lg))
     return hid, lg
 
 
@@ -249,9 +258,9 @@ class Pacer:
     """Algorithm 1 with access to every stage (for stage-by-stage comparisons)."""
 
     def __init__(self, T: OracleModel, D: OracleModel, B: Optional[OracleModel], max_ctx: int, b=4, gamma_cap=8,
-                 t0=0.5, rho=1.05, criterion=0, mode=0, seed=0, seq_id=0, use_posemb=1):
+                 t0=0.5, rho=1.05, criterion=0, mode=0, seed=0, seq_id=0, use_posemb=1, scope=0):
         self.T, self.D, self.B, self.max_ctx = T, D, B, max_ctx
-        self.prm = Params(b, gamma_cap, t0, rho, criterion, mode, seed, seq_id, use_posemb)
+        self.prm = Params(b, gamma_cap, t0, rho, criterion, mode, seed, seq_id, use_posemb, scope, 0)
         self.h = lib().orc_new(T.ref(), D.ref(), B.ref() if B else None, max_ctx, C.byref(self.prm))
         self._override = None
 
@@ -354,6 +363,23 @@ def generate_sd(T: OracleModel, D: OracleModel, prompt, max_new, gamma, mode=0, 
     st = Stats()
     steps = lib().orc_generate_sd(T.ref(), D.ref(), _ptr(p), p.shape[0], max_new, gamma, mode, seed, seq, max_ctx,
                                   _ptr(out), _ptr(dl), _ptr(al), C.byref(st))
+    return out, dl[:steps], al[:steps], st.as_dict()
+
+
+def generate_sched(T: OracleModel, D: OracleModel, prompt, max_new, windows, mode=0, seed=0, seq=0, max_ctx=None):
+    """Speculative decoding with the window of every step prescribed (Section 3.1's gamma* when the windows are the
+    accepted lengths of a large-window run).  Returns (tokens, draft_len, accept_len, stats)."""
+    p = np.ascontiguousarray(np.asarray(prompt, dtype=np.int32))
+    w = np.ascontiguousarray(np.asarray(windows, dtype=np.int32))
+    assert w.ndim == 1 and w.shape[0] >= 1 and w.min() >= 0
+    if max_ctx is None:
+        max_ctx = p.shape[0] + max_new + int(w.max()) + 2
+    out = np.zeros(max_new, np.int32)
+    dl = np.full(max_new, -1, np.int32)
+    al = np.full(max_new, -1, np.int32)
+    st = Stats()
+    steps = lib().orc_generate_sched(T.ref(), D.ref(), _ptr(p), p.shape[0], max_new, _ptr(w), w.shape[0], mode, seed,
+                                     seq, max_ctx, _ptr(out), _ptr(dl), _ptr(al), C.byref(st))
     return out, dl[:steps], al[:steps], st.as_dict()
 
 

@@ -38,7 +38,7 @@ class ModelCfg(C.Structure):
 class Cfg(C.Structure):
     _fields_ = [("target", ModelCfg), ("draft", ModelCfg), ("max_batch", C.c_int32), ("max_ctx", C.c_int32),
                 ("gamma_cap", C.c_int32), ("block_b", C.c_int32), ("rho", C.c_float), ("criterion", C.c_int32),
-                ("succ_bias", C.c_float), ("use_posemb", C.c_int32)]
+                ("succ_bias", C.c_float), ("use_posemb", C.c_int32), ("mb_scope", C.c_int32)]
 
 
 class Tensor(C.Structure):
@@ -78,10 +78,13 @@ _lib.pacer_load_weights.argtypes = [_P, C.c_int, C.POINTER(Tensor), C.c_int, _P]
 _lib.pacer_prefill.argtypes = [_P, _P, C.c_int, C.c_int, C.c_int, C.c_int, C.c_float, C.c_int, C.c_uint64]
 for _n in ("pacer_draft_step", "pacer_preverify", "pacer_verify", "pacer_accept_rollback"):
     getattr(_lib, _n).argtypes = [_P]
+_lib.pacer_debug_set_device_status.argtypes = [_P, C.c_int, C.c_int, C.c_int, C.c_int]
 _lib.pacer_read_state.argtypes = [_P, C.POINTER(SeqState), C.c_int]
 _lib.pacer_read_buffer.argtypes = [_P, C.c_int, _P, C.c_size_t]
 _lib.pacer_generate.argtypes = [_P, _P, C.c_int, C.c_int, C.c_int, C.c_int, C.c_float, C.c_int, C.c_uint64,
                                 _P, _P, _P, _P, C.POINTER(Stats)]
+_lib.pacer_generate_sched.argtypes = [_P, _P, C.c_int, C.c_int, C.c_int, _P, C.c_int, C.c_int, C.c_uint64,
+                                      _P, _P, _P, _P, C.POINTER(Stats)]
 _lib.pacer_generate_ar.argtypes = [_P, _P, C.c_int, C.c_int, C.c_int, C.c_int, C.c_uint64, _P, C.POINTER(Stats)]
 _lib.pacer_profile_begin.argtypes = [_P]
 _lib.pacer_profile_end.argtypes = [_P, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_int64)]
@@ -100,7 +103,8 @@ def exported_symbols():
     """The C entry points this binding resolved (all declared in pacer.h)."""
     return ["pacer_strerror", "pacer_last_error", "pacer_workspace_bytes", "pacer_create", "pacer_destroy",
             "pacer_load_weights", "pacer_prefill", "pacer_draft_step", "pacer_preverify", "pacer_verify",
-            "pacer_accept_rollback", "pacer_read_state", "pacer_read_buffer", "pacer_generate", "pacer_generate_ar",
+            "pacer_accept_rollback", "pacer_read_state", "pacer_read_buffer", "pacer_generate", "pacer_generate_sched",
+            "pacer_generate_ar", "pacer_debug_set_device_status",
             "pacer_profile_begin", "pacer_profile_end", "pacer_linear_scratch_bytes", "pacer_linear", "pacer_linear_static"]
 
 
@@ -109,10 +113,10 @@ def _model_cfg(s) -> ModelCfg:
 
 
 def make_cfg(target, draft, max_batch, max_ctx, gamma_cap, block_b=4, rho=1.05, criterion=0, succ_bias=8.0,
-             use_posemb=1) -> Cfg:
+             use_posemb=1, mb_scope=0) -> Cfg:
     """target/draft: objects with n_layers, d_model, n_heads, n_kv_heads, d_ffn, vocab, rope_theta, rms_eps."""
     return Cfg(_model_cfg(target), _model_cfg(draft), max_batch, max_ctx, gamma_cap, block_b, rho, criterion,
-               succ_bias, use_posemb)
+               succ_bias, use_posemb, mb_scope)
 
 
 def pacer_workspace_bytes(cfg: Cfg) -> int:
@@ -197,6 +201,10 @@ class Context:
         with torch.cuda.device(self.device):
             self._check(_lib.pacer_accept_rollback(self._h))
 
+    def pacer_debug_set_device_status(self, code, block=0, warp=0, detail=0):
+        with torch.cuda.device(self.device):
+            self._check(_lib.pacer_debug_set_device_status(self._h, code, block, warp, detail))
+
     def pacer_read_state(self, batch=1):
         arr = (SeqState * batch)()
         with torch.cuda.device(self.device):
@@ -234,6 +242,28 @@ class Context:
             self._check(_lib.pacer_generate(self._h, p.ctypes.data, B, p.shape[1], max_new, gamma_max, threshold, mode,
                                             seed, tok.ctypes.data, ns.ctypes.data, dl.ctypes.data, al.ctypes.data,
                                             C.byref(st)))
+        return tok, ns, dl, al, st.as_dict()
+
+    def pacer_generate_sched(self, prompt, max_new, windows, mode=PACER_GREEDY, seed=0):
+        """Speculative decoding with prescribed windows (int32 [batch][n_windows] or [n_windows]); returns like
+        pacer_generate."""
+        p = _i32(prompt)
+        if p.ndim == 1:
+            p = p[None]
+        w = _i32(windows)
+        if w.ndim == 1:
+            w = w[None]
+        B = p.shape[0]
+        assert w.shape[0] == B
+        tok = np.zeros((B, max_new), np.int32)
+        ns = np.zeros(B, np.int32)
+        dl = np.zeros((B, max_new), np.int32)
+        al = np.zeros((B, max_new), np.int32)
+        st = Stats()
+        with torch.cuda.device(self.device):
+            self._check(_lib.pacer_generate_sched(self._h, p.ctypes.data, B, p.shape[1], max_new, w.ctypes.data,
+                                                  w.shape[1], mode, seed, tok.ctypes.data, ns.ctypes.data,
+                                                  dl.ctypes.data, al.ctypes.data, C.byref(st)))
         return tok, ns, dl, al, st.as_dict()
 
     def pacer_generate_ar(self, prompt, max_new, mode=PACER_GREEDY, seed=0):

@@ -30,6 +30,10 @@ struct SeqState {
     int32_t mode;         // PACER_GREEDY / PACER_SAMPLE
     int32_t active;       // 1 for sequences 0..batch-1 of the current run
     uint64_t seed;
+    int32_t mb_start;     // M_B cache position of the first draft row of this step (local-draft attention context)
+    int32_t sched;        // 1: the window of every step is prescribed (no pre-verification), see DevPtrs::sched_win
+    int32_t n_sched;      // prescribed windows per sequence (steps beyond reuse the last one)
+    int32_t pad_;
 };
 
 enum RowKind {
@@ -56,6 +60,8 @@ struct DevPtrs {
     int32_t *hpend_e;    // [max_batch][b+1] draft index (1-based) or 0 for history rows
     int32_t *draft_len;  // [max_batch][max_steps]
     int32_t *accept_len; // [max_batch][max_steps]
+    int32_t *sched_win;  // [max_batch][max_steps] prescribed windows (runs with SeqState::sched)
+    int32_t sched_rows;  // rows per sequence of a draft forward in such a run (the draft may have rows to catch up on)
     float *verify_logits;// [max_batch][gamma_cap+1][V]
     float *draft_logits; // [max_batch][gamma_cap][V]
     // per-forward scratch
@@ -65,15 +71,13 @@ struct DevPtrs {
     int32_t *row_arg;    // [rtot] argmax of the LM-head row
     float *row_margin;   // [rtot] top1 - top2
     float *xres;         // [rtot][d] fp32 residual stream
-    bf16 *xn;            // unused by the forward kernel (its x * gain buffer is FwdBufs::xg)
     bf16 *att;           // attention output, split bf16 in tensor-core operand order (K = H*hd)
     bf16 *act;           // SwiGLU output, split bf16 in tensor-core operand order (K = F)
-    float *q;            // [rtot][H*hd] fp32 rotated queries
     float *hidden;       // [rtot][d] fp32 final-norm output
     float *part;         // split-K partial sums [S][nt*8][N]
     int32_t max_batch, max_ctx, gamma_cap, block_b, max_steps;
     float rho, succ_bias;
-    int32_t criterion, use_posemb;
+    int32_t criterion, use_posemb, mb_scope;
 };
 
 struct ModelDev {

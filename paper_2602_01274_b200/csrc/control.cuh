@@ -46,26 +46,19 @@ __device__ __forceinline__ Top2 block_top2(Top2 t, Top2 *sm) {
     return sm[0];
 }
 
-// Greedy acceptance (Eq. 5 with one-hot distributions), commit, rollback, logs.
-__global__ void k_accept_greedy(DevPtrs d, Geom g) {
-    const int s = blockIdx.x * blockDim.x + threadIdx.x;
-    if (s >= g.batch) return;
-    SeqState &st = d.st[s];
-    if (!st.active || st.finished || d.n_rows[s] == 0) return;
+// Commit of one step (Algorithm 1, after Eq. 5): [y_1..y_n, next] joins the accepted tokens, the three caches are
+// cut back to the accepted rows, the per-step state restarts, (gamma, n) is logged.  One thread per sequence.
+__device__ __forceinline__ void commit_step(const DevPtrs &d, SeqState &st, int s, int n, int next) {
     const int gamma = st.gamma, P = st.P;
     const int32_t *y = d.y + (size_t)s * d.gamma_cap;
-    const int32_t *arg = d.row_arg + s * g.rps;
-    int n = 0;
-    while (n < gamma && y[n] == arg[n]) ++n;
-    const int next = arg[n];
     int32_t *x = d.x + (size_t)s * d.max_ctx;
     for (int i = 0; i < n; ++i) x[P + i] = y[i];
     x[P + n] = next;
     st.P = P + n + 1;
     st.len_T = P + n;                                     // verify wrote rows P-1 .. P-1+gamma
     const int keep = P - 1 + (n + 1 < gamma ? n + 1 : gamma);   // the draft never processed y_gamma
-    st.len_D = keep;
-    st.len_B = keep;
+    if (keep < st.len_D) st.len_D = keep;                 // (a step without drafts leaves the draft cache as it is)
+    st.len_B = st.len_D;
     st.last_n = n; st.last_next = next;
     if (st.n_steps < d.max_steps) {
         d.draft_len[(size_t)s * d.max_steps + st.n_steps] = gamma;
@@ -74,5 +67,32 @@ __global__ void k_accept_greedy(DevPtrs d, Geom g) {
     st.n_steps += 1;
     st.n_target_fwd += 1;
     st.gamma = 0; st.k_round = 0; st.t_k = st.t0; st.drafting = 1; st.n_pend = 0;
+    if (st.sched) {                                       // the next step's prescribed window
+        int w = d.sched_win[(size_t)s * d.max_steps + (st.n_steps < st.n_sched ? st.n_steps : st.n_sched - 1)];
+        if (w > d.gamma_cap) w = d.gamma_cap;
+        if (w == 0 && st.P - st.len_D >= d.sched_rows) w = 1;   // the draft's backlog must fit one forward
+        st.gamma_max = w;
+        st.drafting = w > 0;
+    }
     if (st.P - st.n_prompt >= st.max_new) { st.finished = 1; st.drafting = 0; }
+}
+
+// Greedy acceptance (Eq. 5 with one-hot distributions) of sequence s: the longest prefix of the drafts that equals
+// the target's arg-max tokens, then the commit.  One thread.
+__device__ __forceinline__ void accept_greedy_seq(const DevPtrs &d, const Geom &g, int s) {
+    SeqState &st = d.st[s];
+    if (!st.active || st.finished || d.n_rows[s] == 0) return;
+    const int gamma = st.gamma;
+    const int32_t *y = d.y + (size_t)s * d.gamma_cap;
+    const int32_t *arg = d.row_arg + s * g.rps;
+    int n = 0;
+    while (n < gamma && y[n] == arg[n]) ++n;
+    commit_step(d, st, s, n, arg[n]);
+}
+
+// The same as a kernel of its own, for the stage-by-stage interface (the whole-loop entry points take the
+// decision in the tail of the verify forward).
+__global__ void k_accept_greedy(DevPtrs d, Geom g) {
+    const int s = blockIdx.x * blockDim.x + threadIdx.x;
+    if (s < g.batch) accept_greedy_seq(d, g, s);
 }

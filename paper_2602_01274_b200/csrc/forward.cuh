@@ -198,6 +198,8 @@ struct Ctx {
     uint32_t tmem;                 // tensor-memory address of the accumulator
     int32_t *row_pos, *row_tok;    // [MAX_ROWS]
     int32_t *n_rows;               // [MAX_ROWS] per sequence
+    int32_t *key_start;            // [MAX_ROWS] per sequence: first cache position the rows attend to (0 unless the
+                                   // pre-verification model runs with a restricted attention context)
     float *inv_rms;                // [MAX_ROWS]
     volatile int32_t *ready_op;    // [0] projections whose inputs are complete; [1] projections whose inv_rms is ready
     int32_t *flag;                 // block-wide scratch word

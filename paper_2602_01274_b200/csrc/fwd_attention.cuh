@@ -153,8 +153,8 @@ __device__ __forceinline__ void attention_prefetch(const Ctx &c, const bf16 *kca
 // Products of two remainders (2^-18 relative) are left out.
 template <int HD>
 __device__ __forceinline__ void attention_keys(Ctx &c, const bf16 *kcache, const bf16 *vcache, size_t kv_lo, int lo, int hi,
-                                               int n_new, int n_r, int mt, int kw, int KW, float (&mx)[2], float (&lsum)[2],
-                                               float (&o)[HD / 8][4]) {
+                                               int n_new, int n_r, int fresh_lo, int mt, int kw, int KW, float (&mx)[2],
+                                               float (&lsum)[2], float (&o)[HD / 8][4]) {
     using SM = AttSmem<HD>;
     constexpr int NCH = HD / 32, NOT = HD / 8, QP = SM::QP, VP = SM::VP;
     const int g = c.lane >> 2, t = c.lane & 3;
@@ -218,7 +218,9 @@ __device__ __forceinline__ void attention_keys(Ctx &c, const bf16 *kcache, const
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             const int key = key0 + 2 * t + (i & 1), row = mt * 16 + g + 8 * (i >> 1);
-            const bool ok = key < kend && (!fresh || key <= row);
+            // (with a restricted attention context the keys of this forward before fresh_lo are outside it;
+            // a row always sees itself)
+            const bool ok = key < kend && (!fresh || (key <= row && (key >= fresh_lo || key == row)));
             if (!ok) s[i] = -INFINITY;
             rmax[i >> 1] = fmaxf(rmax[i >> 1], s[i]);
         }
@@ -284,7 +286,9 @@ __device__ __forceinline__ void attention_item(Ctx &c, const Args &a, int layer,
     const int H = m.cfg.n_heads, Hkv = m.cfg.n_kv_heads, group = H / Hkv, kh = h / group;
     const int n_r = c.n_rows[seq], r_base = seq * a.g.rps, pos0 = c.row_pos[r_base];
     const size_t cbase = (((size_t)layer * d.max_batch + seq) * Hkv + kh) * (size_t)d.max_ctx * HD;
-    const int lo = (int)((long long)pos0 * split / nsplit), hi = (int)((long long)pos0 * (split + 1) / nsplit);
+    const int ks = min(c.key_start[seq], pos0), span = pos0 - ks;      // cached keys in the attention context: [ks, pos0)
+    const int lo = ks + (int)((long long)span * split / nsplit), hi = ks + (int)((long long)span * (split + 1) / nsplit);
+    const int fresh_lo = max(0, c.key_start[seq] - pos0);
     const int two = n_r > 16 ? 1 : 0;                    // two query tiles: warps 0..3 take rows 0..15, warps 4..7 rows 16..31
     const int mt = two ? (c.warp >> 2) : 0, kw = two ? (c.warp & 3) : c.warp, KW = two ? 4 : 8;
     const int g = c.lane >> 2, t = c.lane & 3;
@@ -296,7 +300,7 @@ __device__ __forceinline__ void attention_item(Ctx &c, const Args &a, int layer,
     float o[NOT][4];
 #pragma unroll
     for (int i = 0; i < NOT; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
-    attention_keys<HD>(c, m.kcache + cbase, m.vcache + cbase, m.kv_lo, lo, hi, split == nsplit - 1 ? n_r : 0, n_r, mt, kw, KW, mx, lsum, o);
+    attention_keys<HD>(c, m.kcache + cbase, m.vcache + cbase, m.kv_lo, lo, hi, split == nsplit - 1 ? n_r : 0, n_r, fresh_lo, mt, kw, KW, mx, lsum, o);
 
     bsync();                                             // every warp is done with q, the new rows and the slots
     float *red = reinterpret_cast<float *>(c.scratch);   // [8 warps][16 rows][PW]

@@ -40,16 +40,17 @@ __device__ __forceinline__ void tail_draft(Ctx &c, const Args &a, int s) {
     if (st.mode == PACER_SAMPLE)                          // y_i ~ q_i by the Gumbel-max rule at the token's position
         y_new = gumbel_argmax(d.draft_logits + ((size_t)s * d.gamma_cap + gamma) * a.m.cfg.vocab, a.m.cfg.vocab, st.seed,
                               st.P + gamma, s, TAG_DRAFT, MMA_THREADS, reinterpret_cast<BestD *>(c.scratch), true);
-    for (int jj = 0; jj < n_in; ++jj) {
+    const bool queue = !st.sched;                        // with prescribed windows nothing is pre-verified
+    for (int jj = 0; queue && jj < n_in; ++jj) {
         float *dst = d.hpend + ((size_t)s * (d.block_b + 1) + n_pend + jj) * dm;
         for (int i = threadIdx.x; i < dm; i += MMA_THREADS) dst[i] = hidden_at(a, c, s * a.g.rps + jj, i);
     }
     bsync();
     if (threadIdx.x == 0) {
-        for (int jj = 0; jj < n_in; ++jj)
+        for (int jj = 0; queue && jj < n_in; ++jj)
             d.hpend_e[s * (d.block_b + 1) + n_pend + jj] = (jj == n_in - 1) ? gamma + 1 : 0;
         d.y[(size_t)s * d.gamma_cap + gamma] = st.mode == PACER_SAMPLE ? y_new : d.row_arg[r_last];
-        st.n_pend = n_pend + n_in;
+        if (queue) st.n_pend = n_pend + n_in;
         st.gamma = gamma + 1;
         st.len_D += n_in;
         st.n_draft_fwd += 1;
@@ -89,6 +90,11 @@ __device__ __forceinline__ void tail_mb(Ctx &c, const Args &a, int s) {
         if (gamma + b > st.gamma_max) stop = 1;
         if (stop) st.drafting = 0;
         else { st.t_k = st.t_k * d.rho; st.k_round += 1; }
+        if (gamma == b) {                     // first call of the step: where its drafts begin in the cache
+            int n_hist = 0;
+            while (n_hist < n && c.row_tok[s * a.g.rps + n_hist] == 0) ++n_hist;
+            st.mb_start = st.len_B + n_hist;
+        }
         st.len_B += n;
         st.n_pend = 0;
         st.n_mb_calls += 1;
@@ -164,6 +170,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
     Top2 *top_sm = reinterpret_cast<Top2 *>(misc + 1024 + 384);              // [8]
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(misc + 1536);
     c.pass_done = reinterpret_cast<volatile int32_t *>(misc + 1540);
+    c.key_start = reinterpret_cast<int32_t *>(misc + 1664);                  // [MAX_ROWS], ends at 1792
     c.bar_target = 0;
     c.np = 0;
     c.tmem = 0;
@@ -186,10 +193,19 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
     __syncthreads();
     if (threadIdx.x < MAX_ROWS) {
         const int s = threadIdx.x;
-        int n = 0;
-        if (s < g.batch)
+        int n = 0, ks = 0;
+        if (s < g.batch) {
             for (int j = 0; j < g.rps; ++j) n += c.row_pos[s * g.rps + j] >= 0;
+            if (kind == KIND_MB && d.mb_scope != 0 && n > 0) {
+                // restricted attention context: from the first draft row of the block, or of the step
+                int n_hist = 0;
+                while (n_hist < n && c.row_tok[s * g.rps + n_hist] == 0) ++n_hist;
+                const int first = c.row_pos[s * g.rps] + n_hist;
+                ks = (d.mb_scope == 2 || d.st[s].gamma == d.block_b) ? first : d.st[s].mb_start;
+            }
+        }
         c.n_rows[s] = n;
+        c.key_start[s] = ks;
     }
     __syncthreads();
     int any = 0;
@@ -337,6 +353,10 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
         stamp();
         if (kind == KIND_VERIFY) {
             if (c.cta < g.rtot && row_dst[c.cta]) head_row_argmax(a, c.cta, top_sm);
+            if (a.aux) {                    // whole-loop runs, greedy: acceptance (Eq. 5), commit and rollback right here
+                grid_barrier(c, a.fb);
+                if (c.cta < g.batch && threadIdx.x == 0) accept_greedy_seq(d, g, c.cta);
+            }
         } else if (c.cta < g.batch && c.n_rows[c.cta] > 0) {
             head_row_argmax(a, c.cta * g.rps + c.n_rows[c.cta] - 1, top_sm);
         }
@@ -408,11 +428,14 @@ static inline Plan make_plan(const ModelDev &m, const DevPtrs &d, const FwdBufs 
 
 template <int NT, bool TWO>
 static inline cudaError_t launch_nt(const Args &a, int which, int ncta, cudaStream_t st) {
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(k_forward<NT, TWO>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    static bool attr_set[64] = {};           // the opt-in is per device
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+        e = cudaFuncSetAttribute(k_forward<NT, TWO>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
         if (e != cudaSuccess) return e;
-        attr_set = true;
+        if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
     void *params[] = {(void *)&a, (void *)&which};
     return cudaLaunchCooperativeKernel((const void *)k_forward<NT, TWO>, dim3(ncta), dim3(THREADS), params, SMEM_BYTES, st);

@@ -31,7 +31,7 @@ __device__ __forceinline__ RowDesc row_desc(int kind, const DevPtrs &d, int s, i
         case KIND_DRAFT: {
             if (!st.drafting || st.finished) break;
             // a draft step beyond the window, or before the queued hidden rows were scored, is a no-op
-            if (st.gamma >= st.gamma_max || st.gamma - st.k_round * d.block_b >= d.block_b) break;
+            if (st.gamma >= st.gamma_max || (!st.sched && st.gamma - st.k_round * d.block_b >= d.block_b)) break;
             if (st.gamma == 0) {
                 const int n_in = st.P - st.len_D;            // 1, or 2 after a fully accepted step
                 if (j < n_in) { r.active = 1; r.pos = st.len_D + j; r.tok = d.x[(size_t)s * d.max_ctx + r.pos]; }
@@ -61,6 +61,7 @@ __device__ __forceinline__ RowDesc row_desc(int kind, const DevPtrs &d, int s, i
         }
         case KIND_MB: {
             if (st.finished) break;
+            if (st.gamma - st.k_round * d.block_b < d.block_b) break;     // no whole block is waiting: a no-op
             if (j < st.n_pend) { r.active = 1; r.pos = st.len_B + j; r.tok = d.hpend_e[s * (d.block_b + 1) + j]; }
             break;
         }

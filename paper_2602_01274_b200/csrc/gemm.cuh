@@ -177,11 +177,14 @@ static inline GemmPlan gemm_plan(int N, int K, int NT) {
 
 template <int NT>
 static cudaError_t gemm_launch_nt(const GemmArgs &a, const GemmPlan &p, cudaStream_t st) {
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(k_gemm_skinny<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
+    static bool attr_set[64] = {};           // the opt-in is per device
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+        e = cudaFuncSetAttribute(k_gemm_skinny<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
         if (e != cudaSuccess) return e;
-        attr_set = true;
+        if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
     k_gemm_skinny<NT><<<p.grid, GEMM_THREADS, p.smem, st>>>(a);
     return cudaGetLastError();

@@ -4,6 +4,7 @@
 // end of generation) is taken by kernels from the device-resident SeqState.
 #include <math.h>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <string>
@@ -33,6 +34,8 @@ struct pacer_ctx {
     int prefilled;
     int64_t launches;
     cudaEvent_t ev[4];
+    int32_t *fin_host;         // pinned: finished flags of the sequences, one row per step in flight
+    cudaEvent_t fin_ev[8];
     std::vector<float2> rope_host[3];
     std::string err;
     size_t buf_bytes[16];
@@ -93,6 +96,7 @@ static bool cfg_ok(const pacer_cfg *c) {
     if (c->max_batch < 1 || c->max_batch > 64 || c->max_ctx < 4) return false;
     if (c->block_b < 1 || c->gamma_cap < c->block_b || c->gamma_cap % c->block_b) return false;
     if (c->criterion < 0 || c->criterion > 2) return false;
+    if (c->mb_scope < 0 || c->mb_scope > 2) return false;
     if (!(c->rho > 0.f)) return false;
     if ((int64_t)c->max_batch * (c->gamma_cap + 1) > fwd::MAX_ROWS) return false;   // rows of one verify forward
     return true;
@@ -114,7 +118,7 @@ struct Carver {
 };
 
 struct Layout {
-    size_t st, x, y, alpha, hpend, hpend_e, draft_len, accept_len, verify_logits, draft_logits;
+    size_t st, x, y, alpha, hpend, hpend_e, draft_len, accept_len, sched_win, verify_logits, draft_logits;
     size_t row_pos, row_tok, n_rows, row_arg, row_margin, xres, att, act, hidden, part;
     size_t att_cnt, bar, abort_flag, qkv, xg, ssq, tile_top, attp, prof;
     size_t kc[3], vc[3], rope[3];
@@ -160,6 +164,7 @@ static Layout make_layout(const pacer_cfg &c) {
     L.hpend_e = cv.take(sizeof(int32_t) * B * (c.block_b + 1));
     L.draft_len = cv.take(sizeof(int32_t) * B * L.max_steps);
     L.accept_len = cv.take(sizeof(int32_t) * B * L.max_steps);
+    L.sched_win = cv.take(sizeof(int32_t) * B * L.max_steps);
     L.row_pos = cv.take(sizeof(int32_t) * fwd::MAX_ROWS);
     L.row_tok = cv.take(sizeof(int32_t) * fwd::MAX_ROWS);
     L.n_rows = cv.take(sizeof(int32_t) * fwd::MAX_ROWS);
@@ -220,9 +225,10 @@ static Geom make_geom(int batch, int rps) {
     return g;
 }
 
-static void set_geoms(pacer_ctx *c, int batch) {
+static void set_geoms(pacer_ctx *c, int batch, int draft_rows = 2) {
     c->batch = batch;
-    c->g_draft = make_geom(batch, 2);
+    c->g_draft = make_geom(batch, draft_rows);
+    c->d.sched_rows = draft_rows;
     c->g_mb = make_geom(batch, c->cfg.block_b + 1);
     c->g_verify = make_geom(batch, c->cfg.gamma_cap + 1);
     c->g_ar = make_geom(batch, 1);
@@ -252,11 +258,12 @@ extern "C" int pacer_create(const pacer_cfg *cfg, void *dev_workspace, size_t wo
     d.st = (SeqState *)(w + L.st); d.x = (int32_t *)(w + L.x); d.y = (int32_t *)(w + L.y);
     d.alpha = (float *)(w + L.alpha); d.hpend = (float *)(w + L.hpend); d.hpend_e = (int32_t *)(w + L.hpend_e);
     d.draft_len = (int32_t *)(w + L.draft_len); d.accept_len = (int32_t *)(w + L.accept_len);
+    d.sched_win = (int32_t *)(w + L.sched_win); d.sched_rows = 2;
     d.verify_logits = (float *)(w + L.verify_logits); d.draft_logits = (float *)(w + L.draft_logits);
     d.row_pos = (int32_t *)(w + L.row_pos); d.row_tok = (int32_t *)(w + L.row_tok); d.n_rows = (int32_t *)(w + L.n_rows);
     d.row_arg = (int32_t *)(w + L.row_arg); d.row_margin = (float *)(w + L.row_margin);
-    d.xres = (float *)(w + L.xres); d.xn = nullptr; d.att = (bf16 *)(w + L.att); d.act = (bf16 *)(w + L.act);
-    d.q = nullptr; d.hidden = (float *)(w + L.hidden); d.part = (float *)(w + L.part);
+    d.xres = (float *)(w + L.xres); d.att = (bf16 *)(w + L.att); d.act = (bf16 *)(w + L.act);
+    d.hidden = (float *)(w + L.hidden); d.part = (float *)(w + L.part);
     c->fb.qkv = (float *)(w + L.qkv); c->fb.xg = (bf16 *)(w + L.xg); c->fb.ssq = (float *)(w + L.ssq);
     c->fb.part = (float *)(w + L.part);
     c->fb.tile_top = (float *)(w + L.tile_top); c->fb.attp = (float *)(w + L.attp);
@@ -268,6 +275,7 @@ extern "C" int pacer_create(const pacer_cfg *cfg, void *dev_workspace, size_t wo
     d.max_batch = cfg->max_batch; d.max_ctx = cfg->max_ctx; d.gamma_cap = cfg->gamma_cap; d.block_b = cfg->block_b;
     d.max_steps = L.max_steps; d.rho = cfg->rho; d.succ_bias = cfg->succ_bias; d.criterion = cfg->criterion;
     d.use_posemb = cfg->use_posemb;
+    d.mb_scope = cfg->mb_scope;
     const pacer_model_cfg mb = mb_cfg(*cfg);
     const pacer_model_cfg *ms[3] = {&cfg->target, &cfg->draft, &mb};
     for (int i = 0; i < 3; ++i) {
@@ -311,6 +319,9 @@ extern "C" int pacer_create(const pacer_cfg *cfg, void *dev_workspace, size_t wo
     for (int i = 0; i < 3 && e == cudaSuccess; ++i)
         e = cudaMemcpyAsync((void *)c->model[i].rope, c->rope_host[i].data(), L.rope_bytes[i], cudaMemcpyHostToDevice, c->stream);
     for (int i = 0; i < 4 && e == cudaSuccess; ++i) e = cudaEventCreate(&c->ev[i]);
+    for (int i = 0; i < 8 && e == cudaSuccess; ++i) e = cudaEventCreateWithFlags(&c->fin_ev[i], cudaEventDisableTiming);
+    c->fin_host = nullptr;
+    if (e == cudaSuccess) e = cudaHostAlloc((void **)&c->fin_host, sizeof(int32_t) * 8 * cfg->max_batch, cudaHostAllocDefault);
     if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
     if (e != cudaSuccess) {
         std::string msg = std::string("pacer_create: ") + cudaGetErrorString(e);
@@ -325,6 +336,8 @@ extern "C" int pacer_destroy(pacer_ctx *c) {
     if (!c) return PACER_EINVAL;
     cudaStreamSynchronize(c->stream);
     for (int i = 0; i < 4; ++i) cudaEventDestroy(c->ev[i]);
+    for (int i = 0; i < 8; ++i) cudaEventDestroy(c->fin_ev[i]);
+    if (c->fin_host) cudaFreeHost(c->fin_host);
     for (cudaEvent_t e : c->prof_ev) cudaEventDestroy(e);
     delete c;
     return PACER_OK;
@@ -455,9 +468,15 @@ static int need_ready(pacer_ctx *c, bool prefilled) {
 
 // ------------------------------------------------------------------ stages
 
+// windows: NULL, or host [batch][n_windows] prescribed draft windows (speculative decoding without pre-verification)
 static int start_run(pacer_ctx *c, const int32_t *prompt, int batch, int n_prompt, int max_new, int gamma_max,
-                     float threshold, int mode, uint64_t seed) {
+                     float threshold, int mode, uint64_t seed, const int32_t *windows = nullptr, int n_windows = 0) {
     const pacer_cfg &k = c->cfg;
+    if (windows) {
+        if (n_windows < 1 || n_windows > c->d.max_steps) return fail(c, PACER_EINVAL, "prescribed windows: bad count");
+        for (int i = 0; i < batch * n_windows; ++i)
+            if (windows[i] < 0 || windows[i] > k.gamma_cap) return fail(c, PACER_EINVAL, "prescribed window outside [0, gamma_cap]");
+    }
     if (!prompt || batch < 1 || batch > k.max_batch || n_prompt < 1 || max_new < 1)
         return fail(c, PACER_EINVAL, "prefill: bad batch / n_prompt / max_new");
     const int gm = gamma_max / k.block_b * k.block_b;
@@ -468,7 +487,11 @@ static int start_run(pacer_ctx *c, const int32_t *prompt, int batch, int n_promp
         for (int i = 0; i < n_prompt; ++i)
             if (prompt[(size_t)s * n_prompt + i] < 0 || prompt[(size_t)s * n_prompt + i] >= k.target.vocab)
                 return fail(c, PACER_EINVAL, "prefill: token id out of range");
-    set_geoms(c, batch);
+    // with prescribed windows a step may draft nothing, so the draft model can fall several rows behind: its
+    // forwards then take up to 16 rows per sequence (as many as fit the row limit of a forward)
+    const int draft_rows = windows ? std::min(16, fwd::MAX_ROWS / batch) : 2;
+    if (draft_rows < 2) return fail(c, PACER_EINVAL, "prescribed windows: batch too large");
+    set_geoms(c, batch, draft_rows);
     c->mode = mode;
     std::vector<SeqState> hs(k.max_batch);
     memset(hs.data(), 0, sizeof(SeqState) * hs.size());
@@ -476,7 +499,15 @@ static int start_run(pacer_ctx *c, const int32_t *prompt, int batch, int n_promp
         SeqState &st = hs[s];
         st.P = n_prompt; st.n_prompt = n_prompt; st.max_new = max_new; st.gamma_max = gm; st.t0 = threshold;
         st.t_k = threshold; st.mode = mode; st.seed = seed; st.active = 1; st.drafting = 1;
+        if (windows) {
+            st.sched = 1; st.n_sched = n_windows;
+            st.gamma_max = windows[(size_t)s * n_windows];
+            st.drafting = st.gamma_max > 0;
+        }
     }
+    if (windows)
+        CK(cudaMemcpy2DAsync(c->d.sched_win, sizeof(int32_t) * c->d.max_steps, windows, sizeof(int32_t) * n_windows,
+                             sizeof(int32_t) * n_windows, batch, cudaMemcpyHostToDevice, c->stream));
     CK(cudaMemcpyAsync(c->d.st, hs.data(), sizeof(SeqState) * hs.size(), cudaMemcpyHostToDevice, c->stream));
     // arrival counters, grid barrier and abort flag start from zero (they are contiguous in the workspace)
     CK(cudaMemsetAsync(c->fb.att_cnt, 0, (char *)c->fb.abort_flag + 4 * sizeof(int32_t) - (char *)c->fb.att_cnt, c->stream));
@@ -486,7 +517,7 @@ static int start_run(pacer_ctx *c, const int32_t *prompt, int batch, int n_promp
     return PACER_OK;
 }
 
-static int prefill_models(pacer_ctx *c, int n_prompt, bool target, bool draft_and_mb) {
+static int prefill_models(pacer_ctx *c, int n_prompt, bool target, bool draft_and_mb, bool mb = true) {
     const Geom &g = c->g_verify;
     for (int c0 = 0; c0 < n_prompt - 1; c0 += g.rps) {
         int rc;
@@ -495,7 +526,7 @@ static int prefill_models(pacer_ctx *c, int n_prompt, bool target, bool draft_an
         }
         if (draft_and_mb) {
             if ((rc = run_forward(c, PACER_DRAFT, g, KIND_PREFILL, c0, false))) return rc;
-            if ((rc = run_forward(c, PACER_PREVERIFY, g, KIND_PREFILL_B, c0, false))) return rc;
+            if (mb && (rc = run_forward(c, PACER_PREVERIFY, g, KIND_PREFILL_B, c0, false))) return rc;
         }
     }
     return PACER_OK;
@@ -538,11 +569,33 @@ extern "C" int pacer_accept_rollback(pacer_ctx *c) {
     return PACER_OK;
 }
 
+// After a synchronisation: the device status word.  A bounded wait inside a kernel that ran out leaves its code
+// there (and the block, warp and detail of the first such wait); the kernels then fall through to their end, and
+// every [sync] entry point reports PACER_EDEVICE until the next run resets the word.
+static int device_status(pacer_ctx *c) {
+    int32_t aborted[4] = {0, 0, 0, 0};
+    CK(cudaMemcpy(aborted, c->fb.abort_flag, sizeof aborted, cudaMemcpyDeviceToHost));
+    if (aborted[0])
+        return fail(c, PACER_EDEVICE, "a bounded wait inside the forward kernel ran out (wait code " + std::to_string(aborted[0]) +
+                                          ", block " + std::to_string(aborted[1]) + ", warp " + std::to_string(aborted[2]) +
+                                          ", detail " + std::to_string(aborted[3]) + ")");
+    return PACER_OK;
+}
+
+extern "C" int pacer_debug_set_device_status(pacer_ctx *c, int code, int block, int warp, int detail) {
+    if (!c) return fail(nullptr, PACER_EINVAL, "ctx is null");
+    const int32_t v[4] = {code, block, warp, detail};
+    CK(cudaMemcpyAsync(c->fb.abort_flag, v, sizeof v, cudaMemcpyHostToDevice, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    return PACER_OK;
+}
+
 extern "C" int pacer_read_state(pacer_ctx *c, pacer_seq_state *out, int batch) {
     if (!c || !out || batch < 1 || batch > c->cfg.max_batch) return fail(c, PACER_EINVAL, "pacer_read_state: bad argument");
     std::vector<SeqState> hs(batch);
     CK(cudaMemcpyAsync(hs.data(), c->d.st, sizeof(SeqState) * batch, cudaMemcpyDeviceToHost, c->stream));
     CK(cudaStreamSynchronize(c->stream));
+    const int status = device_status(c);
     for (int s = 0; s < batch; ++s) {
         const SeqState &a = hs[s];
         pacer_seq_state &o = out[s];
@@ -551,7 +604,7 @@ extern "C" int pacer_read_state(pacer_ctx *c, pacer_seq_state *out, int batch) {
         o.last_next = a.last_next; o.n_pend = a.n_pend; o.err = a.err; o.n_draft_fwd = a.n_draft_fwd;
         o.n_mb_calls = a.n_mb_calls; o.n_target_fwd = a.n_target_fwd;
     }
-    return PACER_OK;
+    return status;
 }
 
 extern "C" int pacer_read_buffer(pacer_ctx *c, int which, void *host_dst, size_t bytes) {
@@ -559,7 +612,7 @@ extern "C" int pacer_read_buffer(pacer_ctx *c, int which, void *host_dst, size_t
     if (bytes > c->buf_bytes[which]) return fail(c, PACER_EINVAL, "pacer_read_buffer: more bytes than the buffer holds");
     CK(cudaMemcpyAsync(host_dst, c->buf_ptr[which], bytes, cudaMemcpyDeviceToHost, c->stream));
     CK(cudaStreamSynchronize(c->stream));
-    return PACER_OK;
+    return device_status(c);
 }
 
 extern "C" int pacer_profile_begin(pacer_ctx *c) {
@@ -593,6 +646,17 @@ extern "C" int pacer_profile_end(pacer_ctx *c, double *gemm_ms, double *gemm_wei
 
 // ------------------------------------------------------------------ whole loops
 
+// The verify forward of a whole-loop run: greedy runs take the acceptance in the forward's tail, sampling
+// runs in the acceptance kernel that follows.
+static int enqueue_verify_accept(pacer_ctx *c) {
+    int rc = need_ready(c, true);
+    if (rc) return rc;
+    if (c->mode == PACER_GREEDY) return run_forward(c, PACER_TARGET, c->g_verify, KIND_VERIFY, 1, true);
+    if ((rc = run_forward(c, PACER_TARGET, c->g_verify, KIND_VERIFY, 0, true))) return rc;
+    return pacer_accept_rollback(c);
+}
+
+// One draft-and-verify step of Algorithm 1.  Forwards of sequences that have stopped drafting are no-ops.
 static int enqueue_step(pacer_ctx *c, int gamma_max) {
     int rc;
     const int b = c->cfg.block_b;
@@ -601,8 +665,32 @@ static int enqueue_step(pacer_ctx *c, int gamma_max) {
             if ((rc = pacer_draft_step(c))) return rc;
         if ((rc = pacer_preverify(c))) return rc;
     }
-    if ((rc = pacer_verify(c))) return rc;
-    return pacer_accept_rollback(c);
+    return enqueue_verify_accept(c);
+}
+
+// Enqueues steps until every sequence is finished.  The end of generation is decided on the device; the host only
+// learns of it, without ever waiting for the step it has just enqueued: after each step the finished flags are
+// copied to pinned memory behind an event, and the host looks at the flags of the step it enqueued RUN_AHEAD steps
+// ago.  Steps enqueued after the last real one are no-ops on the device.
+template <class Enqueue>
+static int run_steps(pacer_ctx *c, int batch, int max_steps, Enqueue enqueue) {
+    constexpr int RUN_AHEAD = 2, SLOTS = 8;
+    for (int step = 0; step < max_steps; ++step) {
+        int rc = enqueue(step);
+        if (rc) return rc;
+        const int slot = step % SLOTS;
+        CK(cudaMemcpy2DAsync(c->fin_host + (size_t)slot * c->cfg.max_batch, sizeof(int32_t), &c->d.st[0].finished, sizeof(SeqState),
+                             sizeof(int32_t), batch, cudaMemcpyDeviceToHost, c->stream));
+        CK(cudaEventRecord(c->fin_ev[slot], c->stream));
+        if (step >= RUN_AHEAD) {
+            const int seen = (step - RUN_AHEAD) % SLOTS;
+            CK(cudaEventSynchronize(c->fin_ev[seen]));
+            bool all = true;
+            for (int q = 0; q < batch; ++q) all = all && c->fin_host[(size_t)seen * c->cfg.max_batch + q];
+            if (all) break;
+        }
+    }
+    return PACER_OK;
 }
 
 static int collect(pacer_ctx *c, int batch, int max_new, int n_prompt, int32_t *out_tokens, int32_t *out_n_steps,
@@ -613,16 +701,10 @@ static int collect(pacer_ctx *c, int batch, int max_new, int n_prompt, int32_t *
     CK(cudaMemcpy2DAsync(out_tokens, sizeof(int32_t) * max_new, c->d.x + n_prompt, sizeof(int32_t) * k.max_ctx,
                          sizeof(int32_t) * max_new, batch, cudaMemcpyDeviceToHost, c->stream));
     CK(cudaStreamSynchronize(c->stream));
-    int32_t aborted[4] = {0, 0, 0, 0};
-    CK(cudaMemcpy(aborted, c->fb.abort_flag, sizeof aborted, cudaMemcpyDeviceToHost));
-    if (aborted[0])
-        return fail(c, PACER_EDEVICE, "a bounded wait inside the forward kernel ran out (wait code " + std::to_string(aborted[0]) +
-                                          ", block " + std::to_string(aborted[1]) + ", warp " + std::to_string(aborted[2]) +
-                                          ", detail " + std::to_string(aborted[3]) + ")");
+    if (int rc = device_status(c)) return rc;
     int64_t nd = 0, nm = 0, nt = 0, ns = 0, ng = 0;
     for (int s = 0; s < batch; ++s) {
         const SeqState &a = hs[s];
-        if (a.err) return fail(c, PACER_EDEVICE, "device status word set");
         nd += a.n_draft_fwd; nm += a.n_mb_calls; nt += a.n_target_fwd; ns += a.n_steps; ng += a.P - a.n_prompt;
         if (out_n_steps) out_n_steps[s] = a.n_steps;
         if (out_draft_len && out_accept_len) {
@@ -656,15 +738,33 @@ extern "C" int pacer_generate(pacer_ctx *c, const int32_t *prompt, int batch, in
     CK(cudaEventRecord(c->ev[1], c->stream));
     const int64_t launches0 = c->launches;
     const int gm = gamma_max / c->cfg.block_b * c->cfg.block_b;
-    std::vector<SeqState> hs(batch);
-    for (int step = 0; step < max_new; ++step) {
-        if ((rc = enqueue_step(c, gm))) return rc;
-        CK(cudaMemcpyAsync(hs.data(), c->d.st, sizeof(SeqState) * batch, cudaMemcpyDeviceToHost, c->stream));
-        CK(cudaStreamSynchronize(c->stream));
-        bool all = true;
-        for (int s = 0; s < batch; ++s) all = all && hs[s].finished;
-        if (all) break;
-    }
+    if ((rc = run_steps(c, batch, max_new, [&](int) { return enqueue_step(c, gm); }))) return rc;
+    CK(cudaEventRecord(c->ev[2], c->stream));
+    return collect(c, batch, max_new, n_prompt, out_tokens, out_n_steps, out_draft_len, out_accept_len, stats, launches0);
+}
+
+extern "C" int pacer_generate_sched(pacer_ctx *c, const int32_t *prompt, int batch, int n_prompt, int max_new,
+                                    const int32_t *windows, int n_windows, int mode, uint64_t seed, int32_t *out_tokens,
+                                    int32_t *out_n_steps, int32_t *out_draft_len, int32_t *out_accept_len, pacer_stats *stats) {
+    int rc = need_ready(c, false);
+    if (rc) return rc;
+    if (!out_tokens || !windows) return fail(c, PACER_EINVAL, "pacer_generate_sched: out_tokens or windows is null");
+    if ((rc = start_run(c, prompt, batch, n_prompt, max_new, c->cfg.gamma_cap, -1.f, mode, seed, windows, n_windows))) return rc;
+    CK(cudaEventRecord(c->ev[0], c->stream));
+    if ((rc = prefill_models(c, n_prompt, true, true, false))) return rc;
+    c->prefilled = 1;
+    CK(cudaEventRecord(c->ev[1], c->stream));
+    const int64_t launches0 = c->launches;
+    rc = run_steps(c, batch, max_new, [&](int step) {
+        int w = 1;                        // (a backlog of the draft model can turn a window of 0 into 1 on the device)
+        for (int q = 0; q < batch; ++q) w = std::max(w, (int)windows[(size_t)q * n_windows + std::min(step, n_windows - 1)]);
+        for (int i = 0; i < w; ++i) {
+            int r = pacer_draft_step(c);
+            if (r) return r;
+        }
+        return enqueue_verify_accept(c);
+    });
+    if (rc) return rc;
     CK(cudaEventRecord(c->ev[2], c->stream));
     return collect(c, batch, max_new, n_prompt, out_tokens, out_n_steps, out_draft_len, out_accept_len, stats, launches0);
 }

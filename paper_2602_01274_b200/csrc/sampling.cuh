@@ -9,6 +9,7 @@
 // Gumbel noise -log(-log u) is evaluated in fp64 (u can be within 2^-25 of 1).
 #pragma once
 #include "common.cuh"
+#include "control.cuh"
 
 enum { TAG_DRAFT = 1, TAG_ACCEPT = 2, TAG_NEXT = 3 };
 
@@ -161,22 +162,5 @@ __global__ void __launch_bounds__(ACCEPT_THREADS) k_accept_sample(DevPtrs d, Geo
             next = block_best(a, smb, false).i;
         }
     }
-    if (threadIdx.x != 0) return;
-    int32_t *x = d.x + (size_t)s * d.max_ctx;
-    for (int i = 0; i < n; ++i) x[P + i] = y[i];
-    x[P + n] = next;
-    st.P = P + n + 1;
-    st.len_T = P + n;                                     // verify wrote rows P-1 .. P-1+gamma
-    const int keep = P - 1 + (n + 1 < gamma ? n + 1 : gamma);   // the draft never processed y_gamma
-    st.len_D = keep;
-    st.len_B = keep;
-    st.last_n = n; st.last_next = next;
-    if (st.n_steps < d.max_steps) {
-        d.draft_len[(size_t)s * d.max_steps + st.n_steps] = gamma;
-        d.accept_len[(size_t)s * d.max_steps + st.n_steps] = n;
-    }
-    st.n_steps += 1;
-    st.n_target_fwd += 1;
-    st.gamma = 0; st.k_round = 0; st.t_k = st.t0; st.drafting = 1; st.n_pend = 0;
-    if (st.P - st.n_prompt >= st.max_new) { st.finished = 1; st.drafting = 0; }
+    if (threadIdx.x == 0) commit_step(d, st, s, n, next);
 }

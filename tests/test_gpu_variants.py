@@ -1,6 +1,7 @@
 """GPU parity of the method's switches (the ablations of Section 4.3 and Appendix B are parameters of the same
 kernels): halting criterion mean / any token / last token, the draft position embedding switched off, other block
-sizes b and growth factors rho.  Whole runs of Algorithm 1 on the tiny pair, compared with the oracle token for
+sizes b and growth factors rho, and the attention context of the pre-verification layer (full / local draft / local
+block).  Whole runs of Algorithm 1 on the tiny pair, compared with the oracle token for
 token and step for step; the comparison is asserted where the oracle's deciding margins exceed the tolerances."""
 import numpy as np
 import pytest
@@ -14,8 +15,9 @@ pytestmark = pytest.mark.gpu
 LOGIT_TOL = 2e-2
 ALPHA_TOL = 2e-3
 
-# (criterion, use_posemb, block b, rho)
-VARIANTS = [(1, 1, 4, 1.05), (2, 1, 4, 1.05), (0, 0, 4, 1.05), (0, 1, 2, 1.05), (0, 1, 1, 1.05), (0, 1, 4, 1.2), (1, 0, 2, 1.0)]
+# (criterion, use_posemb, block b, rho, attention context of M_B: 0 full, 1 local draft, 2 local block)
+VARIANTS = [(1, 1, 4, 1.05, 0), (2, 1, 4, 1.05, 0), (0, 0, 4, 1.05, 0), (0, 1, 2, 1.05, 0), (0, 1, 1, 1.05, 0),
+            (0, 1, 4, 1.2, 0), (1, 0, 2, 1.0, 0), (0, 1, 4, 1.05, 1), (0, 1, 4, 1.05, 2), (0, 1, 2, 1.05, 1), (0, 1, 2, 1.0, 2)]
 
 
 @pytest.fixture(scope="module")
@@ -28,19 +30,19 @@ def pair():
     return dict(cfg=cfg, pair_gpu=pair_gpu, T=T, D=D, B=B, prompt=prompt)
 
 
-@pytest.mark.parametrize("criterion,use_posemb,bb,rho", VARIANTS)
-def test_variant_matches_oracle(pair, criterion, use_posemb, bb, rho):
+@pytest.mark.parametrize("criterion,use_posemb,bb,rho,scope", VARIANTS)
+def test_variant_matches_oracle(pair, criterion, use_posemb, bb, rho, scope):
     from paper_2602_01274_b200 import binding as b
     cfg = pair["cfg"]
     gamma_cap = cfg.gamma_max // bb * bb
     max_ctx = cfg.n_prompt + cfg.max_new + gamma_cap + 2
-    ctx = b.Context(b.make_cfg(cfg.target, cfg.draft, 1, max_ctx, gamma_cap, bb, rho, criterion, cfg.succ_bias, use_posemb))
+    ctx = b.Context(b.make_cfg(cfg.target, cfg.draft, 1, max_ctx, gamma_cap, bb, rho, criterion, cfg.succ_bias, use_posemb, scope))
     try:
         b.load_pair(ctx, pair["pair_gpu"])
         compared = 0
         for t0 in (0.49, 0.505, 0.47, 0.52):
             o = orc.Pacer(pair["T"], pair["D"], pair["B"], max_ctx, b=bb, gamma_cap=gamma_cap, t0=t0, rho=rho,
-                          criterion=criterion, use_posemb=use_posemb)
+                          criterion=criterion, use_posemb=use_posemb, scope=scope)
             out_o, dl_o, al_o, st_o = o.generate(pair["prompt"], cfg.max_new)
             if not (st_o["min_margin_target"] > 2 * LOGIT_TOL and st_o["min_margin_draft"] > 2 * LOGIT_TOL
                     and st_o["min_margin_stop"] > ALPHA_TOL):

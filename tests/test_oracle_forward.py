@@ -208,3 +208,47 @@ def test_linear_helper_is_a_matmul():
     w = synth.normal_bf16(1, 5, (37, 24), std=1.0)
     x = np.random.default_rng(0).normal(size=(3, 24))
     np.testing.assert_allclose(orc.linear(w, x), x @ w.double().numpy().T, atol=1e-12)
+
+
+def test_restricted_context_equals_the_suffix_run_alone_at_position_zero():
+    """The "attention context" variants of the pre-verification layer restrict a row to the cache positions from
+    key_start on.  Rotary scores depend on position differences only, so rows that start at key_start and see
+    nothing before it must come out exactly as the same rows run alone, at positions 0.., on an empty cache
+    (the plain forward, pinned above).  A dropped lower bound, an off-by-one in it, or a bound applied to the
+    values but not the scores all break the equality."""
+    shape = synth.ModelShape(1, 32, 4, 2, 48, 40)
+    w = _random_model(shape, "preverify", seed=11)
+    m = orc.OracleModel(shape, w)
+    rng = np.random.default_rng(3)
+    hist, blk = rng.standard_normal((5, 32)), rng.standard_normal((4, 32))
+    full = orc.Cache(m, 16)
+    orc.forward(m, full, x_in=hist, want_logits=False)
+    got, _ = orc.forward(m, full, x_in=blk, want_logits=False, key_start=5)
+    alone, _ = orc.forward(m, orc.Cache(m, 16), x_in=blk, want_logits=False)
+    np.testing.assert_allclose(got, alone, atol=1e-9)
+    # with the bound one position earlier the last history row is visible and the result must differ
+    full.truncate(5)
+    other, _ = orc.forward(m, full, x_in=blk, want_logits=False, key_start=4)
+    assert np.abs(other - alone).max() > 1e-4
+    # key_start = 0 is the ordinary forward
+    full.truncate(5)
+    a, _ = orc.forward(m, full, x_in=blk, want_logits=False, key_start=0)
+    full.truncate(5)
+    b, _ = orc.forward(m, full, x_in=blk, want_logits=False)
+    np.testing.assert_array_equal(a, b)
+
+
+def test_rows_before_the_restricted_context_see_themselves_only():
+    """A history row that lies before key_start attends to itself alone: its output is the single-row forward."""
+    shape = synth.ModelShape(1, 32, 4, 4, 48, 40)
+    w = _random_model(shape, "preverify", seed=12)
+    m = orc.OracleModel(shape, w)
+    rng = np.random.default_rng(4)
+    rows = rng.standard_normal((3, 32))
+    c = orc.Cache(m, 16)
+    orc.forward(m, c, x_in=rng.standard_normal((2, 32)), want_logits=False)
+    got, _ = orc.forward(m, c, x_in=rows, want_logits=False, key_start=3)     # rows at 2, 3, 4; context from 3
+    single, _ = orc.forward(m, orc.Cache(m, 16), x_in=rows[:1], want_logits=False)
+    np.testing.assert_allclose(got[0], single[0], atol=1e-9)
+    pair, _ = orc.forward(m, orc.Cache(m, 16), x_in=rows[1:], want_logits=False)
+    np.testing.assert_allclose(got[1:], pair, atol=1e-9)

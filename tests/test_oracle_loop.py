@@ -369,3 +369,82 @@ def test_preverify_inputs_are_hidden_plus_position_embedding_of_the_draft_index(
         p.verify()
         assert p.accept() == 4
         mirror.truncate(p.cache_len(2))
+
+
+@pytest.mark.parametrize("scope", [1, 2])
+def test_restricted_attention_context_of_the_preverification_layer(scope):
+    """"Attention context" ablation (Section 5): local block = the drafts of the current block only, local draft =
+    the drafts of the current step.  alpha_hat is rebuilt from the separately pinned plain forward run on exactly
+    those rows, alone, at positions 0.. (rotary scores depend on position differences only); the second step
+    follows a fully accepted one, so its first call carries a catch-up history row that must stay outside."""
+    chain = list(range(10, 40))
+    cfg, (T, D, B) = _scripted_pair(chain, draft_agree_upto=[])
+    p = orc.Pacer(T, D, B, 64, b=2, gamma_cap=4, t0=-1.0, rho=1.0, scope=scope)
+    prompt = np.array([3, 7, 10], np.int32)
+    p.prefill(prompt)
+    posemb = torch.from_numpy(B.keep["posemb"].copy()).view(torch.bfloat16).double().numpy()
+    head_b = torch.from_numpy(B.keep["head_b"].copy()).view(torch.bfloat16).double().numpy()
+    full = orc.Pacer(T, D, B, 64, b=2, gamma_cap=4, t0=-1.0, rho=1.0, scope=0)
+    full.prefill(prompt)
+    differs = False
+    for step in range(2):
+        drafted, step_rows = 0, []
+        while p.drafting:
+            p.draft_block(); full.draft_block()
+            h = p.hpend()
+            n_hist = h.shape[0] - 2
+            assert n_hist == (1 if (step == 1 and drafted == 0) else 0)
+            rows = h[n_hist:].copy()
+            for j in range(2):
+                rows[j] += posemb[drafted + j]
+            step_rows.append(rows)
+            ctx_rows = rows if scope == 2 else np.concatenate(step_rows)
+            hid, _ = orc.forward(B, orc.Cache(B, 16), x_in=ctx_rows, want_logits=False)
+            z = hid[-2:] @ head_b.T
+            expect = np.exp(z[:, 1]) / np.exp(z).sum(1)
+            p.preverify(); full.preverify()
+            np.testing.assert_allclose(p.alpha()[drafted:drafted + 2], expect, atol=1e-9)
+            differs |= bool(np.abs(p.alpha()[drafted:drafted + 2] - full.alpha()[drafted:drafted + 2]).max() > 1e-6)
+            drafted += 2
+        p.verify(); full.verify()
+        assert p.accept() == 4 and full.accept() == 4
+        assert p.cache_len(2) == full.cache_len(2)
+    assert differs, "a restricted context must change alpha_hat"
+
+
+def test_prescribed_windows_reduce_to_the_fixed_window_and_stay_lossless(tiny):
+    """Speculative decoding with a window per step: a constant list is the separately written fixed-window loop,
+    any list gives the target's greedy output (Section 2.2), and #draft forwards = the sum of the windows."""
+    cfg = tiny["cfg"]
+    a = orc.generate_sd(tiny["T"], tiny["D"], tiny["prompt"], cfg.max_new, 4)
+    b = orc.generate_sched(tiny["T"], tiny["D"], tiny["prompt"], cfg.max_new, [4])
+    for u, v in zip(a[:3], b[:3]):
+        np.testing.assert_array_equal(u, v)
+    assert a[3]["n_draft_fwd"] == b[3]["n_draft_fwd"]
+    windows = [0, 3, 0, 0, 7, 1, 0, 2, 5, 0, 0, 0, 4]
+    out, dl, al, st = orc.generate_sched(tiny["T"], tiny["D"], tiny["prompt"], cfg.max_new, windows)
+    np.testing.assert_array_equal(out, tiny["ar"])
+    want = [windows[min(i, len(windows) - 1)] for i in range(len(dl))]
+    np.testing.assert_array_equal(dl, want)
+    assert (al <= dl).all() and st["n_draft_fwd"] == int(dl.sum()) and st["n_target_fwd"] == len(dl)
+    assert int((al + 1).sum()) >= cfg.max_new > int((al[:-1] + 1).sum())
+    # accept lengths are the longest common prefix of the drafts with the target's own continuation (brute force
+    # through the fixed-window run started from the same position is covered above; here: a window of 0 is one
+    # plain target step)
+    assert (al[dl == 0] == 0).all()
+
+
+def test_optimal_windows_replay_wastes_no_draft(tiny):
+    """Section 3.1: take the accepted lengths L_A* of a large-window run as the windows of a second run (the
+    optimal draft length gamma*).  The replay meets the same step boundaries, every draft is accepted
+    (n_s = gamma_s = L_A*_s), the output is unchanged, and it needs no more target forwards and fewer draft
+    forwards than the large-window run."""
+    cfg = tiny["cfg"]
+    big = orc.generate_sd(tiny["T"], tiny["D"], tiny["prompt"], cfg.max_new, 12)
+    out, dl, al, st = orc.generate_sched(tiny["T"], tiny["D"], tiny["prompt"], cfg.max_new, big[2])
+    np.testing.assert_array_equal(out, big[0])
+    np.testing.assert_array_equal(dl, big[2])
+    np.testing.assert_array_equal(al, big[2])
+    assert st["n_target_fwd"] == big[3]["n_target_fwd"]
+    assert st["n_draft_fwd"] == int(big[2].sum()) < big[3]["n_draft_fwd"]
+    assert (big[2] < 12).any() and (big[2] > 0).any()
