@@ -99,19 +99,20 @@ def verify_bytes(cfg: synth.PairConfig, ctx_len: int, rows: int) -> float:
     return t.streamed_weight_bytes() + t.kv_bytes_per_token() * (ctx_len + rows)
 
 
-def oracle_sample(cfg: synth.PairConfig, pair_cpu, prompt, n_prompt_s, max_new_s, t0):
-    """Times the CPU oracle, as it stands, on a bounded sample of the workload:
-    the first n_prompt_s prompt tokens and max_new_s new tokens of Algorithm 1."""
+def oracle_sample(cfg: synth.PairConfig, pair_cpu, prompt, n_prompt_s, n_steps_s, t0):
+    """Times the CPU oracle, as it stands, on a bounded sample of the workload: the first n_prompt_s prompt tokens
+    (prefill, untimed like the GPU arm's), then n_steps_s draft-and-verify steps of Algorithm 1 (timed).
+    Returns (tokens/s, tokens made, seconds)."""
     from oracle import pacer_oracle as orc
     T = orc.OracleModel(cfg.target, pair_cpu["target"], pair_cpu["succ_T"], cfg.succ_bias)
     D = orc.OracleModel(cfg.draft, pair_cpu["draft"], pair_cpu["succ_D"], cfg.succ_bias)
     B = orc.OracleModel(synth.preverify_shape(cfg.draft), pair_cpu["preverify"])
-    o = orc.Pacer(T, D, B, n_prompt_s + max_new_s + cfg.gamma_cap + 2, b=cfg.block_b, gamma_cap=cfg.gamma_cap, t0=t0,
-                  rho=cfg.rho)
+    o = orc.Pacer(T, D, B, n_prompt_s + n_steps_s * (cfg.gamma_cap + 1) + cfg.gamma_cap + 2, b=cfg.block_b,
+                  gamma_cap=cfg.gamma_cap, t0=t0, rho=cfg.rho)
     o.prefill(prompt[:n_prompt_s])
     t = time.perf_counter()
     made = 0
-    while made < max_new_s:
+    for _ in range(n_steps_s):
         while o.drafting:
             o.draft_block(); o.preverify()
         o.verify()
@@ -120,10 +121,27 @@ def oracle_sample(cfg: synth.PairConfig, pair_cpu, prompt, n_prompt_s, max_new_s
     return made / dt, made, dt
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum of a k_forward verify launch divided by its algorithmic bytes, from
-# the ncu capture summarised under profiles/ (traffic grows with the layer count like the algorithmic bytes do).
-# Taken with the kernel as it is now; None would be right after any later change to the kernel.
-NCU_TRAFFIC_RATIO = 1.008
+def kernel_source_digest() -> str:
+    """sha1 over the CUDA sources: ties the DRAM counters kept under profiles/ to the kernel they were taken on."""
+    import hashlib
+    h = hashlib.sha1()
+    d = os.path.join(ROOT, "paper_2602_01274_b200", "csrc")
+    for f in sorted(os.listdir(d)):
+        if f.endswith((".cu", ".cuh")):
+            h.update(open(os.path.join(d, f), "rb").read())
+    return h.hexdigest()[:16]
+
+
+def measured_traffic_ratio():
+    """(dram bytes of a verify launch / its algorithmic bytes, note) from the ncu counters kept with the profile
+    summaries, or (None, why) when there are none for the kernel as it is now."""
+    p = os.path.join(ROOT, "profiles", "k_forward_dram_counters.txt")
+    if not os.path.exists(p):
+        return None, "no ncu counters on record"
+    kv = dict(line.split(None, 1) for line in open(p) if line.strip() and not line.startswith("#"))
+    if kv.get("kernel_source_digest", "").strip() != kernel_source_digest():
+        return None, "the kernel has changed since the ncu counters were taken"
+    return float(kv["dram_bytes_over_algorithmic_bytes"]), kv.get("capture", "").strip()
 
 
 def verify_forward_numbers(ctx, cfg, prompt, n_ver, n_warm):
@@ -155,11 +173,13 @@ def verify_forward_numbers(ctx, cfg, prompt, n_ver, n_warm):
     vbytes = verify_bytes(cfg, ctx_len, cfg.gamma_cap + 1)
     launch_ms = fwd_ms / max(1, fwd_n)
     gbs = vbytes / (launch_ms * 1e-3) / 1e9
+    ratio, ratio_note = measured_traffic_ratio()
     roofline = {"bound": "hbm", "kernel": "k_forward (one launch = one verify forward)", "achieved": gbs, "peak": peak,
-                "unit": "GB/s", "frac": gbs / peak, "peak_kind": f"of {peak_kind}", "traffic": vbytes * NCU_TRAFFIC_RATIO,
-                "traffic_note": "dram read + write bytes of one launch from the ncu capture of the 4-layer cut "
-                                "(profiles/k_forward_7b_l4_verify17.md: 1.008 x its algorithmic bytes), scaled to this "
-                                "launch by its algorithmic bytes",
+                "unit": "GB/s", "frac": gbs / peak, "peak_kind": f"of {peak_kind}",
+                "traffic": None if ratio is None else vbytes * ratio,
+                "traffic_note": ratio_note if ratio is None else
+                "from profiles: dram read + write bytes of one launch in the ncu capture of a layer-cut model (%s), "
+                "%.3f x its algorithmic bytes, scaled to this launch by its algorithmic bytes" % (ratio_note, ratio),
                 "launches_timed": fwd_n, "bytes_per_launch": vbytes, "weight_bytes_per_launch": weight_bytes / max(1, fwd_n),
                 "ms_per_launch": launch_ms}
     verify = {"ms": ver_ms, "algorithmic_gb": vbytes / 1e9, "achieved_gbs": vbytes / (ver_ms * 1e-3) / 1e9,
@@ -190,10 +210,12 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=3)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--config", default="7b_68m")
+    ap.add_argument("--config", default="33b_1b3",
+                    help="synthetic pair (default: the largest single-GPU batch-1 configuration)")
     ap.add_argument("--impl", default="pacer", choices=["pacer", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--cpu-sample-new", type=int, default=4)
+    ap.add_argument("--cpu-sample-steps", type=int, default=1,
+                    help="draft-and-verify steps of Algorithm 1 the CPU oracle is timed on")
     ap.add_argument("--sample", action="store_true", help="temperature-1 rejection sampling (Philox seed 1) instead of greedy")
     ap.add_argument("--only", default="all", choices=["all", "verify"],
                     help="verify: short prefill, one full draft window, then timed verify forwards only "
@@ -226,13 +248,14 @@ def main():
         prompt = synth.make_prompts(cfg.target.vocab, 1, cfg.n_prompt, seed=0)[0].numpy()
         vals = []
         for i in range(args.warmup + args.steps):
-            v, made, dt = oracle_sample(cfg, pair, prompt, 4, args.cpu_sample_new, t0)
+            v, made, dt = oracle_sample(cfg, pair, prompt, 2, args.cpu_sample_steps, t0)
             if i >= args.warmup:
                 vals.append((v, made, dt))
         tot_tok = sum(m for _, m, _ in vals); tot_t = sum(d for _, _, d in vals)
         val = tot_tok / tot_t
         cores = int(os.environ.get("OMP_NUM_THREADS", os.cpu_count()))
-        sample = f"first 4 prompt tokens, Algorithm 1 until >= {args.cpu_sample_new} new tokens, per step"
+        sample = (f"per step: first 2 prompt tokens prefilled (untimed), then {args.cpu_sample_steps} draft-and-verify "
+                  f"step(s) of Algorithm 1 timed")
         print(json.dumps({"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
                           "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * tot_t / max(1, len(vals)),
                           "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
@@ -300,11 +323,29 @@ def main():
         top = np.argsort(lg)[-2:][::-1]
         mismatch = {"new_token_index": i, "ar_top2_logits": [float(lg[top[0]]), float(lg[top[1]])],
                     "ar_top2_margin": float(lg[top[0]] - lg[top[1]]), "tolerance": 2e-2}
-    fixed = {}
+    fixed, fixed_fwd, logs_cap = {}, {}, None
     for g in range(cfg.block_b, cfg.gamma_cap + 1, cfg.block_b):
-        _, _, _, _, s2 = ctx.pacer_generate(prompt, cfg.max_new, g, -1.0, mode, seed)
+        _, ns2, dl2, al2, s2 = ctx.pacer_generate(prompt, cfg.max_new, g, -1.0, mode, seed)
         fixed[g] = cfg.max_new / (s2["ms_decode"] * 1e-3)
+        fixed_fwd[g] = {"draft": s2["n_draft_fwd"], "preverify": s2["n_mb_calls"], "target": s2["n_target_fwd"]}
+        if g == cfg.gamma_cap:
+            logs_cap = (dl2[0, : ns2[0]].copy(), al2[0, : ns2[0]].copy())
     best_g = max(fixed, key=fixed.get)
+
+    # Realised acceptance by draft position, from the run with the largest window (the analogue of the paper's
+    # acceptance-rate-versus-draft-position curve): of the steps that drafted position i, the share in which it was accepted.
+    dl_cap, al_cap = logs_cap
+    accept_by_pos = [float((al_cap >= i).sum() / max(1, (dl_cap >= i).sum())) for i in range(1, cfg.gamma_cap + 1)]
+    # Oracle-knowledge optimum (Section 3.1): replay with every step's window set to the accepted length L_A* of
+    # that step in the largest-window run (L_A* is capped by that window).
+    opt = None
+    if not args.sample:
+        tok_o, ns_o, dl_o, al_o, s_o = ctx.pacer_generate_sched(prompt, cfg.max_new, al_cap, mode, seed)
+        opt = {"tokens_per_s": cfg.max_new / (s_o["ms_decode"] * 1e-3),
+               "forwards": {"draft": s_o["n_draft_fwd"], "preverify": 0, "target": s_o["n_target_fwd"]},
+               "mean_window": float(al_cap.mean()), "all_drafts_accepted": bool((al_o[0, : ns_o[0]] == dl_o[0, : ns_o[0]]).all()),
+               "same_tokens": bool((tok_o[0] == toks[0]).all()),
+               "note": "windows = accepted lengths of the run with the largest fixed window (capped at gamma_cap)"}
 
     vf = verify_forward_numbers(ctx, cfg, prompt, 10, 3)
     roofline, verify = vf["roofline"], vf["verify_forward"]
@@ -325,18 +366,21 @@ def main():
            "loop": {"tokens_per_s_ar_same_kernels": ar_tps, "speedup_vs_ar": value / ar_tps,
                     "tokens_per_s_fixed_gamma": fixed, "best_fixed_gamma": best_g,
                     "speedup_vs_best_fixed": value / fixed[best_g], "tau": float(al.mean()),
-                    "mean_gamma": float(dl.mean()), "steps": int(ns), "n_draft_fwd": st["n_draft_fwd"],
-                    "n_mb_calls": st["n_mb_calls"], "n_target_fwd": st["n_target_fwd"],
+                    "mean_gamma": float(dl.mean()), "steps": int(ns),
+                    "forwards": {"pacer": {"draft": st["n_draft_fwd"], "preverify": st["n_mb_calls"], "target": st["n_target_fwd"]},
+                                 "fixed_gamma": fixed_fwd, "autoregressive": {"target": ar_st["n_target_fwd"]}},
+                    "accept_rate_by_draft_position": accept_by_pos,
+                    "optimal_window": opt,
                     "ms_prefill": st["ms_prefill"], "lossless_vs_gpu_ar": lossless,
                     "first_mismatch_vs_gpu_ar": mismatch},
            "wall_s_timed_region": wall}
     if not args.no_cpu_baseline:
         try:
-            v, made, dt = oracle_sample(cfg, pair_to_cpu(pair), prompt, 4, args.cpu_sample_new, t0)
+            v, made, dt = oracle_sample(cfg, pair_to_cpu(pair), prompt, 2, args.cpu_sample_steps, t0)
             out["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": int(os.environ.get("OMP_NUM_THREADS", os.cpu_count())),
                                    "kind": "oracle",
-                                   "sample": f"first 4 prompt tokens, Algorithm 1 until >= {args.cpu_sample_new} new "
-                                             f"tokens ({made} made in {dt:.1f} s)"}
+                                   "sample": f"first 2 prompt tokens prefilled (untimed), then {args.cpu_sample_steps} "
+                                             f"draft-and-verify step(s) of Algorithm 1 ({made} tokens in {dt:.1f} s)"}
         except Exception as ex:  # the baseline must not take the GPU numbers down with it
             out["cpu_baseline"] = {"value": None, "unit": UNIT, "cores": 0, "kind": "oracle", "sample": f"failed: {ex}"}
     print(json.dumps(out))

@@ -172,6 +172,11 @@ CONFIGS: Dict[str, PairConfig] = {
     "33b_1b3": PairConfig("33b_1b3", ModelShape(62, 7168, 56, 8, 19200, 32256),
                           ModelShape(24, 2048, 16, 16, 5504, 32256),
                           agree=0.85, n_prompt=2048, max_new=512, gamma_max=24),
+    # a second workload: grouped-query models with a large vocabulary (the shapes of a 1.5B / 32B pair of the
+    # Qwen2.5 family, the other family the paper measures): the draft's LM head is a fifth of its weights
+    "qwen_32b_1b5": PairConfig("qwen_32b_1b5", ModelShape(64, 5120, 40, 8, 27648, 151936),
+                               ModelShape(28, 1536, 12, 2, 8960, 151936),
+                               agree=0.80, n_prompt=1024, max_new=256, gamma_max=16),
     "7b_68m_long_b8": PairConfig("7b_68m_long_b8", ModelShape(32, 4096, 32, 32, 11008, 32000), _D68M,
                                  agree=0.80, n_prompt=8192, max_new=256, gamma_max=16, batch=8),
 }

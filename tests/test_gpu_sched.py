@@ -34,7 +34,7 @@ def _safe(st):
     return st["min_margin_target"] > 2 * LOGIT_TOL and st["min_margin_draft"] > 2 * LOGIT_TOL
 
 
-@pytest.mark.parametrize("windows", [[3], [0, 3, 0, 0, 7, 1, 0, 2, 5, 0, 0, 0, 4], [8, 0], [0]])
+@pytest.mark.parametrize("windows", [[3], [0, 3, 0, 0, 7, 1, 0, 2, 5, 0, 0, 0, 4], [8, 0, 0, 0, 0, 2], [0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 1]])
 def test_prescribed_windows_match_oracle(tiny2, windows):
     cfg, ctx = tiny2["cfg"], tiny2["ctx"]
     prompt = tiny2["prompts"][0]
@@ -46,6 +46,22 @@ def test_prescribed_windows_match_oracle(tiny2, windows):
     np.testing.assert_array_equal(dl[0, : ns[0]], dl_o)
     np.testing.assert_array_equal(al[0, : ns[0]], al_o)
     assert st["n_draft_fwd"] == st_o["n_draft_fwd"] and st["n_target_fwd"] == st_o["n_target_fwd"] and st["n_mb_calls"] == 0
+
+
+def test_draft_backlog_limit_turns_a_zero_window_into_one(tiny2):
+    """Windows of 0 forever: the draft model falls one row further behind per step, and a draft forward holds 16
+    rows per sequence here, so every 16th step or so must draft one token (the documented limit of the entry
+    point).  The output is the target's own greedy text all the same."""
+    cfg, ctx = tiny2["cfg"], tiny2["ctx"]
+    prompt = tiny2["prompts"][0]
+    tok, ns, dl, al, st = ctx.pacer_generate_sched(prompt, cfg.max_new, [0])
+    ar, _ = ctx.pacer_generate_ar(prompt, cfg.max_new)
+    np.testing.assert_array_equal(tok[0], ar[0])
+    w = dl[0, : ns[0]]
+    assert set(w.tolist()) == {0, 1} and int(w.sum()) >= 2
+    runs = np.diff(np.flatnonzero(np.concatenate([[1], w, [1]])))
+    assert runs.max() - 1 <= 15
+    assert (w[:15] == 0).all() and w[15] == 1
 
 
 def test_optimal_window_replay(tiny2):
