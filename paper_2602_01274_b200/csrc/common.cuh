@@ -45,9 +45,13 @@ enum RowKind {
     KIND_PREFILL_B = 5   // draft hidden rows of a prefill chunk, for M_B
 };
 
-// Row geometry of a forward: row r = seq * rps + j.
+// Row geometry of a forward: row r = seq * rps + j.  For the tensor cores the rows form G groups of nt
+// eight-row tiles (a group's values and rounding remainders together fill at most the 128 rows of one MMA).
 struct Geom {
-    int32_t batch, rps, rtot, nt;   // nt = ceil(rtot / 8) eight-row tiles
+    int32_t batch, rps, rtot;
+    int32_t nt;                     // eight-row tiles per group: 1..4, 6 or 8
+    int32_t G;                      // groups: 1, or up to 3 when nt is 6 or 8
+    int32_t rpad;                   // G * nt * 8 >= rtot
 };
 
 // Device addresses of everything a kernel may need, passed by value.

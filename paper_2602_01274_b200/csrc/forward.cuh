@@ -41,7 +41,8 @@ constexpr int X_PRODUCER = 12, X_PRODUCERS = 4;  // warps 12..14 provide the act
 constexpr int THREADS = 32 * (X_PRODUCER + X_PRODUCERS);
 constexpr int KB = 64;                          // k columns of a weight stage: one 128-byte swizzle row
 constexpr int NB = 16;                          // weight stages that can be in flight (barrier pairs)
-constexpr int RING_BYTES = 136 * 1024;          // weight ring (bytes; a stage takes 128 B per weight row of the block)
+constexpr int RING_BYTES = 132 * 1024;          // weight ring of the forwards with at most 32 rows (a stage takes 128 B per
+                                                // weight row of the block); wider forwards give part of it to the activations
 constexpr int XS_MAX = 3;                       // activation stages: as many as fit, at most 3 (one producer warp each)
 constexpr int XK = 256;                         // k columns of one activation stage (four k blocks)
 // Per k block an activation stage holds NT atoms of bf16 values and then NT atoms of bf16 rounding remainders.
@@ -49,13 +50,16 @@ __host__ __device__ constexpr int xstage_bytes(int NT) { return (XK / KB) * 2 * 
 __host__ __device__ constexpr int x_stages(int NT) { return (80 * 1024) / xstage_bytes(NT) < XS_MAX ? (80 * 1024) / xstage_bytes(NT) : XS_MAX; }
 constexpr int SCRATCH_BYTES = 88 * 1024;        // the activation ring lives in its first 72 KB at most; the epilogues' copy
                                                 // of the accumulator, the attention phase and the tails use all of it
-constexpr int MISC_BYTES = 2048;
-constexpr int SMEM_BYTES = SCRATCH_BYTES + RING_BYTES + MISC_BYTES;
+constexpr int MISC_BYTES = 6144;
+constexpr int SMEM_BYTES = SCRATCH_BYTES + RING_BYTES + MISC_BYTES;    // the same total for every forward
+static_assert(SMEM_BYTES <= 227 * 1024, "more shared memory than a block can have");
 constexpr int MMA_TILES = 16;                   // 16-row tiles one tcgen05.mma covers (N = 256)
 constexpr int MAX_TILES = 2 * MMA_TILES;        // tiles of one pass of a block: two accumulators, two MMAs per 16 k columns
                                                 // (a block that has one tile too many for N = 256 still reads the activations once)
 constexpr int ACC_COLS = 256;                   // fp32 accumulator columns of one accumulator (one per weight row)
-constexpr int MAX_ROWS = 32;                    // rows of one forward (all sequences together)
+constexpr int MAX_ROWS = 192;                   // rows of one forward (all sequences together): three groups of 64
+constexpr int MAX_SEQ = 32;                     // sequences of one forward
+constexpr int BIG_XBYTES = 144 * 1024;          // activation ring of a forward with more than 32 rows, at most
 constexpr int MAX_SPLIT = 16;                   // key-range splits of one attention head
 constexpr unsigned SPIN_LIMIT = 1u << 22;        // polls of a global word or a shared counter
 constexpr unsigned MBAR_SPIN_LIMIT = 1u << 18;   // polls of an mbarrier (each may suspend for microseconds)
@@ -82,6 +86,13 @@ struct Plan {
     GemmOp op[N_OPS];
     int32_t n_layers, has_head;
     int32_t max_tiles;       // tiles of one pass: MMA_TILES, or MAX_TILES in the kernel variant with two accumulators
+                             // (10 with three row groups: their accumulators share the 512 tensor-memory columns)
+    // shared-memory plan (bytes): [activation ring / scratch][weight ring][barriers and row tables]
+    int32_t scratch_bytes, ring_bytes;
+    int32_t xkb;             // 64-column k blocks per activation stage
+    int32_t xs;              // activation stages
+    int32_t xkb_bytes;       // bytes of one k block of activations: 2 KB per eight-row tile (values + remainders)
+    int32_t acc_stride;      // tensor-memory columns between the accumulators of two row groups
 };
 
 // Device buffers of the forward kernel beyond DevPtrs (all in the workspace).
@@ -191,14 +202,15 @@ struct Ctx {
     // shared memory
     unsigned char *scratch;        // SCRATCH_BYTES (activation ring in front)
     unsigned char *ring;           // weight ring
+    int ring_bytes;
     uint64_t *wfull, *wempty;      // [NB]
     uint64_t *xfull, *xempty;      // [XS_MAX]
     uint64_t *acc_full, *acc_empty; // the accumulator of a pass is complete / has been copied out
     volatile int32_t *pass_done;   // passes whose epilogue is over (the activation ring may be overwritten)
     uint32_t tmem;                 // tensor-memory address of the accumulator
     int32_t *row_pos, *row_tok;    // [MAX_ROWS]
-    int32_t *n_rows;               // [MAX_ROWS] per sequence
-    int32_t *key_start;            // [MAX_ROWS] per sequence: first cache position the rows attend to (0 unless the
+    int32_t *n_rows;               // [MAX_SEQ] per sequence
+    int32_t *key_start;            // [MAX_SEQ] per sequence: first cache position the rows attend to (0 unless the
                                    // pre-verification model runs with a restricted attention context)
     float *inv_rms;                // [MAX_ROWS]
     volatile int32_t *ready_op;    // [0] projections whose inputs are complete; [1] projections whose inv_rms is ready
@@ -218,14 +230,21 @@ struct Ctx {
 // 1 KB in the 128-byte swizzle layout (the 16-byte chunk c of row r sits at chunk c ^ r); atoms 0 .. nt-1 of a
 // k block hold the values of rows 8a .. 8a+7, atoms nt .. 2nt-1 the remainders.  As the A operand of an MMA with
 // M = 128 the values are accumulator lanes 0 .. 8nt-1 and the remainders lanes 8nt .. 16nt-1; the epilogue adds them.
-__device__ __forceinline__ size_t xatom_index(int r, int k, int nt, int plane) {
-    const int kk = k & 63, rr = r & 7;
-    return ((size_t)(k >> 6) * (2 * nt) + plane * nt + (r >> 3)) * 512 + rr * 64 + ((((kk >> 3) ^ rr) << 3) | (kk & 7));
+//
+// With more than 64 rows the rows form G groups of 8 * nt rows; a k block then holds the groups one after the other
+// (each its values, then its remainders), and every group is the A operand of its own MMA and accumulator.
+struct XLay {
+    int nt, G;                     // eight-row tiles per group, groups
+};
+__device__ __forceinline__ size_t xatom_index(int r, int k, XLay x, int plane) {
+    const int kk = k & 63, rr = r & 7, rg = 8 * x.nt, g = r / rg, rl = r - g * rg;
+    return ((size_t)(k >> 6) * (2 * x.nt * x.G) + g * (2 * x.nt) + plane * x.nt + (rl >> 3)) * 512 + rr * 64 +
+           ((((kk >> 3) ^ rr) << 3) | (kk & 7));
 }
-__device__ __forceinline__ void store_split(bf16 *base, int nt, int r, int k, float v) {
+__device__ __forceinline__ void store_split(bf16 *base, XLay x, int r, int k, float v) {
     const bf16 h = __float2bfloat16(v);
-    base[xatom_index(r, k, nt, 0)] = h;
-    base[xatom_index(r, k, nt, 1)] = __float2bfloat16(v - __bfloat162float(h));
+    base[xatom_index(r, k, x, 0)] = h;
+    base[xatom_index(r, k, x, 1)] = __float2bfloat16(v - __bfloat162float(h));
 }
 
 // Barrier of the eight phase warps (the producer warps never join it).

@@ -277,8 +277,8 @@ __device__ __forceinline__ void attention_keys(Ctx &c, const bf16 *kcache, const
 }
 
 template <int HD>
-__device__ __forceinline__ void attention_item(Ctx &c, const Args &a, int layer, int seq, int h, int split, int nsplit,
-                                               int nt_total) {
+__device__ __forceinline__ void attention_item(Ctx &c, const Args &a, int layer, int seq, int h, int split, int nsplit) {
+    const XLay xl{a.g.nt, a.g.G};
     using SM = AttSmem<HD>;
     constexpr int PW = SM::PW, NOT = HD / 8;
     const DevPtrs &d = a.d;
@@ -340,7 +340,7 @@ __device__ __forceinline__ void attention_item(Ctx &c, const Args &a, int layer,
         float ov = 0.f;
         for (int w = 0; w < KW; ++w) ov += red[((size_t)(w0 + w) * 16 + rr) * PW + ch] * fw[j * MMA_WARPS + w];
         if (nsplit == 1) {
-            store_split(d.att, nt_total, r_base + j, h * HD + ch, ov / rowL[j]);
+            store_split(d.att, xl, r_base + j, h * HD + ch, ov / rowL[j]);
         } else {
             float *op = outp + (size_t)j * PW;
             op[ch] = ov;
@@ -350,19 +350,30 @@ __device__ __forceinline__ void attention_item(Ctx &c, const Args &a, int layer,
     bsync();
 }
 
-// Key-range splits of a head in this forward (the same value in every block).
+// Key-range splits of a head in this forward (the same value in every block).  With fewer (sequence, head)
+// pairs than blocks: as many splits as give every block at most one item.  With more pairs than blocks (batches
+// with long contexts) the items take several rounds, and the number of splits is the one with the least
+// rounds x (keys of an item + the fixed cost of an item, about 128 keys' worth).
 __device__ __forceinline__ int attention_splits(const Ctx &c, const Args &a) {
     int lmax = 0;
     for (int s = 0; s < a.g.batch; ++s)
         if (c.n_rows[s] > 0) lmax = max(lmax, c.row_pos[s * a.g.rps]);
-    const int nsplit = c.ncta / (a.g.batch * a.m.cfg.n_heads);
-    return max(1, min(nsplit, min(MAX_SPLIT, lmax / 64)));
+    const int pairs = a.g.batch * a.m.cfg.n_heads, cap = max(1, min(MAX_SPLIT, lmax / 64));
+    if (pairs <= c.ncta) return max(1, min(c.ncta / pairs, cap));
+    int best = 1;
+    long long best_cost = -1;
+    for (int n = 1; n <= cap; ++n) {
+        const long long rounds = (pairs * n + c.ncta - 1) / c.ncta, cost = rounds * (lmax / n + 128);
+        if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = n; }
+    }
+    return best;
 }
 
 // All blocks, after the grid barrier that follows the items: the splits of every
 // (sequence, head, row) merged by one warp each, into the bf16 attention output in
 // the operand order the output projection reads.
-__device__ __forceinline__ void phase_attention_merge(Ctx &c, const Args &a, int nsplit, int nt_total) {
+__device__ __forceinline__ void phase_attention_merge(Ctx &c, const Args &a, int nsplit) {
+    const XLay xl{a.g.nt, a.g.G};
     const int H = a.m.cfg.n_heads, hd = a.m.hd, PW = hd + 2, rps = a.g.rps;
     const int tasks = a.g.batch * H * rps;
     for (int task = c.cta * MMA_WARPS + c.warp; task < tasks; task += c.ncta * MMA_WARPS) {
@@ -385,19 +396,19 @@ __device__ __forceinline__ void phase_attention_merge(Ctx &c, const Args &a, int
 #pragma unroll
         for (int e = 0; e < 4; ++e)
             if (c.lane + 32 * e < hd)
-                store_split(a.d.att, nt_total, seq * rps + j, h * hd + c.lane + 32 * e, ov[e] * inv);
+                store_split(a.d.att, xl, seq * rps + j, h * hd + c.lane + 32 * e, ov[e] * inv);
     }
 }
 
 // All blocks: the attention items of one layer.
-__device__ __forceinline__ void phase_attention(Ctx &c, const Args &a, int layer, int nsplit, int nt_total) {
+__device__ __forceinline__ void phase_attention(Ctx &c, const Args &a, int layer, int nsplit) {
     const int H = a.m.cfg.n_heads, batch = a.g.batch;
     const int items = batch * H * nsplit;
     for (int it = c.cta; it < items; it += c.ncta) {
         const int split = it % nsplit, sh = it / nsplit, h = sh % H, seq = sh / H;
         if (c.n_rows[seq] == 0) continue;
-        if (a.m.hd == 64) attention_item<64>(c, a, layer, seq, h, split, nsplit, nt_total);
-        else attention_item<128>(c, a, layer, seq, h, split, nsplit, nt_total);
+        if (a.m.hd == 64) attention_item<64>(c, a, layer, seq, h, split, nsplit);
+        else attention_item<128>(c, a, layer, seq, h, split, nsplit);
     }
 }
 

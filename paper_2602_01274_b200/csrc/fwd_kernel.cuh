@@ -140,7 +140,7 @@ __device__ __forceinline__ void tail_ar(Ctx &c, const Args &a, int s) {
 
 // ------------------------------------------------------------------ the kernel
 
-template <int NT, bool TWO>
+template <int NT, bool TWO, bool BIG>
 __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ Args a, const int which) {
     extern __shared__ __align__(1024) unsigned char smem[];
     if (smem_u32(smem) & 1023u) {           // the swizzled operand layout needs this alignment (the same in every block)
@@ -150,8 +150,9 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
     Ctx c;
     c.warp = threadIdx.x >> 5; c.lane = threadIdx.x & 31; c.cta = blockIdx.x; c.ncta = gridDim.x;
     c.scratch = smem;
-    c.ring = smem + SCRATCH_BYTES;
-    unsigned char *misc = smem + SCRATCH_BYTES + RING_BYTES;
+    c.ring = smem + a.P.scratch_bytes;
+    c.ring_bytes = a.P.ring_bytes;
+    unsigned char *misc = smem + a.P.scratch_bytes + a.P.ring_bytes;
     c.wfull = reinterpret_cast<uint64_t *>(misc);                            // NB
     c.wempty = c.wfull + NB;                                                 // NB
     c.xfull = c.wempty + NB;                                                 // XS_MAX
@@ -159,18 +160,20 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
     c.acc_full = c.xempty + XS_MAX;
     c.acc_empty = c.acc_full + 1;                                            // ends at 8 * (2*NB + 2*XS_MAX + 2) = 320
     static_assert(8 * (2 * NB + 2 * XS_MAX + 2) <= 320, "barriers overlap the row tables");
-    c.row_pos = reinterpret_cast<int32_t *>(misc + 320);
+    c.row_pos = reinterpret_cast<int32_t *>(misc + 320);                     // four tables of MAX_ROWS words
     c.row_tok = c.row_pos + MAX_ROWS;
-    c.n_rows = c.row_tok + MAX_ROWS;
-    c.inv_rms = reinterpret_cast<float *>(c.n_rows + MAX_ROWS);
-    c.ready_op = reinterpret_cast<volatile int32_t *>(c.inv_rms + MAX_ROWS); // 2 words
-    c.flag = reinterpret_cast<int32_t *>(misc + 320 + 4 * 128 + 16);         // 4 words
-    float **row_dst = reinterpret_cast<float **>(misc + 1024);               // [MAX_ROWS]
-    int32_t *bias_at = reinterpret_cast<int32_t *>(misc + 1024 + 256);       // [MAX_ROWS]
-    Top2 *top_sm = reinterpret_cast<Top2 *>(misc + 1024 + 384);              // [8]
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(misc + 1536);
-    c.pass_done = reinterpret_cast<volatile int32_t *>(misc + 1540);
-    c.key_start = reinterpret_cast<int32_t *>(misc + 1664);                  // [MAX_ROWS], ends at 1792
+    c.inv_rms = reinterpret_cast<float *>(c.row_tok + MAX_ROWS);
+    int32_t *bias_at = reinterpret_cast<int32_t *>(c.inv_rms + MAX_ROWS);
+    float **row_dst = reinterpret_cast<float **>(misc + 320 + 16 * MAX_ROWS); // [MAX_ROWS] pointers
+    unsigned char *tail_misc = misc + 320 + 24 * MAX_ROWS;
+    c.n_rows = reinterpret_cast<int32_t *>(tail_misc);                       // [MAX_SEQ]
+    c.key_start = c.n_rows + MAX_SEQ;                                        // [MAX_SEQ]
+    c.ready_op = reinterpret_cast<volatile int32_t *>(c.key_start + MAX_SEQ); // 2 words
+    c.flag = reinterpret_cast<int32_t *>(tail_misc + 8 * MAX_SEQ + 16);      // 4 words
+    Top2 *top_sm = reinterpret_cast<Top2 *>(tail_misc + 8 * MAX_SEQ + 32);   // [8]
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(tail_misc + 8 * MAX_SEQ + 160);
+    c.pass_done = reinterpret_cast<volatile int32_t *>(tail_misc + 8 * MAX_SEQ + 164);
+    static_assert(320 + 24 * MAX_ROWS + 8 * MAX_SEQ + 168 <= MISC_BYTES, "row tables do not fit");
     c.bar_target = 0;
     c.np = 0;
     c.tmem = 0;
@@ -179,6 +182,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
     const ModelDev &m = a.m;
     const Geom &g = a.g;
     const int kind = a.kind;
+    constexpr int TMEM_COLS = (TWO || BIG) ? 2 * ACC_COLS : ACC_COLS;
 
     // rows of this forward, from the sequence state
     if (threadIdx.x < MAX_ROWS) {
@@ -191,7 +195,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
         c.row_pos[r] = pos; c.row_tok[r] = tok;
     }
     __syncthreads();
-    if (threadIdx.x < MAX_ROWS) {
+    if (threadIdx.x < MAX_SEQ) {
         const int s = threadIdx.x;
         int n = 0, ks = 0;
         if (s < g.batch) {
@@ -211,7 +215,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
     int any = 0;
     for (int s = 0; s < g.batch; ++s) any |= c.n_rows[s];
     if (c.cta == 0 && threadIdx.x < MAX_ROWS) {
-        if (threadIdx.x < g.batch) d.n_rows[threadIdx.x] = c.n_rows[threadIdx.x];
+        if (threadIdx.x < g.batch && threadIdx.x < MAX_SEQ) d.n_rows[threadIdx.x] = c.n_rows[threadIdx.x];
         if (threadIdx.x < g.rtot) { d.row_pos[threadIdx.x] = c.row_pos[threadIdx.x]; d.row_tok[threadIdx.x] = c.row_tok[threadIdx.x]; }
     }
     if (!any) return;                       // every sequence idles: the same decision in every block
@@ -242,7 +246,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (c.warp == MMA_ISSUER) {             // the accumulator's tensor memory, held until the end of the kernel
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TWO ? 2 * ACC_COLS : ACC_COLS) : "memory");
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     fence_proxy_async();
@@ -257,17 +261,20 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
         return;
     }
     if (c.warp == MMA_ISSUER) {
-        if (c.lane == 0) mma_issuer<NT, TWO>(c, a.fb, a.P);
+        if (c.lane == 0) mma_issuer<NT, TWO, BIG>(c, a.fb, a.P, g.G);
         __syncwarp();
         asm volatile("bar.sync 2, 288;" ::: "memory");        // the phase warps have read their last accumulator
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(c.tmem), "r"(TWO ? 2 * ACC_COLS : ACC_COLS) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(c.tmem), "r"(TMEM_COLS) : "memory");
         return;
     }
-    if (c.warp == X_PRODUCER + X_PRODUCERS - 1) { helper_warp(c, a.fb, a.P, m.cfg.d_model, m.cfg.rms_eps); return; }
+    if (c.warp == X_PRODUCER + X_PRODUCERS - 1) {           // (in the wide forwards the phase warps compute 1/rms themselves)
+        if (!BIG) helper_warp(c, a.fb, a.P, m.cfg.d_model, m.cfg.rms_eps);
+        return;
+    }
     if (c.warp >= X_PRODUCER) {
         uint64_t keep;
         asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(keep));
-        activation_producer<NT>(c, a.fb, a.P, c.warp - X_PRODUCER, keep);
+        activation_producer<NT, BIG>(c, a.fb, a.P, c.warp - X_PRODUCER, keep);
         return;
     }
 
@@ -278,7 +285,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
             a.fb.prof[(size_t)c.cta * PROF_STAMPS + n_stamp++] = globaltimer_ns();
     };
     stamp();
-    phase_begin(c, a, NT);
+    phase_begin(c, a);
     stamp();
     grid_barrier(c, a.fb);
     stamp();
@@ -287,18 +294,18 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
     for (int l = 0; l < L; ++l) {
         {
             const int slice = op_slice(a.P.op[OP_QKV], c.cta, c.ncta);
-            gemm_op<NT, TWO>(c, a.fb, a.P, 4 * l + OP_QKV, nullptr, 0,
-                        [&](int tile, float (&acc)[NT][4]) { epi_qkv<NT>(c, a, slice, tile, acc); });
+            gemm_op<NT, TWO, BIG>(c, a.fb, a.P, 4 * l + OP_QKV, g.G, dm, m.cfg.rms_eps, nullptr, 0,
+                        [&](int tile, int rb, float (&acc)[NT][4]) { epi_qkv<NT>(c, a, slice, tile, rb, acc); });
         }
         stamp();
         grid_barrier(c, a.fb);
         stamp();
         const int nsplit = attention_splits(c, a);
-        phase_attention(c, a, l, nsplit, NT);
+        phase_attention(c, a, l, nsplit);
         stamp();
         grid_barrier(c, a.fb);
         if (nsplit > 1) {                       // the same decision in every block
-            phase_attention_merge(c, a, nsplit, NT);
+            phase_attention_merge(c, a, nsplit);
             grid_barrier(c, a.fb);
         }
         stamp();
@@ -306,22 +313,22 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
             const GemmOp &op = a.P.op[OP_O];
             const bf16 *gain_next = m.norm2 + (size_t)l * dm;
             if (op.S == 1) {
-                gemm_op<NT, TWO>(c, a.fb, a.P, 4 * l + OP_O, d.xres, dm,
-                            [&](int tile, float (&acc)[NT][4]) { epi_residual<NT>(c, a, gain_next, tile, acc); });
+                gemm_op<NT, TWO, BIG>(c, a.fb, a.P, 4 * l + OP_O, g.G, dm, m.cfg.rms_eps, d.xres, dm,
+                            [&](int tile, int rb, float (&acc)[NT][4]) { epi_residual<NT>(c, a, gain_next, tile, rb, acc); });
             } else {
                 const int slice = op_slice(op, c.cta, c.ncta);
-                gemm_op<NT, TWO>(c, a.fb, a.P, 4 * l + OP_O, nullptr, 0,
-                            [&](int tile, float (&acc)[NT][4]) { epi_partial<NT>(c, a, op, slice, tile, acc); });
+                gemm_op<NT, TWO, BIG>(c, a.fb, a.P, 4 * l + OP_O, g.G, dm, m.cfg.rms_eps, nullptr, 0,
+                            [&](int tile, int rb, float (&acc)[NT][4]) { epi_partial<NT>(c, a, op, slice, tile, rb, acc); });
             }
             stamp();
             grid_barrier(c, a.fb);
             if (op.S > 1) {
-                phase_residual<NT>(c, a, op, gain_next);
+                phase_residual(c, a, op, gain_next);
                 grid_barrier(c, a.fb);
             }
             stamp();
         }
-        gemm_op<NT, TWO>(c, a.fb, a.P, 4 * l + OP_GU, nullptr, 0, [&](int tile, float (&acc)[NT][4]) { epi_swiglu<NT>(c, a, tile, acc); });
+        gemm_op<NT, TWO, BIG>(c, a.fb, a.P, 4 * l + OP_GU, g.G, dm, m.cfg.rms_eps, nullptr, 0, [&](int tile, int rb, float (&acc)[NT][4]) { epi_swiglu<NT>(c, a, tile, rb, acc); });
         stamp();
         grid_barrier(c, a.fb);
         stamp();
@@ -329,25 +336,25 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
             const GemmOp &op = a.P.op[OP_DOWN];
             const bf16 *gain_next = l + 1 < L ? m.norm1 + (size_t)(l + 1) * dm : m.normf;
             if (op.S == 1) {
-                gemm_op<NT, TWO>(c, a.fb, a.P, 4 * l + OP_DOWN, d.xres, dm,
-                            [&](int tile, float (&acc)[NT][4]) { epi_residual<NT>(c, a, gain_next, tile, acc); });
+                gemm_op<NT, TWO, BIG>(c, a.fb, a.P, 4 * l + OP_DOWN, g.G, dm, m.cfg.rms_eps, d.xres, dm,
+                            [&](int tile, int rb, float (&acc)[NT][4]) { epi_residual<NT>(c, a, gain_next, tile, rb, acc); });
             } else {
                 const int slice = op_slice(op, c.cta, c.ncta);
-                gemm_op<NT, TWO>(c, a.fb, a.P, 4 * l + OP_DOWN, nullptr, 0,
-                            [&](int tile, float (&acc)[NT][4]) { epi_partial<NT>(c, a, op, slice, tile, acc); });
+                gemm_op<NT, TWO, BIG>(c, a.fb, a.P, 4 * l + OP_DOWN, g.G, dm, m.cfg.rms_eps, nullptr, 0,
+                            [&](int tile, int rb, float (&acc)[NT][4]) { epi_partial<NT>(c, a, op, slice, tile, rb, acc); });
             }
             stamp();
             grid_barrier(c, a.fb);
             if (op.S > 1) {
-                phase_residual<NT>(c, a, op, gain_next);
+                phase_residual(c, a, op, gain_next);
                 grid_barrier(c, a.fb);
             }
             stamp();
         }
     }
     if (a.P.has_head) {
-        gemm_op<NT, TWO>(c, a.fb, a.P, 4 * L, nullptr, 0,
-                    [&](int tile, float (&acc)[NT][4]) { epi_head<NT>(c, a, row_dst, bias_at, tile, acc); });
+        gemm_op<NT, TWO, BIG>(c, a.fb, a.P, 4 * L, g.G, dm, m.cfg.rms_eps, nullptr, 0,
+                    [&](int tile, int rb, float (&acc)[NT][4]) { epi_head<NT>(c, a, row_dst, bias_at, tile, rb, acc); });
         stamp();
         grid_barrier(c, a.fb);
         stamp();
@@ -379,7 +386,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
 
 namespace fwd {
 
-static inline Plan make_plan(const ModelDev &m, const DevPtrs &d, const FwdBufs &fb, int ncta, bool has_head) {
+static inline Plan make_plan(const ModelDev &m, const DevPtrs &d, const FwdBufs &fb, int ncta, bool has_head, const Geom &geom) {
     Plan P;
     memset(&P, 0, sizeof P);
     const pacer_model_cfg &k = m.cfg;
@@ -415,40 +422,60 @@ static inline Plan make_plan(const ModelDev &m, const DevPtrs &d, const FwdBufs 
     // one pass per projection where N = 256 allows it; a model in which some block has up to twice as many tiles
     // runs the kernel variant with two accumulators (the activations are then still read once)
     P.max_tiles = MMA_TILES;
-    for (int i = 0; i < N_OPS; ++i) {
+    const bool big = geom.nt > 4;
+    for (int i = 0; i < N_OPS && !big; ++i) {
         if (i == OP_HEAD && !has_head) continue;
         const GemmOp &o = P.op[i];
         const int groups = ncta / o.S, per_block = (o.MT + groups - 1) / groups;
         if (per_block > MMA_TILES && per_block <= MAX_TILES) P.max_tiles = MAX_TILES;
+    }
+    // shared memory: the forwards with at most 32 rows keep 88 KB of scratch (activation stages of 256 k columns
+    // in front) and the large weight ring; the wide ones stage one k block of all row groups at a time, three
+    // stages deep, and leave the rest to the weight ring
+    P.xkb_bytes = 2 * geom.nt * geom.G * 1024;
+    if (!big) {
+        P.xkb = XK / KB; P.xs = x_stages(geom.nt);
+        P.scratch_bytes = SCRATCH_BYTES; P.ring_bytes = RING_BYTES;
+        P.acc_stride = 0;
+    } else {
+        P.xkb = std::max(1, std::min(XK / KB, (32 * 1024) / P.xkb_bytes));
+        P.xs = std::max(1, std::min(XS_MAX, BIG_XBYTES / (P.xkb * P.xkb_bytes)));
+        P.scratch_bytes = std::max(SCRATCH_BYTES, P.xs * P.xkb * P.xkb_bytes);
+        P.ring_bytes = SCRATCH_BYTES + RING_BYTES - P.scratch_bytes;
+        P.acc_stride = geom.G == 3 ? 160 : ACC_COLS;
+        if (geom.G == 3) P.max_tiles = 10;
     }
     P.n_layers = k.n_layers;
     P.has_head = has_head ? 1 : 0;
     return P;
 }
 
-template <int NT, bool TWO>
+template <int NT, bool TWO, bool BIG>
 static inline cudaError_t launch_nt(const Args &a, int which, int ncta, cudaStream_t st) {
     static bool attr_set[64] = {};           // the opt-in is per device
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-        e = cudaFuncSetAttribute(k_forward<NT, TWO>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+        e = cudaFuncSetAttribute(k_forward<NT, TWO, BIG>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
     void *params[] = {(void *)&a, (void *)&which};
-    return cudaLaunchCooperativeKernel((const void *)k_forward<NT, TWO>, dim3(ncta), dim3(THREADS), params, SMEM_BYTES, st);
+    return cudaLaunchCooperativeKernel((const void *)k_forward<NT, TWO, BIG>, dim3(ncta), dim3(THREADS), params, SMEM_BYTES, st);
 }
 
-// The variant with two accumulators runs the models in which some block has more than MMA_TILES tiles of a projection.
+// The variant with two accumulators runs the models in which some block has more than MMA_TILES tiles of a
+// projection; the wide variants (6 or 8 tiles per row group, up to three groups) the forwards with more than 32 rows.
 static inline cudaError_t launch(const Args &a, int which, int ncta, cudaStream_t st) {
     const bool two = a.P.max_tiles > MMA_TILES;
     switch (a.g.nt) {
-        case 1: return two ? launch_nt<1, true>(a, which, ncta, st) : launch_nt<1, false>(a, which, ncta, st);
-        case 2: return two ? launch_nt<2, true>(a, which, ncta, st) : launch_nt<2, false>(a, which, ncta, st);
-        case 3: return two ? launch_nt<3, true>(a, which, ncta, st) : launch_nt<3, false>(a, which, ncta, st);
-        case 4: return two ? launch_nt<4, true>(a, which, ncta, st) : launch_nt<4, false>(a, which, ncta, st);
+        case 1: return two ? launch_nt<1, true, false>(a, which, ncta, st) : launch_nt<1, false, false>(a, which, ncta, st);
+        case 2: return two ? launch_nt<2, true, false>(a, which, ncta, st) : launch_nt<2, false, false>(a, which, ncta, st);
+        case 3: return two ? launch_nt<3, true, false>(a, which, ncta, st) : launch_nt<3, false, false>(a, which, ncta, st);
+        case 4: return two ? launch_nt<4, true, false>(a, which, ncta, st) : launch_nt<4, false, false>(a, which, ncta, st);
+        case 6: return launch_nt<6, false, true>(a, which, ncta, st);
+        case 8: return launch_nt<8, false, true>(a, which, ncta, st);
     }
     return cudaErrorInvalidValue;
 }

@@ -75,44 +75,47 @@ __device__ __forceinline__ RowDesc row_desc(int kind, const DevPtrs &d, int s, i
 // hidden row during its prefill), spread over the MMA warps of the grid by
 // 16-column tiles.  Leaves x (fp32), x * gain of the first RMSNorm (split bf16,
 // operand order) and the per-tile sums of squares.
-__device__ __forceinline__ void phase_begin(Ctx &c, const Args &a, int nt_total) {
+__device__ __forceinline__ void phase_begin(Ctx &c, const Args &a) {
     const DevPtrs &d = a.d;
     const ModelDev &m = a.m;
-    const int dm = m.cfg.d_model, ntiles = dm >> 4, rpad = nt_total * 8;
+    const XLay xl{a.g.nt, a.g.G};
+    const int dm = m.cfg.d_model, ntiles = dm >> 4, rpad = a.g.rpad;
     const int half = c.lane >> 4, col16 = c.lane & 15;
     for (int tile = c.cta * MMA_WARPS + c.warp; tile < ntiles; tile += c.ncta * MMA_WARPS) {
         const int col = tile * 16 + col16;
         const float gain = __bfloat162float(m.norm1[col]);
-        float vv[MAX_ROWS / 2];                         // all rows' loads in flight together (the phase is a latency chain)
+        for (int rc = 0; rc < rpad; rc += 32) {             // 32 rows at a time
+            float vv[16];                                   // their loads in flight together (the phase is a latency chain)
 #pragma unroll
-        for (int it = 0; it < MAX_ROWS / 2; ++it) {
-            const int r = 2 * it + half;
-            float v = 0.f;
-            if (2 * it < rpad && r < a.g.rtot && c.row_pos[r] >= 0) {
-                const int s = r / a.g.rps, j = r - s * a.g.rps;
-                if (a.kind == KIND_MB) {
-                    v = d.hpend[((size_t)s * (d.block_b + 1) + j) * dm + col];
-                    const int e = c.row_tok[r];
-                    if (e > 0 && d.use_posemb) v += __bfloat162float(m.posemb[(size_t)(e - 1) * dm + col]);
-                } else if (a.kind == KIND_PREFILL_B) {
-                    v = __ldcg(d.hidden + (size_t)r * dm + col);
-                } else {
-                    v = __bfloat162float(m.embed[(size_t)c.row_tok[r] * dm + col]);
+            for (int it = 0; it < 16; ++it) {
+                const int r = rc + 2 * it + half;
+                float v = 0.f;
+                if (rc + 2 * it < rpad && r < a.g.rtot && c.row_pos[r] >= 0) {
+                    const int s = r / a.g.rps, j = r - s * a.g.rps;
+                    if (a.kind == KIND_MB) {
+                        v = d.hpend[((size_t)s * (d.block_b + 1) + j) * dm + col];
+                        const int e = c.row_tok[r];
+                        if (e > 0 && d.use_posemb) v += __bfloat162float(m.posemb[(size_t)(e - 1) * dm + col]);
+                    } else if (a.kind == KIND_PREFILL_B) {
+                        v = __ldcg(d.hidden + (size_t)r * dm + col);
+                    } else {
+                        v = __bfloat162float(m.embed[(size_t)c.row_tok[r] * dm + col]);
+                    }
                 }
+                vv[it] = v;
             }
-            vv[it] = v;
-        }
 #pragma unroll
-        for (int it = 0; it < MAX_ROWS / 2; ++it) {
-            if (2 * it >= rpad) break;
-            const int r = 2 * it + half;
-            const float v = vv[it];
-            d.xres[(size_t)r * dm + col] = v;          // idle rows hold zeros: they stay finite through the layers
-            store_split(a.fb.xg, nt_total, r, col, v * gain);
-            float ss = v * v;
+            for (int it = 0; it < 16; ++it) {
+                if (rc + 2 * it >= rpad) break;
+                const int r = rc + 2 * it + half;
+                const float v = vv[it];
+                d.xres[(size_t)r * dm + col] = v;          // idle rows hold zeros: they stay finite through the layers
+                store_split(a.fb.xg, xl, r, col, v * gain);
+                float ss = v * v;
 #pragma unroll
-            for (int o = 8; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-            if (col16 == 0) a.fb.ssq[tile * MAX_ROWS + r] = ss;
+                for (int o = 8; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+                if (col16 == 0) a.fb.ssq[tile * MAX_ROWS + r] = ss;
+            }
         }
     }
 }
@@ -123,12 +126,12 @@ __device__ __forceinline__ void phase_begin(Ctx &c, const Args &a, int nt_total)
 // q/k/v tile: the deferred 1/rms of the input RMSNorm, then qkv[k slice][row][column] (the attention phase
 // adds the k slices' shares when it reads the rows).
 template <int NT>
-__device__ __forceinline__ void epi_qkv(Ctx &c, const Args &a, int slice, int tile, float (&acc)[NT][4]) {
+__device__ __forceinline__ void epi_qkv(Ctx &c, const Args &a, int slice, int tile, int rb, float (&acc)[NT][4]) {
     const int g = c.lane >> 2, t = c.lane & 3, N = a.m.qrows;
     const int n0 = tile * 16 + g, n1 = n0 + 8;
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
-        const int r0 = nt * 8 + 2 * t;
+        const int r0 = rb + nt * 8 + 2 * t;
         const float i0 = c.inv_rms[r0], i1 = c.inv_rms[r0 + 1];
         float *q0 = a.fb.qkv + ((size_t)slice * MAX_ROWS + r0) * N, *q1 = q0 + N;
         if (n0 < N) { q0[n0] = acc[nt][0] * i0; q1[n0] = acc[nt][1] * i1; }
@@ -141,8 +144,9 @@ __device__ __forceinline__ void epi_qkv(Ctx &c, const Args &a, int slice, int ti
 // RMSNorm that follows as split bf16 in operand order (the next projection's input),
 // and the tile's share of sum(x^2) per row.
 template <int NT>
-__device__ __forceinline__ void epi_residual(Ctx &c, const Args &a, const bf16 *gain_next, int tile, float (&acc)[NT][4]) {
+__device__ __forceinline__ void epi_residual(Ctx &c, const Args &a, const bf16 *gain_next, int tile, int rb, float (&acc)[NT][4]) {
     const int g = c.lane >> 2, t = c.lane & 3, dm = a.m.cfg.d_model;
+    const XLay xl{a.g.nt, a.g.G};
     const int n0 = tile * 16 + g, n1 = n0 + 8;
     const float g0 = n0 < dm ? __bfloat162float(gain_next[n0]) : 0.f, g1 = n1 < dm ? __bfloat162float(gain_next[n1]) : 0.f;
 #pragma unroll
@@ -150,17 +154,17 @@ __device__ __forceinline__ void epi_residual(Ctx &c, const Args &a, const bf16 *
         float ss[2] = {0.f, 0.f};
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
-            const int r = nt * 8 + 2 * t + i;
+            const int r = rb + nt * 8 + 2 * t + i;
             float *x = a.d.xres + (size_t)r * dm;
             if (n0 < dm) {
                 const float v = acc[nt][i];
                 x[n0] = v; ss[i] += v * v;
-                store_split(a.fb.xg, NT, r, n0, v * g0);
+                store_split(a.fb.xg, xl, r, n0, v * g0);
             }
             if (n1 < dm) {
                 const float v = acc[nt][2 + i];
                 x[n1] = v; ss[i] += v * v;
-                store_split(a.fb.xg, NT, r, n1, v * g1);
+                store_split(a.fb.xg, xl, r, n1, v * g1);
             }
         }
 #pragma unroll
@@ -169,20 +173,20 @@ __device__ __forceinline__ void epi_residual(Ctx &c, const Args &a, const bf16 *
             ss[1] += __shfl_xor_sync(0xffffffffu, ss[1], o);
         }
         if (g == 0) {
-            a.fb.ssq[tile * MAX_ROWS + nt * 8 + 2 * t] = ss[0];
-            a.fb.ssq[tile * MAX_ROWS + nt * 8 + 2 * t + 1] = ss[1];
+            a.fb.ssq[tile * MAX_ROWS + rb + nt * 8 + 2 * t] = ss[0];
+            a.fb.ssq[tile * MAX_ROWS + rb + nt * 8 + 2 * t + 1] = ss[1];
         }
     }
 }
 
 // One k slice of a residual-projection tile: stored as a partial, nothing waits for it.
 template <int NT>
-__device__ __forceinline__ void epi_partial(Ctx &c, const Args &a, const GemmOp &op, int slice, int tile, float (&acc)[NT][4]) {
+__device__ __forceinline__ void epi_partial(Ctx &c, const Args &a, const GemmOp &op, int slice, int tile, int rb, float (&acc)[NT][4]) {
     const int g = c.lane >> 2, t = c.lane & 3;
-    float *mine = a.fb.part + ((size_t)slice * op.MT + tile) * (NT * 8 * 16);
+    float *mine = a.fb.part + ((size_t)slice * op.MT + tile) * (a.g.rpad * 16);
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
-        const int r0 = nt * 8 + 2 * t;
+        const int r0 = rb + nt * 8 + 2 * t;
         mine[r0 * 16 + g] = acc[nt][0];
         mine[(r0 + 1) * 16 + g] = acc[nt][1];
         mine[r0 * 16 + g + 8] = acc[nt][2];
@@ -194,39 +198,43 @@ __device__ __forceinline__ void epi_partial(Ctx &c, const Args &a, const GemmOp 
 // projection: x += the slices' sums (slice order, so the result does not depend
 // on timing); x * gain of the next RMSNorm as split bf16; sum(x^2) per tile.
 // Spread over the MMA warps of the grid by 16-column tiles.
-template <int NT>
 __device__ __forceinline__ void phase_residual(Ctx &c, const Args &a, const GemmOp &op, const bf16 *gain_next) {
-    constexpr int RPAD = NT * 8, NIT = RPAD / 2;
-    const int dm = a.m.cfg.d_model, ntiles = dm >> 4;
+    const XLay xl{a.g.nt, a.g.G};
+    const int dm = a.m.cfg.d_model, ntiles = dm >> 4, rpad = a.g.rpad;
     const int half = c.lane >> 4, col16 = c.lane & 15;
     for (int tile = c.cta * MMA_WARPS + c.warp; tile < ntiles; tile += c.ncta * MMA_WARPS) {
         const int col = tile * 16 + col16;
         const float gain = __bfloat162float(gain_next[col]);
-        float v[NIT];
+        for (int rc = 0; rc < rpad; rc += 32) {             // 32 rows at a time (fewer in the last round)
+            constexpr int NIT = 16;
+            float v[NIT];
 #pragma unroll
-        for (int it = 0; it < NIT; ++it) v[it] = __ldcg(a.d.xres + (size_t)(2 * it + half) * dm + col);
-        for (int s0 = 0; s0 < op.S; s0 += 4) {          // four slices' loads in flight together
-            float p[4][NIT];
+            for (int it = 0; it < NIT; ++it)
+                v[it] = rc + 2 * it < rpad ? __ldcg(a.d.xres + (size_t)(rc + 2 * it + half) * dm + col) : 0.f;
+            for (int s0 = 0; s0 < op.S; s0 += 4) {          // four slices' loads in flight together
+                float p[4][NIT];
 #pragma unroll
-            for (int ds = 0; ds < 4; ++ds)
+                for (int ds = 0; ds < 4; ++ds)
 #pragma unroll
-                for (int it = 0; it < NIT; ++it)
-                    p[ds][it] = s0 + ds < op.S
-                        ? __ldcg(a.fb.part + (((size_t)(s0 + ds) * op.MT + tile) * RPAD + 2 * it + half) * 16 + col16) : 0.f;
+                    for (int it = 0; it < NIT; ++it)
+                        p[ds][it] = (s0 + ds < op.S && rc + 2 * it < rpad)
+                            ? __ldcg(a.fb.part + (((size_t)(s0 + ds) * op.MT + tile) * rpad + rc + 2 * it + half) * 16 + col16) : 0.f;
 #pragma unroll
-            for (int ds = 0; ds < 4; ++ds)              // slice order: the sum does not depend on timing
+                for (int ds = 0; ds < 4; ++ds)              // slice order: the sum does not depend on timing
 #pragma unroll
-                for (int it = 0; it < NIT; ++it) v[it] += p[ds][it];
-        }
+                    for (int it = 0; it < NIT; ++it) v[it] += p[ds][it];
+            }
 #pragma unroll
-        for (int it = 0; it < NIT; ++it) {
-            const int r = 2 * it + half;
-            a.d.xres[(size_t)r * dm + col] = v[it];
-            store_split(a.fb.xg, NT, r, col, v[it] * gain);
-            float ss = v[it] * v[it];
+            for (int it = 0; it < NIT; ++it) {
+                if (rc + 2 * it >= rpad) break;
+                const int r = rc + 2 * it + half;
+                a.d.xres[(size_t)r * dm + col] = v[it];
+                store_split(a.fb.xg, xl, r, col, v[it] * gain);
+                float ss = v[it] * v[it];
 #pragma unroll
-            for (int o = 8; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-            if (col16 == 0) a.fb.ssq[tile * MAX_ROWS + r] = ss;
+                for (int o = 8; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+                if (col16 == 0) a.fb.ssq[tile * MAX_ROWS + r] = ss;
+            }
         }
     }
 }
@@ -235,19 +243,20 @@ __device__ __forceinline__ void phase_residual(Ctx &c, const Args &a, const Gemm
 // up rows of the same f, so a lane holds both; 1/rms of the input RMSNorm, then
 // silu(gate) * up as split bf16 in the operand order the down projection reads.
 template <int NT>
-__device__ __forceinline__ void epi_swiglu(Ctx &c, const Args &a, int tile, float (&acc)[NT][4]) {
+__device__ __forceinline__ void epi_swiglu(Ctx &c, const Args &a, int tile, int rb, float (&acc)[NT][4]) {
     const int g = c.lane >> 2, t = c.lane & 3, F = a.m.cfg.d_ffn;
+    const XLay xl{a.g.nt, a.g.G};
     const int f = tile * 8 + g;
     if (f >= F) return;
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
-            const int r = nt * 8 + 2 * t + i;
+            const int r = rb + nt * 8 + 2 * t + i;
             const float inv = c.inv_rms[r];
             const float gt = acc[nt][i] * inv, up = acc[nt][2 + i] * inv;
             const float v = (r < a.g.rtot && c.row_pos[r] >= 0) ? gt / (1.f + expf(-gt)) * up : 0.f;
-            store_split(a.d.act, NT, r, f, v);
+            store_split(a.d.act, xl, r, f, v);
         }
     }
 }
@@ -255,7 +264,7 @@ __device__ __forceinline__ void epi_swiglu(Ctx &c, const Args &a, int tile, floa
 // LM-head tile: 1/rms of the final RMSNorm, planted bias, logits to their
 // destination rows, and the tile's (max, argmax, runner-up) per row.
 template <int NT>
-__device__ __forceinline__ void epi_head(Ctx &c, const Args &a, float *const *row_dst, const int *bias_at, int tile,
+__device__ __forceinline__ void epi_head(Ctx &c, const Args &a, float *const *row_dst, const int *bias_at, int tile, int rb,
                                          float (&acc)[NT][4]) {
     const int g = c.lane >> 2, t = c.lane & 3, V = a.m.cfg.vocab;
     const int n0 = tile * 16 + g, n1 = n0 + 8;
@@ -263,7 +272,7 @@ __device__ __forceinline__ void epi_head(Ctx &c, const Args &a, float *const *ro
     for (int nt = 0; nt < NT; ++nt) {
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
-            const int r = nt * 8 + 2 * t + i;
+            const int r = rb + nt * 8 + 2 * t + i;
             float *dst = row_dst[r];
             Top2 tp{-INFINITY, 0x7fffffff, -INFINITY};
             if (dst) {

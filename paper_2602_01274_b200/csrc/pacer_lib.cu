@@ -98,7 +98,8 @@ static bool cfg_ok(const pacer_cfg *c) {
     if (c->criterion < 0 || c->criterion > 2) return false;
     if (c->mb_scope < 0 || c->mb_scope > 2) return false;
     if (!(c->rho > 0.f)) return false;
-    if ((int64_t)c->max_batch * (c->gamma_cap + 1) > fwd::MAX_ROWS) return false;   // rows of one verify forward
+    if ((int64_t)c->max_batch * (c->gamma_cap + 1) > 144) return false;    // rows of one verify forward (see make_geom)
+    if (c->max_batch > fwd::MAX_SEQ) return false;
     return true;
 }
 
@@ -106,6 +107,23 @@ static pacer_model_cfg mb_cfg(const pacer_cfg &c) {
     pacer_model_cfg m = c.draft;
     m.n_layers = 1;
     return m;
+}
+
+// Rows of a forward as groups of eight-row tiles for the tensor cores: up to 32 rows one group of 1..4 tiles;
+// wider forwards groups of 6 or 8 tiles (48 / 64 rows), as few padded rows as possible, three groups at most.
+static Geom make_geom(int batch, int rps) {
+    Geom g;
+    g.batch = batch; g.rps = rps; g.rtot = batch * rps;
+    const int r = g.rtot;
+    if (r <= 32) { g.nt = (r + 7) / 8; g.G = 1; }
+    else if (r <= 48) { g.nt = 6; g.G = 1; }
+    else if (r <= 64) { g.nt = 8; g.G = 1; }
+    else if (r <= 96) { g.nt = 6; g.G = 2; }
+    else if (r <= 128) { g.nt = 8; g.G = 2; }
+    else if (r <= 144) { g.nt = 6; g.G = 3; }
+    else { g.nt = 8; g.G = 3; }
+    g.rpad = g.G * g.nt * 8;
+    return g;
 }
 
 struct Carver {
@@ -147,6 +165,7 @@ static Layout make_layout(const pacer_cfg &c) {
     const int rps_max = gc + 1 > c.block_b + 1 ? gc + 1 : c.block_b + 1;
     L.rtot_max = B * rps_max;
     L.nt_max = (L.rtot_max + 7) / 8;
+    const size_t RP = std::min<size_t>(fwd::MAX_ROWS, make_geom(1, std::max(L.rtot_max, 32)).rpad);   // padded rows of the widest forward
     L.max_steps = c.max_ctx;
     int d_max = 0, f_max = 0, h_max = 0, hd_max = 0, qrows_max = 0;
     for (int i = 0; i < 3; ++i) {
@@ -167,7 +186,7 @@ static Layout make_layout(const pacer_cfg &c) {
     L.sched_win = cv.take(sizeof(int32_t) * B * L.max_steps);
     L.row_pos = cv.take(sizeof(int32_t) * fwd::MAX_ROWS);
     L.row_tok = cv.take(sizeof(int32_t) * fwd::MAX_ROWS);
-    L.n_rows = cv.take(sizeof(int32_t) * fwd::MAX_ROWS);
+    L.n_rows = cv.take(sizeof(int32_t) * fwd::MAX_SEQ);
     L.row_arg = cv.take(sizeof(int32_t) * fwd::MAX_ROWS);
     L.row_margin = cv.take(sizeof(float) * fwd::MAX_ROWS);
     L.att_cnt = cv.take(sizeof(int32_t) * (size_t)B * h_max);
@@ -179,16 +198,16 @@ static Layout make_layout(const pacer_cfg &c) {
     L.verify_logits = cv.take(sizeof(float) * B * (gc + 1) * V);
     L.draft_logits = cv.take(sizeof(float) * B * gc * V);
     L.d_max = d_max; L.f_max = f_max;
-    L.xres = cv.take(sizeof(float) * fwd::MAX_ROWS * d_max);
-    L.hidden = cv.take(sizeof(float) * fwd::MAX_ROWS * d_max);
-    L.att = cv.take(sizeof(bf16) * 2 * fwd::MAX_ROWS * d_max);        // values, then rounding remainders
-    L.act = cv.take(sizeof(bf16) * 2 * fwd::MAX_ROWS * f_max);
-    L.qkv = cv.take(sizeof(float) * 4 * fwd::MAX_ROWS * qrows_max);     // up to four k slices
-    L.xg = cv.take(sizeof(bf16) * 2 * fwd::MAX_ROWS * d_max);
+    L.xres = cv.take(sizeof(float) * RP * d_max);
+    L.hidden = cv.take(sizeof(float) * RP * d_max);
+    L.att = cv.take(sizeof(bf16) * 2 * RP * d_max);        // values, then rounding remainders
+    L.act = cv.take(sizeof(bf16) * 2 * RP * f_max);
+    L.qkv = cv.take(sizeof(float) * 4 * fwd::MAX_ROWS * qrows_max);     // up to four k slices, MAX_ROWS apart
+    L.xg = cv.take(sizeof(bf16) * 2 * RP * d_max);
     L.ssq = cv.take(sizeof(float) * fwd::MAX_ROWS * (d_max / 16 + 1));
     L.tile_top = cv.take(sizeof(float) * 4 * fwd::MAX_ROWS * ((size_t)V / 16 + 1));
     L.attp = cv.take(sizeof(float) * (size_t)B * h_max * fwd::MAX_SPLIT * rps_max * (hd_max + 2));
-    L.part_bytes = sizeof(float) * 8 * (size_t)d_max * fwd::MAX_ROWS;      // up to 8 k slices of [d/16][32][16]
+    L.part_bytes = sizeof(float) * 8 * (size_t)(d_max + 16) * RP;         // up to 8 k slices of [d/16][padded rows][16]
     L.part = cv.take(L.part_bytes);
     for (int i = 0; i < 3; ++i) {
         const int hd = ms[i]->d_model / ms[i]->n_heads;
@@ -217,12 +236,6 @@ static Layout make_layout(const pacer_cfg &c) {
 extern "C" size_t pacer_workspace_bytes(const pacer_cfg *cfg) {
     if (!cfg_ok(cfg)) return 0;
     return make_layout(*cfg).total;
-}
-
-static Geom make_geom(int batch, int rps) {
-    Geom g;
-    g.batch = batch; g.rps = rps; g.rtot = batch * rps; g.nt = (g.rtot + 7) / 8;
-    return g;
 }
 
 static void set_geoms(pacer_ctx *c, int batch, int draft_rows = 2) {
@@ -439,10 +452,11 @@ static double model_weight_bytes(const ModelDev &m, bool head) {
 // persistent forward kernel, which also takes the stage's decisions in its tail.
 static int run_forward(pacer_ctx *c, int which, const Geom &g, int kind, int aux, bool head) {
     ModelDev &m = c->model[which];
-    if (g.rtot > fwd::MAX_ROWS || g.nt > 4) return fail(c, PACER_EUNSUPPORTED, "more than 32 rows in one forward");
-    const int key = which * 2 + (head ? 1 : 0);
+    if (g.rtot > fwd::MAX_ROWS || g.batch > fwd::MAX_SEQ) return fail(c, PACER_EUNSUPPORTED, "too many rows or sequences in one forward");
+    if (head && kind == KIND_VERIFY && g.rtot > c->ncta) return fail(c, PACER_EUNSUPPORTED, "more verify rows than blocks");
+    const int key = ((which * 2 + (head ? 1 : 0)) * 16 + g.nt) * 4 + g.G;
     auto it = c->plans.find(key);
-    if (it == c->plans.end()) it = c->plans.emplace(key, fwd::make_plan(m, c->d, c->fb, c->ncta, head)).first;
+    if (it == c->plans.end()) it = c->plans.emplace(key, fwd::make_plan(m, c->d, c->fb, c->ncta, head, g)).first;
     fwd::Args a;
     a.d = c->d; a.m = m; a.g = g; a.P = it->second; a.fb = c->fb; a.kind = kind; a.aux = aux;
     a.fb.prof = (c->prof_on && c->ncta <= fwd::PROF_BLOCKS) ? c->prof_stamps : nullptr;
