@@ -237,7 +237,7 @@ struct XLay {
     int nt, G;                     // eight-row tiles per group, groups
 };
 __device__ __forceinline__ size_t xatom_index(int r, int k, XLay x, int plane) {
-    const int kk = k & 63, rr = r & 7, rg = 8 * x.nt, g = r / rg, rl = r - g * rg;
+    const int kk = k & 63, rr = r & 7, rg = 8 * x.nt, g = x.G == 1 ? 0 : r / rg, rl = r - g * rg;   // (one group: no division)
     return ((size_t)(k >> 6) * (2 * x.nt * x.G) + g * (2 * x.nt) + plane * x.nt + (rl >> 3)) * 512 + rr * 64 +
            ((((kk >> 3) ^ rr) << 3) | (kk & 7));
 }

@@ -323,7 +323,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
             stamp();
             grid_barrier(c, a.fb);
             if (op.S > 1) {
-                phase_residual(c, a, op, gain_next);
+                phase_residual<NT, BIG>(c, a, op, gain_next);
                 grid_barrier(c, a.fb);
             }
             stamp();
@@ -346,7 +346,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
             stamp();
             grid_barrier(c, a.fb);
             if (op.S > 1) {
-                phase_residual(c, a, op, gain_next);
+                phase_residual<NT, BIG>(c, a, op, gain_next);
                 grid_barrier(c, a.fb);
             }
             stamp();

@@ -146,7 +146,7 @@ __device__ __forceinline__ void epi_qkv(Ctx &c, const Args &a, int slice, int ti
 template <int NT>
 __device__ __forceinline__ void epi_residual(Ctx &c, const Args &a, const bf16 *gain_next, int tile, int rb, float (&acc)[NT][4]) {
     const int g = c.lane >> 2, t = c.lane & 3, dm = a.m.cfg.d_model;
-    const XLay xl{a.g.nt, a.g.G};
+    const XLay xl{NT, NT <= 4 ? 1 : a.g.G};    // (at most 32 rows: one group, known at compile time)
     const int n0 = tile * 16 + g, n1 = n0 + 8;
     const float g0 = n0 < dm ? __bfloat162float(gain_next[n0]) : 0.f, g1 = n1 < dm ? __bfloat162float(gain_next[n1]) : 0.f;
 #pragma unroll
@@ -198,26 +198,28 @@ __device__ __forceinline__ void epi_partial(Ctx &c, const Args &a, const GemmOp 
 // projection: x += the slices' sums (slice order, so the result does not depend
 // on timing); x * gain of the next RMSNorm as split bf16; sum(x^2) per tile.
 // Spread over the MMA warps of the grid by 16-column tiles.
+template <int NT, bool BIG>
 __device__ __forceinline__ void phase_residual(Ctx &c, const Args &a, const GemmOp &op, const bf16 *gain_next) {
-    const XLay xl{a.g.nt, a.g.G};
-    const int dm = a.m.cfg.d_model, ntiles = dm >> 4, rpad = a.g.rpad;
+    const XLay xl{NT, NT <= 4 ? 1 : a.g.G};    // (at most 32 rows: one group, known at compile time)
+    // rows go 32 at a time (the narrow forwards have fewer, known at compile time: all their loads fly together)
+    constexpr int NIT = BIG ? 16 : NT * 4;
+    const int dm = a.m.cfg.d_model, ntiles = dm >> 4, rpad = BIG ? a.g.rpad : NT * 8;
     const int half = c.lane >> 4, col16 = c.lane & 15;
     for (int tile = c.cta * MMA_WARPS + c.warp; tile < ntiles; tile += c.ncta * MMA_WARPS) {
         const int col = tile * 16 + col16;
         const float gain = __bfloat162float(gain_next[col]);
-        for (int rc = 0; rc < rpad; rc += 32) {             // 32 rows at a time (fewer in the last round)
-            constexpr int NIT = 16;
+        for (int rc = 0; rc < rpad; rc += 2 * NIT) {
             float v[NIT];
 #pragma unroll
             for (int it = 0; it < NIT; ++it)
-                v[it] = rc + 2 * it < rpad ? __ldcg(a.d.xres + (size_t)(rc + 2 * it + half) * dm + col) : 0.f;
+                v[it] = (!BIG || rc + 2 * it < rpad) ? __ldcg(a.d.xres + (size_t)(rc + 2 * it + half) * dm + col) : 0.f;
             for (int s0 = 0; s0 < op.S; s0 += 4) {          // four slices' loads in flight together
                 float p[4][NIT];
 #pragma unroll
                 for (int ds = 0; ds < 4; ++ds)
 #pragma unroll
                     for (int it = 0; it < NIT; ++it)
-                        p[ds][it] = (s0 + ds < op.S && rc + 2 * it < rpad)
+                        p[ds][it] = (s0 + ds < op.S && (!BIG || rc + 2 * it < rpad))
                             ? __ldcg(a.fb.part + (((size_t)(s0 + ds) * op.MT + tile) * rpad + rc + 2 * it + half) * 16 + col16) : 0.f;
 #pragma unroll
                 for (int ds = 0; ds < 4; ++ds)              // slice order: the sum does not depend on timing
@@ -226,7 +228,7 @@ __device__ __forceinline__ void phase_residual(Ctx &c, const Args &a, const Gemm
             }
 #pragma unroll
             for (int it = 0; it < NIT; ++it) {
-                if (rc + 2 * it >= rpad) break;
+                if (BIG && rc + 2 * it >= rpad) break;
                 const int r = rc + 2 * it + half;
                 a.d.xres[(size_t)r * dm + col] = v[it];
                 store_split(a.fb.xg, xl, r, col, v[it] * gain);
@@ -245,7 +247,7 @@ __device__ __forceinline__ void phase_residual(Ctx &c, const Args &a, const Gemm
 template <int NT>
 __device__ __forceinline__ void epi_swiglu(Ctx &c, const Args &a, int tile, int rb, float (&acc)[NT][4]) {
     const int g = c.lane >> 2, t = c.lane & 3, F = a.m.cfg.d_ffn;
-    const XLay xl{a.g.nt, a.g.G};
+    const XLay xl{NT, NT <= 4 ? 1 : a.g.G};    // (at most 32 rows: one group, known at compile time)
     const int f = tile * 8 + g;
     if (f >= F) return;
 #pragma unroll
