@@ -337,7 +337,8 @@ def main():
         # Section 3.3: the target's responses to seeded random prompts, drafts from every prefix, labels up to the
         # first mismatch, cross-entropy, AdamW.  Plain PyTorch, outside the decoding path and outside the timed region.
         from paper_2602_01274_b200 import train_preverify
-        tensors, train_report = train_preverify.train(cfg, pair, dev, n_prompts=args.train_prompts, batch_prompts=32,
+        tensors, train_report = train_preverify.train(cfg, pair, dev, n_prompts=args.train_prompts, epochs=12, lr=1e-3,
+                                                      batch_prompts=64 if cfg.draft.n_params() < 5e8 else 32,
                                                       log=lambda m: print(m, file=sys.stderr, flush=True))
         pair["preverify"] = {k: v.to(dev) for k, v in tensors.items()}
         torch.cuda.empty_cache()

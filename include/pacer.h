@@ -214,8 +214,12 @@ int pacer_read_buffer(pacer_ctx *ctx, int which, void *host_dst, size_t bytes);
  * for a sequence that has stopped drafting) and stays two steps ahead of the device:
  * it reads the finished flags of an EARLIER step from pinned memory (copied there
  * behind an event) to know when to stop enqueuing, and never waits for the step it
- * has just enqueued.  Greedy runs take the acceptance (Eq. 5) in the tail of the
- * verify forward; sampling runs in a kernel of its own.
+ * has just enqueued.  The launches of one step (the draft forwards and pre-verification
+ * calls of the whole window, the verify forward, the acceptance) are captured once
+ * per context as a CUDA graph and replayed every step (not on the legacy default
+ * stream, which cannot be captured: there the launches are issued one by one).  Greedy runs take the
+ * acceptance (Eq. 5) in the tail of the verify forward; sampling runs in a kernel of
+ * its own.
  * Outputs, all host, caller-owned:
  *   out_tokens     int32 [batch][max_new]
  *   out_n_steps    int32 [batch]

@@ -140,7 +140,8 @@ class Context:
             self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
             base = self.workspace.data_ptr()
             self._ws_ptr = (base + 255) // 256 * 256
-            self.stream = stream if stream is not None else torch.cuda.current_stream(self.device)
+            # a stream of its own (the legacy default stream cannot be captured into the per-step CUDA graph)
+            self.stream = stream if stream is not None else torch.cuda.Stream(self.device)
             h = _P()
             rc = _lib.pacer_create(C.byref(cfg), self._ws_ptr, nbytes, self.stream.cuda_stream, C.byref(h))
         self._h = h
@@ -175,7 +176,9 @@ class Context:
             self._keep.append(succ)
             sp = succ.data_ptr()
         with torch.cuda.device(self.device):
+            self.stream.wait_stream(torch.cuda.current_stream(self.device))     # the tensors may still be being written
             self._check(_lib.pacer_load_weights(self._h, which, arr, len(tensors), sp))
+            torch.cuda.current_stream(self.device).wait_stream(self.stream)     # later torch work sees the copy done
 
     def pacer_prefill(self, prompt, max_new, gamma_max, threshold, mode=PACER_GREEDY, seed=0):
         p = _i32(prompt)

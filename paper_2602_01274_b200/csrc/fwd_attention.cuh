@@ -44,16 +44,22 @@ __device__ __forceinline__ void split_bf16(float v, bf16 &hi, bf16 &lo) {
     lo = __float2bfloat16(v - __bfloat162float(hi));
 }
 
-// Rotary embedding of the new rows of (seq, head h): q (scaled) to shared memory;
-// k, v of the kv head as the cache holds them, to shared memory and, by one item
-// per kv head, to the cache.  All as split bf16.
-template <int HD>
-__device__ __forceinline__ void attention_rows(Ctx &c, const Args &a, int layer, int seq, int h, bool writer) {
+// Rotary embedding of the new rows of one item: q (scaled) of its query rows to shared memory; k, v of the kv head as
+// the cache holds them, to shared memory and, by one item per kv head, to the cache.  All as split bf16.
+// Query rows are VIRTUAL rows: with grouped-query attention the `group` query heads of a kv head times the n_r rows
+// of the sequence are numbered v = (head within the group) * n_r + row, and an item takes 32 of them (vbase ..
+// vbase + nv - 1), so that the keys of a kv head are read once for a full 32-row tile pair whatever n_r is; without
+// grouping v is the row itself.  Local row lv of the item is virtual row vbase + lv; fresh key/value row lv is row
+// lv of the sequence.
+// KV = false (forwards with more than 32 rows per sequence): only the query rows are staged; the new keys and values
+// went to the cache in a pass of their own (attention_append) and are read from there.
+template <int HD, bool GQA, bool KV>
+__device__ __forceinline__ void attention_rows(Ctx &c, const Args &a, int layer, int seq, int kh, int vbase, int nv, bool writer) {
     using SM = AttSmem<HD>;
     constexpr int half = HD / 2;
     const DevPtrs &d = a.d;
     const ModelDev &m = a.m;
-    const int H = m.cfg.n_heads, Hkv = m.cfg.n_kv_heads, kh = h / (H / Hkv), qrows = m.qrows;
+    const int H = m.cfg.n_heads, Hkv = m.cfg.n_kv_heads, group = GQA ? H / Hkv : 1, qrows = m.qrows;
     const int n_r = c.n_rows[seq], r_base = seq * a.g.rps, pos0 = c.row_pos[r_base];
     bf16 *kn = reinterpret_cast<bf16 *>(c.scratch + SM::KN_OFF), *vn = reinterpret_cast<bf16 *>(c.scratch + SM::VN_OFF);
     const size_t cbase = (((size_t)layer * d.max_batch + seq) * Hkv + kh) * (size_t)d.max_ctx * HD;
@@ -63,8 +69,8 @@ __device__ __forceinline__ void attention_rows(Ctx &c, const Args &a, int layer,
     const int S = a.P.op[OP_QKV].S;
     const size_t sl = (size_t)MAX_ROWS * qrows;
     constexpr int U = 5;                                 // 17 rows of 128 channels are one batch
-    const int n_act = n_r * half;
-    for (int i = n_act + threadIdx.x; i < 32 * half; i += MMA_THREADS) {     // idle query rows are zeros
+    const int n_act = (GQA ? (KV ? max(nv, n_r) : nv) : n_r) * half;
+    for (int i = nv * half + threadIdx.x; i < 32 * half; i += MMA_THREADS) {     // idle query rows are zeros
         const int j = i / half, ii = i - j * half;
         bf16 *qrow = reinterpret_cast<bf16 *>(c.scratch + SM::Q_OFF + j * SM::QP);
         bf16 *qrow_lo = reinterpret_cast<bf16 *>(c.scratch + SM::Q_OFF + (32 + j) * SM::QP);
@@ -73,22 +79,29 @@ __device__ __forceinline__ void attention_rows(Ctx &c, const Args &a, int layer,
     }
     for (int i0 = threadIdx.x; i0 < n_act; i0 += U * MMA_THREADS) {
         float part[U][2][6];
-        float2 cs[U];
+        float2 csq[U], csk[U];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            const int i = i0 + u * MMA_THREADS, j = i / half, ii = i - j * half;
-            const bool on = i < n_act;
-            const float *row = a.fb.qkv + (size_t)(r_base + (on ? j : 0)) * qrows;
+            const int i = i0 + u * MMA_THREADS, lv = i / half, ii = i - lv * half;
+            const bool onk = KV && lv < n_r, onq = GQA ? lv < nv : onk;
+            int h = kh, jq = lv;                                 // query row lv: head and row of the sequence
+            if (GQA) { const int v = vbase + lv, hq = v / n_r; jq = v - hq * n_r; h = kh * group + hq; }
+            const float *rowk = a.fb.qkv + (size_t)(r_base + (onk ? lv : 0)) * qrows;
+            const float *rowq = GQA ? a.fb.qkv + (size_t)(r_base + (onq ? jq : 0)) * qrows : rowk;
             const int col[6] = {h * HD + ii, h * HD + ii + half, (H + kh) * HD + ii, (H + kh) * HD + ii + half,
                                 (H + Hkv + kh) * HD + ii, (H + Hkv + kh) * HD + ii + half};
-            cs[u] = on ? m.rope[(size_t)(pos0 + j) * half + ii] : make_float2(0.f, 0.f);
+            csq[u] = onq ? m.rope[(size_t)(pos0 + jq) * half + ii] : make_float2(0.f, 0.f);
+            csk[u] = !GQA ? csq[u] : (onk ? m.rope[(size_t)(pos0 + lv) * half + ii] : make_float2(0.f, 0.f));
 #pragma unroll
             for (int s = 0; s < 2; ++s)
 #pragma unroll
-                for (int e = 0; e < 6; ++e) part[u][s][e] = (on && s < S) ? __ldcg(row + s * sl + col[e]) : 0.f;
-            if (S > 2 && on) {                                   // slices 2, 3: a second wave of loads
+                for (int e = 0; e < 6; ++e)
+                    part[u][s][e] = ((e < 2 ? onq : onk) && s < S) ? __ldcg((e < 2 ? rowq : rowk) + s * sl + col[e]) : 0.f;
+            if (S > 2) {                                         // slices 2, 3: a second wave of loads
 #pragma unroll
                 for (int e = 0; e < 6; ++e) {
+                    if (!(e < 2 ? onq : onk)) continue;
+                    const float *row = e < 2 ? rowq : rowk;
                     const float p2 = __ldcg(row + 2 * sl + col[e]), p3 = S > 3 ? __ldcg(row + 3 * sl + col[e]) : 0.f;
                     part[u][0][e] += p2; part[u][1][e] += p3;
                 }
@@ -96,21 +109,24 @@ __device__ __forceinline__ void attention_rows(Ctx &c, const Args &a, int layer,
         }
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            const int i = i0 + u * MMA_THREADS, j = i / half, ii = i - j * half;
+            const int i = i0 + u * MMA_THREADS, lv = i / half, ii = i - lv * half;
             if (i >= n_act) continue;
-            bf16 *qrow = reinterpret_cast<bf16 *>(c.scratch + SM::Q_OFF + j * SM::QP);
-            bf16 *qrow_lo = reinterpret_cast<bf16 *>(c.scratch + SM::Q_OFF + (32 + j) * SM::QP);
-            {
-                const int pos = pos0 + j;
-                float in[6];
+            float in[6];
 #pragma unroll
-                for (int e = 0; e < 6; ++e) in[e] = part[u][0][e] + part[u][1][e];
-                const float qa = in[0], qb = in[1], ka = in[2], kb = in[3];
-                split_bf16((qa * cs[u].x - qb * cs[u].y) * scale, qrow[ii], qrow_lo[ii]);
-                split_bf16((qb * cs[u].x + qa * cs[u].y) * scale, qrow[ii + half], qrow_lo[ii + half]);
+            for (int e = 0; e < 6; ++e) in[e] = part[u][0][e] + part[u][1][e];
+            if (GQA ? lv < nv : true) {
+                bf16 *qrow = reinterpret_cast<bf16 *>(c.scratch + SM::Q_OFF + lv * SM::QP);
+                bf16 *qrow_lo = reinterpret_cast<bf16 *>(c.scratch + SM::Q_OFF + (32 + lv) * SM::QP);
+                const float qa = in[0], qb = in[1];
+                split_bf16((qa * csq[u].x - qb * csq[u].y) * scale, qrow[ii], qrow_lo[ii]);
+                split_bf16((qb * csq[u].x + qa * csq[u].y) * scale, qrow[ii + half], qrow_lo[ii + half]);
+            }
+            if (KV && (GQA ? lv < n_r : true)) {
+                const int j = lv, pos = pos0 + j;
+                const float ka = in[2], kb = in[3];
                 bf16 k0, k0l, k1, k1l, v0, v0l, v1, v1l;
-                split_bf16(ka * cs[u].x - kb * cs[u].y, k0, k0l);
-                split_bf16(kb * cs[u].x + ka * cs[u].y, k1, k1l);
+                split_bf16(ka * csk[u].x - kb * csk[u].y, k0, k0l);
+                split_bf16(kb * csk[u].x + ka * csk[u].y, k1, k1l);
                 split_bf16(in[4], v0, v0l);
                 split_bf16(in[5], v1, v1l);
                 kn[j * HD + ii] = k0; kn[j * HD + ii + half] = k1;
@@ -126,6 +142,42 @@ __device__ __forceinline__ void attention_rows(Ctx &c, const Args &a, int layer,
                 }
             }
         }
+    }
+}
+
+// Forwards with more than 32 rows per sequence (prompt chunks): rotary embedding of the new k rows jbase .. jbase+31
+// of (seq, kv head) and append of k, v to the cache as split bf16.  The attention items that follow a grid barrier
+// read every key from the cache, the new ones under a causal mask.
+template <int HD>
+__device__ __forceinline__ void attention_append(Ctx &c, const Args &a, int layer, int seq, int kh, int jbase) {
+    constexpr int half = HD / 2;
+    const DevPtrs &d = a.d;
+    const ModelDev &m = a.m;
+    const int H = m.cfg.n_heads, Hkv = m.cfg.n_kv_heads, qrows = m.qrows;
+    const int n_r = c.n_rows[seq], r_base = seq * a.g.rps, pos0 = c.row_pos[r_base];
+    const size_t cbase = (((size_t)layer * d.max_batch + seq) * Hkv + kh) * (size_t)d.max_ctx * HD;
+    const int S = a.P.op[OP_QKV].S;
+    const size_t sl = (size_t)MAX_ROWS * qrows;
+    const int n_el = min(32, n_r - jbase) * half;
+    for (int i = threadIdx.x; i < n_el; i += MMA_THREADS) {
+        const int j = jbase + i / half, ii = i % half, pos = pos0 + j;
+        const float *row = a.fb.qkv + (size_t)(r_base + j) * qrows;
+        const int col[4] = {(H + kh) * HD + ii, (H + kh) * HD + ii + half, (H + Hkv + kh) * HD + ii, (H + Hkv + kh) * HD + ii + half};
+        float in[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int s_ = 0; s_ < S; ++s_)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) in[e] += __ldcg(row + s_ * sl + col[e]);
+        const float2 cs = m.rope[(size_t)pos * half + ii];
+        bf16 k0, k0l, k1, k1l, v0, v0l, v1, v1l;
+        split_bf16(in[0] * cs.x - in[1] * cs.y, k0, k0l);
+        split_bf16(in[1] * cs.x + in[0] * cs.y, k1, k1l);
+        split_bf16(in[2], v0, v0l);
+        split_bf16(in[3], v1, v1l);
+        bf16 *kc = m.kcache + cbase + (size_t)pos * HD, *vc = m.vcache + cbase + (size_t)pos * HD;
+        kc[ii] = k0; kc[ii + half] = k1;
+        kc[m.kv_lo + ii] = k0l; kc[m.kv_lo + ii + half] = k1l;
+        vc[ii] = v0; vc[ii + half] = v1;
+        vc[m.kv_lo + ii] = v0l; vc[m.kv_lo + ii + half] = v1l;
     }
 }
 
@@ -148,13 +200,14 @@ __device__ __forceinline__ void attention_prefetch(const Ctx &c, const bf16 *kca
 
 // The key loop of one warp: keys in steps of 8 (step st, st + KW, ...), first the
 // cached keys [lo, hi), then (last split only) the n_r keys of this forward, which
-// row j sees up to key j.  mt: the warp's 16-row query tile.  Leaves running max,
+// row j sees up to key j (jrow: the sequence row of the lane's two query rows, -1 for
+// an idle query row).  mt: the warp's 16-row query tile.  Leaves running max,
 // sum (this lane's share) and un-normalised output of rows g and g+8 of the tile.
 // Products of two remainders (2^-18 relative) are left out.
-template <int HD>
+template <int HD, bool WIDE>
 __device__ __forceinline__ void attention_keys(Ctx &c, const bf16 *kcache, const bf16 *vcache, size_t kv_lo, int lo, int hi,
-                                               int n_new, int n_r, int fresh_lo, int mt, int kw, int KW, float (&mx)[2],
-                                               float (&lsum)[2], float (&o)[HD / 8][4]) {
+                                               int n_new, int n_r, int fresh_lo, const int (&jrow)[2], int pos0, int mt, int kw,
+                                               int KW, float (&mx)[2], float (&lsum)[2], float (&o)[HD / 8][4]) {
     using SM = AttSmem<HD>;
     constexpr int NCH = HD / 32, NOT = HD / 8, QP = SM::QP, VP = SM::VP;
     const int g = c.lane >> 2, t = c.lane & 3;
@@ -217,10 +270,11 @@ __device__ __forceinline__ void attention_keys(Ctx &c, const bf16 *kcache, const
         float rmax[2] = {-INFINITY, -INFINITY};
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            const int key = key0 + 2 * t + (i & 1), row = mt * 16 + g + 8 * (i >> 1);
+            const int key = key0 + 2 * t + (i & 1), row = jrow[i >> 1];      // row of the sequence this query row is
             // (with a restricted attention context the keys of this forward before fresh_lo are outside it;
             // a row always sees itself)
-            const bool ok = key < kend && (!fresh || (key <= row && (key >= fresh_lo || key == row)));
+            // (WIDE: the new keys are in the cache too, key index = cache position: row j sees up to position pos0 + j)
+            const bool ok = key < kend && (fresh ? (key <= row && (key >= fresh_lo || key == row)) : (!WIDE || key <= pos0 + row));
             if (!ok) s[i] = -INFINITY;
             rmax[i >> 1] = fmaxf(rmax[i >> 1], s[i]);
         }
@@ -276,31 +330,42 @@ __device__ __forceinline__ void attention_keys(Ctx &c, const bf16 *kcache, const
     }
 }
 
-template <int HD>
-__device__ __forceinline__ void attention_item(Ctx &c, const Args &a, int layer, int seq, int h, int split, int nsplit) {
+template <int HD, bool GQA, bool WIDE>
+__device__ __forceinline__ void attention_item(Ctx &c, const Args &a, int layer, int seq, int kh, int vc, int split, int nsplit) {
     const XLay xl{a.g.nt, a.g.G};
     using SM = AttSmem<HD>;
     constexpr int PW = SM::PW, NOT = HD / 8;
     const DevPtrs &d = a.d;
     const ModelDev &m = a.m;
-    const int H = m.cfg.n_heads, Hkv = m.cfg.n_kv_heads, group = H / Hkv, kh = h / group;
+    const int H = m.cfg.n_heads, Hkv = m.cfg.n_kv_heads, group = GQA ? H / Hkv : 1;
     const int n_r = c.n_rows[seq], r_base = seq * a.g.rps, pos0 = c.row_pos[r_base];
+    const int vbase = GQA ? 32 * vc : 0, nv = GQA ? min(32, group * n_r - vbase) : n_r;      // this item's virtual query rows
     const size_t cbase = (((size_t)layer * d.max_batch + seq) * Hkv + kh) * (size_t)d.max_ctx * HD;
-    const int ks = min(c.key_start[seq], pos0), span = pos0 - ks;      // cached keys in the attention context: [ks, pos0)
+    // cached keys in the attention context: [ks, pos0); WIDE: up to the last new row this item's query rows see
+    int kv_end = pos0;
+    if (WIDE) { const int v_last = vbase + nv - 1; kv_end = pos0 + 1 + (vbase / n_r != v_last / n_r ? n_r - 1 : v_last % n_r); }
+    const int ks = min(c.key_start[seq], pos0), span = kv_end - ks;
     const int lo = ks + (int)((long long)span * split / nsplit), hi = ks + (int)((long long)span * (split + 1) / nsplit);
     const int fresh_lo = max(0, c.key_start[seq] - pos0);
-    const int two = n_r > 16 ? 1 : 0;                    // two query tiles: warps 0..3 take rows 0..15, warps 4..7 rows 16..31
+    const int two = nv > 16 ? 1 : 0;                     // two query tiles: warps 0..3 take rows 0..15, warps 4..7 rows 16..31
     const int mt = two ? (c.warp >> 2) : 0, kw = two ? (c.warp & 3) : c.warp, KW = two ? 4 : 8;
     const int g = c.lane >> 2, t = c.lane & 3;
+    int jrow[2];
+#pragma unroll
+    for (int hr = 0; hr < 2; ++hr) {
+        const int lv = mt * 16 + g + 8 * hr;
+        jrow[hr] = GQA ? (lv < nv ? (vbase + lv) % n_r : -1) : lv;
+    }
     if (hi > lo)
         for (int i = 0; i < ATT_PF; ++i) attention_prefetch<HD>(c, m.kcache + cbase, m.vcache + cbase, m.kv_lo, lo, hi, kw + i * KW);
-    attention_rows<HD>(c, a, layer, seq, h, split == 0 && h == kh * group);
+    attention_rows<HD, GQA, !WIDE>(c, a, layer, seq, kh, vbase, nv, !WIDE && split == 0 && vc == 0);
     bsync();
     float mx[2] = {-INFINITY, -INFINITY}, lsum[2] = {0.f, 0.f};
     float o[NOT][4];
 #pragma unroll
     for (int i = 0; i < NOT; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
-    attention_keys<HD>(c, m.kcache + cbase, m.vcache + cbase, m.kv_lo, lo, hi, split == nsplit - 1 ? n_r : 0, n_r, fresh_lo, mt, kw, KW, mx, lsum, o);
+    attention_keys<HD, WIDE>(c, m.kcache + cbase, m.vcache + cbase, m.kv_lo, lo, hi, (!WIDE && split == nsplit - 1) ? n_r : 0, n_r,
+                             fresh_lo, jrow, pos0, mt, kw, KW, mx, lsum, o);
 
     bsync();                                             // every warp is done with q, the new rows and the slots
     float *red = reinterpret_cast<float *>(c.scratch);   // [8 warps][16 rows][PW]
@@ -316,11 +381,10 @@ __device__ __forceinline__ void attention_item(Ctx &c, const Args &a, int layer,
     bsync();
     // merge the warps of each query tile -> the item's partial in global memory; with a single split the
     // result is final and goes straight to the output projection's input buffer
-    float *outp = a.fb.attp + (((size_t)(seq * H + h) * MAX_SPLIT + split) * a.g.rps) * PW;
     // per (row, warp) the factor exp(max_w - max) once, then one multiply-add per warp and output channel
     float *fw = red + MMA_WARPS * 16 * PW;               // [row][8] factors, then [row] max, [row] sum
     float *rowM = fw + 32 * MMA_WARPS, *rowL = rowM + 32;
-    if (threadIdx.x < n_r) {
+    if (threadIdx.x < nv) {
         const int j = threadIdx.x, w0 = two ? (j >> 4) * 4 : 0, rr = j & 15;
         float M = -INFINITY;
         for (int w = 0; w < KW; ++w) M = fmaxf(M, red[((size_t)(w0 + w) * 16 + rr) * PW + HD]);
@@ -334,20 +398,28 @@ __device__ __forceinline__ void attention_item(Ctx &c, const Args &a, int layer,
         rowM[j] = M; rowL[j] = L;
     }
     bsync();
-    for (int i = threadIdx.x; i < n_r * HD; i += MMA_THREADS) {
-        const int j = i / HD, ch = i - j * HD;
-        const int w0 = two ? (j >> 4) * 4 : 0, rr = j & 15;
+    for (int i = threadIdx.x; i < nv * HD; i += MMA_THREADS) {
+        const int lv = i / HD, ch = i - lv * HD;
+        const int w0 = two ? (lv >> 4) * 4 : 0, rr = lv & 15;
+        int h = kh, j = lv;                              // the head and sequence row this query row is
+        if (GQA) { const int v = vbase + lv, hq = v / n_r; j = v - hq * n_r; h = kh * group + hq; }
         float ov = 0.f;
-        for (int w = 0; w < KW; ++w) ov += red[((size_t)(w0 + w) * 16 + rr) * PW + ch] * fw[j * MMA_WARPS + w];
+        for (int w = 0; w < KW; ++w) ov += red[((size_t)(w0 + w) * 16 + rr) * PW + ch] * fw[lv * MMA_WARPS + w];
         if (nsplit == 1) {
-            store_split(d.att, xl, r_base + j, h * HD + ch, ov / rowL[j]);
+            store_split(d.att, xl, r_base + j, h * HD + ch, ov / rowL[lv]);
         } else {
-            float *op = outp + (size_t)j * PW;
+            float *op = a.fb.attp + ((((size_t)(seq * H + h) * MAX_SPLIT + split) * a.g.rps) + j) * PW;
             op[ch] = ov;
-            if (ch == 0) { op[HD] = rowM[j]; op[HD + 1] = rowL[j]; }
+            if (ch == 0) { op[HD] = rowM[lv]; op[HD + 1] = rowL[lv]; }
         }
     }
     bsync();
+}
+
+// Items of one (sequence, kv head) and key split: one per 32 virtual query rows (group * rows of the sequence).
+__device__ __forceinline__ int attention_chunks(const Args &a) {
+    const int group = a.m.cfg.n_heads / a.m.cfg.n_kv_heads;
+    return (group == 1 && a.g.rps <= 32) ? 1 : (group * a.g.rps + 31) / 32;
 }
 
 // Key-range splits of a head in this forward (the same value in every block).  With fewer (sequence, head)
@@ -357,8 +429,8 @@ __device__ __forceinline__ void attention_item(Ctx &c, const Args &a, int layer,
 __device__ __forceinline__ int attention_splits(const Ctx &c, const Args &a) {
     int lmax = 0;
     for (int s = 0; s < a.g.batch; ++s)
-        if (c.n_rows[s] > 0) lmax = max(lmax, c.row_pos[s * a.g.rps]);
-    const int pairs = a.g.batch * a.m.cfg.n_heads, cap = max(1, min(MAX_SPLIT, lmax / 64));
+        if (c.n_rows[s] > 0) lmax = max(lmax, c.row_pos[s * a.g.rps] + (a.g.rps > 32 ? c.n_rows[s] : 0));
+    const int pairs = a.g.batch * a.m.cfg.n_kv_heads * attention_chunks(a), cap = max(1, min(MAX_SPLIT, lmax / 64));
     if (pairs <= c.ncta) return max(1, min(c.ncta / pairs, cap));
     int best = 1;
     long long best_cost = -1;
@@ -400,15 +472,35 @@ __device__ __forceinline__ void phase_attention_merge(Ctx &c, const Args &a, int
     }
 }
 
-// All blocks: the attention items of one layer.
+// All blocks: the attention items of one layer.  Forwards with more than 32 rows per sequence (prompt chunks) first
+// append all new keys and values to the cache, pass a grid barrier, and then read every key from the cache.
 __device__ __forceinline__ void phase_attention(Ctx &c, const Args &a, int layer, int nsplit) {
-    const int H = a.m.cfg.n_heads, batch = a.g.batch;
-    const int items = batch * H * nsplit;
+    const int Hkv = a.m.cfg.n_kv_heads, group = a.m.cfg.n_heads / Hkv, batch = a.g.batch, nvc = attention_chunks(a);
+    const bool wide = a.g.rps > 32;
+    if (wide) {
+        const int nrc = (a.g.rps + 31) / 32, n_app = batch * Hkv * nrc;
+        for (int it = c.cta; it < n_app; it += c.ncta) {
+            const int jbase = (it % nrc) * 32, r1 = it / nrc, kh = r1 % Hkv, seq = r1 / Hkv;
+            if (jbase >= c.n_rows[seq]) continue;
+            if (a.m.hd == 64) attention_append<64>(c, a, layer, seq, kh, jbase);
+            else attention_append<128>(c, a, layer, seq, kh, jbase);
+        }
+        grid_barrier(c, a.fb);
+    }
+    const int items = batch * Hkv * nvc * nsplit;
     for (int it = c.cta; it < items; it += c.ncta) {
-        const int split = it % nsplit, sh = it / nsplit, h = sh % H, seq = sh / H;
-        if (c.n_rows[seq] == 0) continue;
-        if (a.m.hd == 64) attention_item<64>(c, a, layer, seq, h, split, nsplit);
-        else attention_item<128>(c, a, layer, seq, h, split, nsplit);
+        const int split = it % nsplit, r1 = it / nsplit, vc = r1 % nvc, r2 = r1 / nvc, kh = r2 % Hkv, seq = r2 / Hkv;
+        if (c.n_rows[seq] == 0 || 32 * vc >= group * c.n_rows[seq]) continue;
+        if (wide) {
+            if (a.m.hd == 64) attention_item<64, true, true>(c, a, layer, seq, kh, vc, split, nsplit);
+            else attention_item<128, true, true>(c, a, layer, seq, kh, vc, split, nsplit);
+        } else if (group == 1) {
+            if (a.m.hd == 64) attention_item<64, false, false>(c, a, layer, seq, kh, vc, split, nsplit);
+            else attention_item<128, false, false>(c, a, layer, seq, kh, vc, split, nsplit);
+        } else {
+            if (a.m.hd == 64) attention_item<64, true, false>(c, a, layer, seq, kh, vc, split, nsplit);
+            else attention_item<128, true, false>(c, a, layer, seq, kh, vc, split, nsplit);
+        }
     }
 }
 

@@ -201,42 +201,42 @@ __device__ __forceinline__ void epi_partial(Ctx &c, const Args &a, const GemmOp 
 template <int NT, bool BIG>
 __device__ __forceinline__ void phase_residual(Ctx &c, const Args &a, const GemmOp &op, const bf16 *gain_next) {
     const XLay xl{NT, NT <= 4 ? 1 : a.g.G};    // (at most 32 rows: one group, known at compile time)
-    // rows go 32 at a time (the narrow forwards have fewer, known at compile time: all their loads fly together)
-    constexpr int NIT = BIG ? 16 : NT * 4;
-    const int dm = a.m.cfg.d_model, ntiles = dm >> 4, rpad = BIG ? a.g.rpad : NT * 8;
+    // A task is one 16-column tile x RT rows: a warp's loads (rows x slices) all fly together and must fit its
+    // registers (up to 24 rows they do at once; beyond, 16 rows per task also give every warp of the grid work).
+    constexpr int RT = (NT <= 3 && !BIG) ? NT * 8 : 16, NIT = RT / 2;
+    const int dm = a.m.cfg.d_model, ntiles = dm >> 4, rpad = BIG ? a.g.rpad : NT * 8, nrc = (rpad + RT - 1) / RT;
     const int half = c.lane >> 4, col16 = c.lane & 15;
-    for (int tile = c.cta * MMA_WARPS + c.warp; tile < ntiles; tile += c.ncta * MMA_WARPS) {
+    for (int task = c.cta * MMA_WARPS + c.warp; task < ntiles * nrc; task += c.ncta * MMA_WARPS) {
+        const int tile = task / nrc, rc = (task - tile * nrc) * RT;
         const int col = tile * 16 + col16;
         const float gain = __bfloat162float(gain_next[col]);
-        for (int rc = 0; rc < rpad; rc += 2 * NIT) {
-            float v[NIT];
+        float v[NIT];
 #pragma unroll
-            for (int it = 0; it < NIT; ++it)
-                v[it] = (!BIG || rc + 2 * it < rpad) ? __ldcg(a.d.xres + (size_t)(rc + 2 * it + half) * dm + col) : 0.f;
-            for (int s0 = 0; s0 < op.S; s0 += 4) {          // four slices' loads in flight together
-                float p[4][NIT];
+        for (int it = 0; it < NIT; ++it)
+            v[it] = rc + 2 * it < rpad ? __ldcg(a.d.xres + (size_t)(rc + 2 * it + half) * dm + col) : 0.f;
+        for (int s0 = 0; s0 < op.S; s0 += 4) {          // four slices' loads in flight together
+            float p[4][NIT];
 #pragma unroll
-                for (int ds = 0; ds < 4; ++ds)
+            for (int ds = 0; ds < 4; ++ds)
 #pragma unroll
-                    for (int it = 0; it < NIT; ++it)
-                        p[ds][it] = (s0 + ds < op.S && (!BIG || rc + 2 * it < rpad))
-                            ? __ldcg(a.fb.part + (((size_t)(s0 + ds) * op.MT + tile) * rpad + rc + 2 * it + half) * 16 + col16) : 0.f;
+                for (int it = 0; it < NIT; ++it)
+                    p[ds][it] = (s0 + ds < op.S && rc + 2 * it < rpad)
+                        ? __ldcg(a.fb.part + (((size_t)(s0 + ds) * op.MT + tile) * rpad + rc + 2 * it + half) * 16 + col16) : 0.f;
 #pragma unroll
-                for (int ds = 0; ds < 4; ++ds)              // slice order: the sum does not depend on timing
+            for (int ds = 0; ds < 4; ++ds)              // slice order: the sum does not depend on timing
 #pragma unroll
-                    for (int it = 0; it < NIT; ++it) v[it] += p[ds][it];
-            }
+                for (int it = 0; it < NIT; ++it) v[it] += p[ds][it];
+        }
 #pragma unroll
-            for (int it = 0; it < NIT; ++it) {
-                if (BIG && rc + 2 * it >= rpad) break;
-                const int r = rc + 2 * it + half;
-                a.d.xres[(size_t)r * dm + col] = v[it];
-                store_split(a.fb.xg, xl, r, col, v[it] * gain);
-                float ss = v[it] * v[it];
+        for (int it = 0; it < NIT; ++it) {
+            if (rc + 2 * it >= rpad) break;
+            const int r = rc + 2 * it + half;
+            a.d.xres[(size_t)r * dm + col] = v[it];
+            store_split(a.fb.xg, xl, r, col, v[it] * gain);
+            float ss = v[it] * v[it];
 #pragma unroll
-                for (int o = 8; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-                if (col16 == 0) a.fb.ssq[tile * MAX_ROWS + r] = ss;
-            }
+            for (int o = 8; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+            if (col16 == 0) a.fb.ssq[tile * MAX_ROWS + r] = ss;
         }
     }
 }

@@ -24,7 +24,7 @@ struct pacer_ctx {
     size_t ws_bytes;
     DevPtrs d;
     ModelDev model[3];
-    Geom g_draft, g_mb, g_verify, g_ar;
+    Geom g_draft, g_mb, g_verify, g_ar, g_prefill;
     fwd::FwdBufs fb;
     int ncta;                  // blocks of the forward kernel (one per SM)
     std::map<int, fwd::Plan> plans;   // key: which * 2 + has_head
@@ -34,6 +34,12 @@ struct pacer_ctx {
     int prefilled;
     int64_t launches;
     cudaEvent_t ev[4];
+    // one draft-and-verify step of Algorithm 1 (every draft forward and pre-verification call of the window, the
+    // verify forward, the acceptance) captured once as a CUDA graph and replayed per step: the launches of a step
+    // never change, all that differs from step to step lives in the device-side state.  Key: window, mode, batch.
+    struct StepGraph { cudaGraph_t graph; cudaGraphExec_t exec; int64_t launches; };   // exec == NULL: seen once, not captured yet
+    std::map<int64_t, StepGraph> step_graphs;
+    int use_graphs;
     int32_t *fin_host;         // pinned: finished flags of the sequences, one row per step in flight
     cudaEvent_t fin_ev[8];
     std::vector<float2> rope_host[3];
@@ -163,7 +169,7 @@ static Layout make_layout(const pacer_cfg &c) {
     const pacer_model_cfg *ms[3] = {&c.target, &c.draft, &mb};
     const int B = c.max_batch, gc = c.gamma_cap, V = c.target.vocab;
     const int rps_max = gc + 1 > c.block_b + 1 ? gc + 1 : c.block_b + 1;
-    L.rtot_max = B * rps_max;
+    L.rtot_max = std::max(B * rps_max, B * std::max(gc + 1, 128 / B));      // verify rows, prompt-chunk rows
     L.nt_max = (L.rtot_max + 7) / 8;
     const size_t RP = std::min<size_t>(fwd::MAX_ROWS, make_geom(1, std::max(L.rtot_max, 32)).rpad);   // padded rows of the widest forward
     L.max_steps = c.max_ctx;
@@ -245,6 +251,8 @@ static void set_geoms(pacer_ctx *c, int batch, int draft_rows = 2) {
     c->g_mb = make_geom(batch, c->cfg.block_b + 1);
     c->g_verify = make_geom(batch, c->cfg.gamma_cap + 1);
     c->g_ar = make_geom(batch, 1);
+    // prompt chunks: as many rows per sequence as keep the forward at 128 rows (two full row groups)
+    c->g_prefill = make_geom(batch, std::max(c->cfg.gamma_cap + 1, 128 / batch));
 }
 
 extern "C" int pacer_create(const pacer_cfg *cfg, void *dev_workspace, size_t workspace_bytes, void *cuda_stream,
@@ -263,6 +271,9 @@ extern "C" int pacer_create(const pacer_cfg *cfg, void *dev_workspace, size_t wo
     c->ws_bytes = workspace_bytes;
     c->prefilled = 0;
     c->launches = 0;
+    c->use_graphs = 1;
+    if (const char *e = getenv("PACER_NO_GRAPH")) c->use_graphs = atoi(e) ? 0 : 1;
+    if (c->stream == nullptr || c->stream == cudaStreamLegacy) c->use_graphs = 0;   // the legacy default stream cannot be captured
     c->prof_on = 0;
     c->prof_used = 0;
     c->prof_bytes = 0;
@@ -350,6 +361,8 @@ extern "C" int pacer_destroy(pacer_ctx *c) {
     cudaStreamSynchronize(c->stream);
     for (int i = 0; i < 4; ++i) cudaEventDestroy(c->ev[i]);
     for (int i = 0; i < 8; ++i) cudaEventDestroy(c->fin_ev[i]);
+    for (auto &kv : c->step_graphs)
+        if (kv.second.exec) { cudaGraphExecDestroy(kv.second.exec); cudaGraphDestroy(kv.second.graph); }
     if (c->fin_host) cudaFreeHost(c->fin_host);
     for (cudaEvent_t e : c->prof_ev) cudaEventDestroy(e);
     delete c;
@@ -431,6 +444,9 @@ extern "C" int pacer_load_weights(pacer_ctx *c, int which, const pacer_tensor *t
     m.succ = isB ? nullptr : succ;
     m.loaded = 1;
     c->plans.clear();
+    for (auto &kv : c->step_graphs)
+        if (kv.second.exec) { cudaGraphExecDestroy(kv.second.exec); cudaGraphDestroy(kv.second.graph); }
+    c->step_graphs.clear();                    // captured launches carry the old weight pointers
     return PACER_OK;
 }
 
@@ -532,7 +548,7 @@ static int start_run(pacer_ctx *c, const int32_t *prompt, int batch, int n_promp
 }
 
 static int prefill_models(pacer_ctx *c, int n_prompt, bool target, bool draft_and_mb, bool mb = true) {
-    const Geom &g = c->g_verify;
+    const Geom &g = c->g_prefill;
     for (int c0 = 0; c0 < n_prompt - 1; c0 += g.rps) {
         int rc;
         if (target) {
@@ -682,6 +698,36 @@ static int enqueue_step(pacer_ctx *c, int gamma_max) {
     return enqueue_verify_accept(c);
 }
 
+// One step of Algorithm 1 as a graph launch (captured on first use).  Falls back to plain launches while the
+// per-launch profiling is on (its event records must stay outside a graph).
+static int launch_step(pacer_ctx *c, int gamma_max) {
+    if (!c->use_graphs || c->prof_on) return enqueue_step(c, gamma_max);
+    const int64_t key = ((int64_t)gamma_max * 4 + c->mode) * 256 + c->batch;
+    auto it = c->step_graphs.find(key);
+    if (it == c->step_graphs.end()) {
+        // the first step of a kind runs as plain launches (they set the kernels' shared-memory attributes, which
+        // must not happen inside a capture); the second one is captured
+        c->step_graphs.emplace(key, pacer_ctx::StepGraph{});
+        return enqueue_step(c, gamma_max);
+    }
+    if (!it->second.exec) {
+        pacer_ctx::StepGraph sg{};
+        const int64_t before = c->launches;
+        CK(cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal));
+        const int rc = enqueue_step(c, gamma_max);
+        cudaError_t e = cudaStreamEndCapture(c->stream, &sg.graph);
+        sg.launches = c->launches - before;
+        c->launches = before;
+        if (rc) { if (e == cudaSuccess && sg.graph) cudaGraphDestroy(sg.graph); return rc; }
+        CK(e);
+        CK(cudaGraphInstantiate(&sg.exec, sg.graph, 0));
+        it->second = sg;
+    }
+    CK(cudaGraphLaunch(it->second.exec, c->stream));
+    c->launches += it->second.launches;
+    return PACER_OK;
+}
+
 // Enqueues steps until every sequence is finished.  The end of generation is decided on the device; the host only
 // learns of it, without ever waiting for the step it has just enqueued: after each step the finished flags are
 // copied to pinned memory behind an event, and the host looks at the flags of the step it enqueued RUN_AHEAD steps
@@ -752,7 +798,7 @@ extern "C" int pacer_generate(pacer_ctx *c, const int32_t *prompt, int batch, in
     CK(cudaEventRecord(c->ev[1], c->stream));
     const int64_t launches0 = c->launches;
     const int gm = gamma_max / c->cfg.block_b * c->cfg.block_b;
-    if ((rc = run_steps(c, batch, max_new, [&](int) { return enqueue_step(c, gm); }))) return rc;
+    if ((rc = run_steps(c, batch, max_new, [&](int) { return launch_step(c, gm); }))) return rc;
     CK(cudaEventRecord(c->ev[2], c->stream));
     return collect(c, batch, max_new, n_prompt, out_tokens, out_n_steps, out_draft_len, out_accept_len, stats, launches0);
 }
