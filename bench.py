@@ -266,6 +266,9 @@ def main():
                     help="synthetic pair (default: the largest single-GPU batch-1 configuration)")
     ap.add_argument("--impl", default="pacer", choices=["pacer", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-baselines", action="store_true",
+                    help="only the timed Pacer runs and the verify-forward timing: no autoregressive / fixed-window / "
+                         "optimal-window runs (the short command the ncu launch list is taken on)")
     ap.add_argument("--cpu-sample-steps", type=int, default=1,
                     help="draft-and-verify steps of Algorithm 1 the CPU oracle is timed on")
     ap.add_argument("--preverify", default="trained", choices=["trained", "random"],
@@ -400,6 +403,19 @@ def main():
     barrier()
     wall = time.perf_counter() - wall0
     clocks = sampler.stop()
+
+    if args.no_baselines:
+        vf = verify_forward_numbers(ctx, cfg, prompt, 3, 1)
+        value, e2e_val, ms_step = aggregate_replicas(dec_ms, e2e_s, tok, args.steps, world, dev)
+        if rank == 0:
+            print(json.dumps({"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+                              "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+                              "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": workload,
+                              "clocks": clocks, "gpu_launches": int(launches),
+                              "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": int(prompt.nbytes),
+                                      "d2h_bytes_per_step": int(4 * cfg.max_new * 3 + 4 + 128)},
+                              "roofline": vf["roofline"], "verify_forward": vf["verify_forward"]}))
+        return
 
     # baselines on the same kernels (outside the timed region): autoregressive and fixed windows
     ar_tok, ar_st = ctx.pacer_generate_ar(prompt, cfg.max_new, mode, seed)

@@ -212,7 +212,8 @@ static Layout make_layout(const pacer_cfg &c) {
     L.xg = cv.take(sizeof(bf16) * 2 * RP * d_max);
     L.ssq = cv.take(sizeof(float) * fwd::MAX_ROWS * (d_max / 16 + 1));
     L.tile_top = cv.take(sizeof(float) * 4 * fwd::MAX_ROWS * ((size_t)V / 16 + 1));
-    L.attp = cv.take(sizeof(float) * (size_t)B * h_max * fwd::MAX_SPLIT * rps_max * (hd_max + 2));
+    const int rps_all = std::max(rps_max, std::max(gc + 1, 128 / B));          // rows per sequence: verify, M_B, prompt chunks
+    L.attp = cv.take(sizeof(float) * (size_t)B * h_max * fwd::MAX_SPLIT * rps_all * (hd_max + 2));
     L.part_bytes = sizeof(float) * 8 * (size_t)(d_max + 16) * RP;         // up to 8 k slices of [d/16][padded rows][16]
     L.part = cv.take(L.part_bytes);
     for (int i = 0; i < 3; ++i) {
