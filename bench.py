@@ -274,7 +274,9 @@ def main():
     ap.add_argument("--preverify", default="trained", choices=["trained", "random"],
                     help="trained: the pre-verification layer is trained on this box before the timed region, with the "
                          "paper's label recipe on the synthetic pair (untimed set-up, about a minute); random: N(0,0.02) weights")
-    ap.add_argument("--train-prompts", type=int, default=1024)
+    ap.add_argument("--train-prompts", type=int, default=0,
+                    help="prompts the pre-verification layer is trained on (default: 1024, or 256 for targets above "
+                         "10 B parameters, whose responses take longer to generate)")
     ap.add_argument("--t0", type=float, default=None,
                     help="initial threshold of the Pacer row (default: the best of {0.3, 0.5, 0.7} in an untimed pre-sweep "
                          "with a trained layer, 0.5 with a random one)")
@@ -340,7 +342,8 @@ def main():
         # Section 3.3: the target's responses to seeded random prompts, drafts from every prefix, labels up to the
         # first mismatch, cross-entropy, AdamW.  Plain PyTorch, outside the decoding path and outside the timed region.
         from paper_2602_01274_b200 import train_preverify
-        tensors, train_report = train_preverify.train(cfg, pair, dev, n_prompts=args.train_prompts, epochs=12, lr=1e-3,
+        n_train = args.train_prompts or (1024 if cfg.target.n_params() < 10e9 else 256)
+        tensors, train_report = train_preverify.train(cfg, pair, dev, n_prompts=n_train, epochs=12, lr=1e-3,
                                                       batch_prompts=64 if cfg.draft.n_params() < 5e8 else 32,
                                                       log=lambda m: print(m, file=sys.stderr, flush=True))
         pair["preverify"] = {k: v.to(dev) for k, v in tensors.items()}

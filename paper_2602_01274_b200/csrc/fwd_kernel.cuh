@@ -405,9 +405,10 @@ static inline Plan make_plan(const ModelDev &m, const DevPtrs &d, const FwdBufs 
             const int nks = K / (8 * KB);                    // a slice keeps at least 512 columns
             for (int sdiv = 2; sdiv <= 4; ++sdiv)
                 if (ncta % sdiv == 0 && sdiv <= nks && (MT + ncta / sdiv - 1) / (ncta / sdiv) <= MMA_TILES) o.S = sdiv;
-        } else if (i == OP_DOWN && K >= 32 * KB && MT < ncta && ncta % 4 == 0) {
-            // a small model's down projection: one or two tiles per block over a long k range is a chain of
-            // K / 64 stages of 0.3 - 0.4 us each, longer than the reduction pass that four k slices cost
+        } else if (((i == OP_DOWN && K >= 32 * KB) || (i == OP_O && K >= 24 * KB)) && MT < ncta && ncta % 4 == 0) {
+            // a small model's down (or attention-output) projection: one or two tiles per block over a long k
+            // range is a chain of K / 64 stages of 0.3 - 0.4 us each, longer than the reduction pass that four
+            // k slices cost
             o.S = 4;
         }
         o.rot = rot;
