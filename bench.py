@@ -308,6 +308,7 @@ def main():
         if rank != 0:
             return
         dev = "cuda:0" if torch.cuda.is_available() else "cpu"
+        workload["preverify"] = "random N(0,0.02) weights (the cost of a step does not depend on them)"
         pair = pair_to_cpu(synth.make_pair(cfg, seed=0, device=dev))
         prompt = synth.make_prompts(cfg.target.vocab, 1, cfg.n_prompt, seed=0)[0].numpy()
         vals = []

@@ -289,7 +289,10 @@ int pacer_linear(const void *x, const void *w, float *y, int rows, int N, int K,
  *   - All calls on one device share the one array, which keeps whatever the last
  *     call left in it.  Nothing in it has to start at zero: the kernels overwrite
  *     every element they later read.  Two calls that overlap on the GPU (different
- *     streams, no ordering between them) race on the array; order them. */
+ *     streams, no ordering between them) race on the array; order them.
+ *   - Host threads: the per-device address table is filled without a lock, so the first
+ *     calls on a device must not come from two host threads at once; later calls only
+ *     read it. */
 #define PACER_LINEAR_STATIC_BYTES (4u << 20)
 int pacer_linear_static(const void *x, const void *w, float *y, int rows, int N, int K, void *cuda_stream);
 

@@ -41,7 +41,7 @@ constexpr int X_PRODUCER = 12, X_PRODUCERS = 4;  // warps 12..14 provide the act
 constexpr int THREADS = 32 * (X_PRODUCER + X_PRODUCERS);
 constexpr int KB = 64;                          // k columns of a weight stage: one 128-byte swizzle row
 constexpr int NB = 16;                          // weight stages that can be in flight (barrier pairs)
-constexpr int RING_BYTES = 132 * 1024;          // weight ring of the forwards with at most 32 rows (a stage takes 128 B per
+constexpr int RING_BYTES = 134 * 1024;          // weight ring of the forwards with at most 32 rows (a stage takes 128 B per
                                                 // weight row of the block); wider forwards give part of it to the activations
 constexpr int XS_MAX = 3;                       // activation stages: as many as fit, at most 3 (one producer warp each)
 constexpr int XK = 256;                         // k columns of one activation stage (four k blocks)
@@ -50,14 +50,14 @@ __host__ __device__ constexpr int xstage_bytes(int NT) { return (XK / KB) * 2 * 
 __host__ __device__ constexpr int x_stages(int NT) { return (80 * 1024) / xstage_bytes(NT) < XS_MAX ? (80 * 1024) / xstage_bytes(NT) : XS_MAX; }
 constexpr int SCRATCH_BYTES = 88 * 1024;        // the activation ring lives in its first 72 KB at most; the epilogues' copy
                                                 // of the accumulator, the attention phase and the tails use all of it
-constexpr int MISC_BYTES = 6144;
+constexpr int MISC_BYTES = 5120;
 constexpr int SMEM_BYTES = SCRATCH_BYTES + RING_BYTES + MISC_BYTES;    // the same total for every forward
-static_assert(SMEM_BYTES <= 227 * 1024, "more shared memory than a block can have");
+static_assert(SMEM_BYTES <= 227 * 1024, "more shared memory than a block can have");   // (it is exactly that)
 constexpr int MMA_TILES = 16;                   // 16-row tiles one tcgen05.mma covers (N = 256)
 constexpr int MAX_TILES = 2 * MMA_TILES;        // tiles of one pass of a block: two accumulators, two MMAs per 16 k columns
                                                 // (a block that has one tile too many for N = 256 still reads the activations once)
 constexpr int ACC_COLS = 256;                   // fp32 accumulator columns of one accumulator (one per weight row)
-constexpr int MAX_ROWS = 192;                   // rows of one forward (all sequences together): three groups of 64
+constexpr int MAX_ROWS = 144;                   // rows of one forward (all sequences together): three groups of 48
 constexpr int MAX_SEQ = 32;                     // sequences of one forward
 constexpr int BIG_XBYTES = 144 * 1024;          // activation ring of a forward with more than 32 rows, at most
 constexpr int MAX_SPLIT = 16;                   // key-range splits of one attention head

@@ -153,7 +153,8 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 // order (one warp, lane = row; four running sums keep the loads independent).
 __device__ __forceinline__ void compute_inv(Ctx &c, const FwdBufs &fb, int dm, float eps, int row0 = 0) {
     const int ntiles = dm >> 4;
-    const float *p = fb.ssq + row0 + c.lane;
+    const bool in = row0 + c.lane < MAX_ROWS;            // (the last 32-row round of a wide forward is partial)
+    const float *p = fb.ssq + (in ? row0 + c.lane : 0);
     float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
     int t = 0;
     for (; t + 4 <= ntiles; t += 4) {
@@ -163,7 +164,7 @@ __device__ __forceinline__ void compute_inv(Ctx &c, const FwdBufs &fb, int dm, f
         s3 += __ldcg(p + (t + 3) * MAX_ROWS);
     }
     for (; t < ntiles; ++t) s0 += __ldcg(p + t * MAX_ROWS);
-    c.inv_rms[row0 + c.lane] = rsqrtf(((s0 + s1) + (s2 + s3)) / (float)dm + eps);
+    if (in) c.inv_rms[row0 + c.lane] = rsqrtf(((s0 + s1) + (s2 + s3)) / (float)dm + eps);
     __syncwarp();
 }
 

@@ -126,8 +126,7 @@ static Geom make_geom(int batch, int rps) {
     else if (r <= 64) { g.nt = 8; g.G = 1; }
     else if (r <= 96) { g.nt = 6; g.G = 2; }
     else if (r <= 128) { g.nt = 8; g.G = 2; }
-    else if (r <= 144) { g.nt = 6; g.G = 3; }
-    else { g.nt = 8; g.G = 3; }
+    else { g.nt = 6; g.G = 3; }                 // up to 144 rows, the most a forward takes
     g.rpad = g.G * g.nt * 8;
     return g;
 }
